@@ -1,0 +1,170 @@
+/*
+ * peak_gemm.h -- C ABI of the B200 (sm_100a) dense GEMM library.
+ *
+ * The operation is the matrix multiplication the PEAK paper optimises
+ * (section 2.2, "Matrix Multiplication": A is m x k, B is k x n, C = A x B,
+ * all matrices row-major, elements stored as fp32 or fp16), widened to the
+ * BLAS form
+ *
+ *     C = alpha * op(A) * op(B) + beta * C
+ *
+ * over ROW-MAJOR storage.  alpha, beta, op(), leading dimensions and bfloat16
+ * are additions with the reference-BLAS meaning; the paper has C = A x B only.
+ *
+ * Layout.  op(A) is M x K, op(B) is K x N, C is M x N.
+ *     transA == 0 : A is stored M x K,  op(A)(i,k) = A[i*lda + k],  lda >= K
+ *     transA == 1 : A is stored K x M,  op(A)(i,k) = A[k*lda + i],  lda >= M
+ *     transB == 0 : B is stored K x N,  op(B)(k,j) = B[k*ldb + j],  ldb >= N
+ *     transB == 1 : B is stored N x K,  op(B)(k,j) = B[j*ldb + k],  ldb >= K
+ *     C(i,j) = C[i*ldc + j],  ldc >= N
+ * Leading dimensions count elements, not bytes.  "NT" therefore means weights
+ * stored N x K (the usual linear-layer layout), "TN" means A stored K x M.
+ *
+ * Arithmetic.  Products of the stored values are accumulated in fp32 (tensor
+ * cores with fp32 accumulators for 16-bit inputs; fp32 FMA on the CUDA cores,
+ * never TF32, for fp32 inputs), in an unspecified order.  The epilogue forms
+ * alpha*acc (+ beta*C_old when beta != 0) in fp32 and rounds once, to nearest
+ * even, to the output type.
+ *
+ * Ownership and asynchrony.  Unless stated otherwise A, B, C are DEVICE
+ * pointers owned by the caller; the call enqueues work on `stream` (a
+ * cudaStream_t passed as void*, NULL = the default stream) and returns without
+ * synchronising.  C must not overlap A or B.  C is read only when beta != 0.
+ *
+ * Quick returns (reference-BLAS convention; the paper is silent):
+ *     M == 0 or N == 0        -> nothing is touched
+ *     K == 0 or alpha == 0    -> C = beta*C; A and B are not read
+ *     beta == 0               -> C is not read (NaN in it does not propagate)
+ *     alpha == 0 and beta == 1-> C is left bit-for-bit unchanged
+ *
+ * Errors.  Every entry point returns PEAK_OK or a positive peak_status_t.
+ * Arguments are validated before anything is launched; on an error nothing is
+ * written.  No entry point throws or aborts.
+ */
+#ifndef PEAK_GEMM_H
+#define PEAK_GEMM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* (input, output) storage types.  Accumulation is always fp32. */
+typedef enum peak_dtype {
+    PEAK_F16_F32 = 0,   /* A, B binary16; C binary32 */
+    PEAK_BF16_BF16 = 1, /* A, B bfloat16; C bfloat16 */
+    PEAK_F32_F32 = 2,   /* A, B, C binary32 (CUDA-core SGEMM, no TF32) */
+    PEAK_F16_F16 = 3,   /* A, B, C binary16 */
+    PEAK_BF16_F32 = 4   /* A, B bfloat16; C binary32 */
+} peak_dtype_t;
+
+typedef enum peak_status {
+    PEAK_OK = 0,
+    PEAK_ERR_INVALID_VALUE = 1, /* unknown dtype / trans, negative size, ld too small, null pointer */
+    PEAK_ERR_ARCH = 2,          /* the current device is not compute capability 10.x */
+    PEAK_ERR_CUDA = 3,          /* a CUDA runtime / driver call failed; see peak_last_cuda_error() */
+    PEAK_ERR_UNSUPPORTED = 4,   /* the forced variant cannot run this problem */
+    PEAK_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up; reported by peak_check() */
+    PEAK_ERR_NO_MEMORY = 6      /* staging memory for the host-buffer call could not be allocated */
+} peak_status_t;
+
+/* Kernel families.  PEAK_VARIANT_AUTO lets the dispatcher choose. */
+typedef enum peak_variant {
+    PEAK_VARIANT_AUTO = 0,
+    PEAK_VARIANT_FALLBACK = 1, /* plain tiled CUDA-core kernel: any dtype, layout, alignment (the paper's naive
+                                  kernel of section 2.2 with thread-block tiling) */
+    PEAK_VARIANT_UMMA_1CTA = 2, /* tcgen05.mma, 128x256 tile per CTA, TMA ring, persistent (16-bit inputs) */
+    PEAK_VARIANT_UMMA_2CTA = 3, /* tcgen05.mma cta_group::2, 256x256 tile per CTA pair (16-bit inputs) */
+    PEAK_VARIANT_SGEMM = 4,     /* register-tiled fp32 FMA kernel (fp32 inputs) */
+    PEAK_VARIANT_SCALE = 5,     /* C = beta*C only (K == 0 or alpha == 0) */
+    PEAK_VARIANT_NONE = 6       /* nothing to do (M == 0 or N == 0, or alpha == 0 and beta == 1) */
+} peak_variant_t;
+
+/*
+ * peak_gemm: C = alpha*op(A)*op(B) + beta*C on the current device (paper section 2.2, widened as above).
+ *   dtype          a peak_dtype_t
+ *   transA/transB  0 or 1, meaning as in the layout table above
+ *   M, N, K        >= 0
+ *   alpha, beta    host fp32 scalars, by value
+ *   A, B, C        device pointers (may be NULL only where the matrix is empty or not read)
+ *   lda, ldb, ldc  row pitches in elements
+ *   stream         cudaStream_t
+ * The fastest variant whose preconditions hold is chosen: the tensor-core path needs 16-byte aligned
+ * base pointers and row pitches that are multiples of 16 bytes; anything else runs on the fallback
+ * kernel with the same result contract.  Returns after enqueueing; never synchronises.
+ */
+int peak_gemm(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+              int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream);
+
+/*
+ * peak_gemm_variant: as peak_gemm, but runs the named kernel family (a peak_variant_t) or fails with
+ * PEAK_ERR_UNSUPPORTED when that family cannot run the problem.  Quick returns still apply.  For tests,
+ * A/B measurements and tuning (the paper's "tuning parameters", section 3.1).
+ */
+int peak_gemm_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                      const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc,
+                      void *stream);
+
+/*
+ * peak_gemm_host: the same operation on HOST buffers (the paper's "driver", section 3.1: allocate,
+ * copy in, run, copy out).  A, B, C are host pointers (pinned memory makes the copies faster but is
+ * not required).  Copies A and B (and C when beta != 0) to device staging buffers, runs peak_gemm,
+ * copies C back, and synchronises `stream` before returning.  The staging buffers are owned by the
+ * library, grow on demand and are reused by later calls; peak_release_staging() frees them.
+ * Not thread-safe with respect to other peak_gemm_host calls.
+ */
+int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+                   int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream);
+int peak_release_staging(void);
+
+/*
+ * peak_gemm_xcheck_f64: cross-check kernel.  Writes the UNROUNDED fp64 value
+ *     alpha * sum_k op(A)(i,k)*op(B)(k,j) + beta * C0(i,j)       (fp64 accumulation, k ascending)
+ * to Cref[i*ldcref + j] (device pointer, double).  C0 (device, output type of `dtype`) is read only when
+ * beta != 0 and is never written.  One thread per output element, as in the paper's naive kernel
+ * (section 2.2); slow, meant for full-matrix verification at sizes the CPU cannot cover.
+ */
+int peak_gemm_xcheck_f64(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                         const void *A, int64_t lda, const void *B, int64_t ldb, float beta, const void *C0,
+                         int64_t ldc, double *Cref, int64_t ldcref, void *stream);
+
+/*
+ * peak_query_variant: which kernel family peak_gemm would run for these arguments (a peak_variant_t),
+ * or a negative peak_status_t when they are invalid.  Pure host logic: touches no device.
+ */
+int peak_query_variant(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                       const void *A, int64_t lda, const void *B, int64_t ldb, float beta, const void *C,
+                       int64_t ldc);
+
+/*
+ * peak_tile_coord: the persistent scheduler's map from a linear tile index to tile coordinates
+ * (block swizzle of the paper's optimisation sequences, section 4.3): tiles are visited in groups of
+ * `group` tile-rows, walking down the rows of a group before moving to the next tile-column, so that
+ * CTAs running at the same time share A and B panels in L2.  Host copy of the device function, for
+ * tests.  Returns PEAK_ERR_INVALID_VALUE if tile is outside [0, tiles_m*tiles_n).
+ */
+int peak_tile_coord(int64_t tile, int64_t tiles_m, int64_t tiles_n, int64_t group, int64_t *tile_m,
+                    int64_t *tile_n);
+
+/*
+ * peak_check: synchronises `stream`, then reads and clears the device status word that kernels set
+ * when a bounded wait (on an mbarrier) gives up.  Returns PEAK_OK, PEAK_ERR_TIMEOUT or PEAK_ERR_CUDA.
+ * `detail`, if not NULL, receives the raw status word (role and barrier that gave up).
+ */
+int peak_check(void *stream, uint32_t *detail);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+int64_t peak_kernel_launches(void);
+
+/* The cudaError_t of the most recent failing CUDA call made by this thread's last entry-point call. */
+int peak_last_cuda_error(void);
+
+const char *peak_status_string(int status);
+const char *peak_variant_string(int variant);
+int peak_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PEAK_GEMM_H */

@@ -1,0 +1,279 @@
+// The C ABI: argument validation, quick returns, variant selection, the host-buffer entry point and the
+// small amount of process state (launch counter, last CUDA error, per-device status word, staging buffers).
+#include <atomic>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace peak {
+
+namespace {
+std::atomic<int64_t> g_launches{0};
+thread_local int t_last_cuda_error = 0;
+
+// One status word per device, living in the module's own global memory (no allocation).  Kernels OR
+// a code into it when a bounded wait gives up; peak_check() reads and clears it.
+__device__ uint32_t g_status_word[4];
+
+constexpr int kMaxDevices = 64;
+uint32_t *g_status_ptr[kMaxDevices] = {};
+std::mutex g_status_mutex;
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void set_cuda_error(cudaError_t e) { t_last_cuda_error = (int)e; }
+
+uint32_t *device_status_word() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    if (!g_status_ptr[dev]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_status_word);
+        if (e != cudaSuccess) { set_cuda_error(e); return nullptr; }
+        g_status_ptr[dev] = static_cast<uint32_t *>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+namespace {
+
+bool valid_dtype(int d) { return d >= PEAK_F16_F32 && d <= PEAK_BF16_F32; }
+
+// Returns PEAK_OK or PEAK_ERR_INVALID_VALUE; checks only the arguments, touches no device.
+int validate(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, const void *A, int64_t lda,
+             const void *B, int64_t ldb, float alpha, float beta, const void *C, int64_t ldc) {
+    if (!valid_dtype(dtype)) return PEAK_ERR_INVALID_VALUE;
+    if ((transA != 0 && transA != 1) || (transB != 0 && transB != 1)) return PEAK_ERR_INVALID_VALUE;
+    if (M < 0 || N < 0 || K < 0) return PEAK_ERR_INVALID_VALUE;
+    if (lda < 1 || ldb < 1 || ldc < 1) return PEAK_ERR_INVALID_VALUE;
+    if (lda < (transA ? M : K) || ldb < (transB ? K : N) || ldc < N) return PEAK_ERR_INVALID_VALUE;
+    if (M == 0 || N == 0) return PEAK_OK;
+    if (!C) return PEAK_ERR_INVALID_VALUE;
+    if (K > 0 && alpha != 0.0f && (!A || !B)) return PEAK_ERR_INVALID_VALUE;
+    (void)beta;
+    return PEAK_OK;
+}
+
+// The dispatcher's choice, as a peak_variant_t (arguments already validated).
+int choose_variant(const GemmArgs &g) {
+    if (g.M == 0 || g.N == 0) return PEAK_VARIANT_NONE;
+    if (g.K == 0 || g.alpha == 0.0f) return (g.beta == 1.0f) ? PEAK_VARIANT_NONE : PEAK_VARIANT_SCALE;
+    if (in_elem(g.dtype) == Elem::F32) return sgemm_supports(g) ? PEAK_VARIANT_SGEMM : PEAK_VARIANT_FALLBACK;
+    if (umma_supports(g, 1)) return PEAK_VARIANT_UMMA_1CTA;
+    return PEAK_VARIANT_FALLBACK;
+}
+
+int check_arch() {
+    static int result[kMaxDevices];
+    static bool init = false;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices) return PEAK_ERR_ARCH;
+    static std::mutex m;
+    std::lock_guard<std::mutex> lock(m);
+    if (!init) { for (int i = 0; i < kMaxDevices; ++i) result[i] = -1; init = true; }
+    if (result[dev] < 0) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+        result[dev] = (major == 10) ? PEAK_OK : PEAK_ERR_ARCH;
+    }
+    return result[dev];
+}
+
+int run_variant(int variant, const GemmArgs &g) {
+    switch (variant) {
+        case PEAK_VARIANT_NONE: return PEAK_OK;
+        case PEAK_VARIANT_SCALE: return launch_scale(g);
+        case PEAK_VARIANT_FALLBACK: return launch_fallback(g);
+        case PEAK_VARIANT_SGEMM: return launch_sgemm(g);
+        case PEAK_VARIANT_UMMA_1CTA: return launch_umma(g, 1);
+        case PEAK_VARIANT_UMMA_2CTA: return launch_umma(g, 2);
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
+int gemm_impl(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+              const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream) {
+    t_last_cuda_error = 0;
+    int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
+    if (rc != PEAK_OK) return rc;
+    if (variant < PEAK_VARIANT_AUTO || variant > PEAK_VARIANT_NONE) return PEAK_ERR_INVALID_VALUE;
+    GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, C, lda, ldb, ldc, (cudaStream_t)stream};
+    const int chosen = choose_variant(g);
+    int v = chosen;
+    if (variant != PEAK_VARIANT_AUTO && chosen != PEAK_VARIANT_NONE && chosen != PEAK_VARIANT_SCALE) {
+        if (variant == PEAK_VARIANT_NONE || variant == PEAK_VARIANT_SCALE) return PEAK_ERR_UNSUPPORTED;
+        v = variant;
+    }
+    if (v == PEAK_VARIANT_NONE) return PEAK_OK;
+    rc = check_arch();
+    if (rc != PEAK_OK) return rc;
+    return run_variant(v, g);
+}
+
+// ---- staging buffers for the host-buffer entry point ------------------------------------------------
+struct Staging {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+Staging g_stage[3];
+std::mutex g_stage_mutex;
+
+int ensure(Staging &s, size_t need) {
+    if (need <= s.bytes) return PEAK_OK;
+    if (s.ptr) { cudaFree(s.ptr); s.ptr = nullptr; s.bytes = 0; }
+    cudaError_t e = cudaMalloc(&s.ptr, need);
+    if (e != cudaSuccess) { set_cuda_error(e); s.ptr = nullptr; return PEAK_ERR_NO_MEMORY; }
+    s.bytes = need;
+    return PEAK_OK;
+}
+
+size_t span_bytes(int64_t rows, int64_t cols, int64_t ld, int eb) {
+    if (rows <= 0 || cols <= 0) return 0;
+    return (size_t)((rows - 1) * ld + cols) * (size_t)eb;
+}
+
+}  // namespace
+}  // namespace peak
+
+using namespace peak;
+
+extern "C" {
+
+int peak_gemm(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+              int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream) {
+    return gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, stream);
+}
+
+int peak_gemm_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                      const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc,
+                      void *stream) {
+    return gemm_impl(variant, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, stream);
+}
+
+int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+                   int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream) {
+    t_last_cuda_error = 0;
+    int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
+    if (rc != PEAK_OK) return rc;
+    if (M == 0 || N == 0) return PEAK_OK;
+    rc = check_arch();
+    if (rc != PEAK_OK) return rc;
+    const int ib = elem_bytes(in_elem(dtype)), ob = elem_bytes(out_elem(dtype));
+    const bool need_ab = (K > 0 && alpha != 0.0f);
+    const size_t a_bytes = need_ab ? span_bytes(transA ? K : M, transA ? M : K, lda, ib) : 0;
+    const size_t b_bytes = need_ab ? span_bytes(transB ? N : K, transB ? K : N, ldb, ib) : 0;
+    const size_t c_bytes = span_bytes(M, N, ldc, ob);
+    cudaStream_t st = (cudaStream_t)stream;
+    std::lock_guard<std::mutex> lock(g_stage_mutex);
+    if ((rc = ensure(g_stage[0], a_bytes)) || (rc = ensure(g_stage[1], b_bytes)) || (rc = ensure(g_stage[2], c_bytes)))
+        return rc;
+    cudaError_t e = cudaSuccess;
+    if (a_bytes) e = cudaMemcpyAsync(g_stage[0].ptr, A, a_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && b_bytes) e = cudaMemcpyAsync(g_stage[1].ptr, B, b_bytes, cudaMemcpyHostToDevice, st);
+    // C travels to the device when its old values are needed, or when the pitch leaves gaps that the
+    // copy back would otherwise overwrite with stale staging contents
+    if (e == cudaSuccess && (beta != 0.0f || ldc != N))
+        e = cudaMemcpyAsync(g_stage[2].ptr, C, c_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, g_stage[0].ptr, lda, g_stage[1].ptr, ldb,
+                   beta, g_stage[2].ptr, ldc, stream);
+    if (rc != PEAK_OK) return rc;
+    e = cudaMemcpyAsync(C, g_stage[2].ptr, c_bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+int peak_release_staging(void) {
+    std::lock_guard<std::mutex> lock(g_stage_mutex);
+    for (auto &s : g_stage) {
+        if (s.ptr) cudaFree(s.ptr);
+        s.ptr = nullptr;
+        s.bytes = 0;
+    }
+    return PEAK_OK;
+}
+
+int peak_gemm_xcheck_f64(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                         const void *A, int64_t lda, const void *B, int64_t ldb, float beta, const void *C0,
+                         int64_t ldc, double *Cref, int64_t ldcref, void *stream) {
+    t_last_cuda_error = 0;
+    int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, 1.0f, beta, Cref, ldc);
+    if (rc != PEAK_OK) return rc;
+    if (ldcref < N || (K > 0 && (!A || !B) && M > 0 && N > 0)) return PEAK_ERR_INVALID_VALUE;
+    if (beta != 0.0f && !C0 && M > 0 && N > 0) return PEAK_ERR_INVALID_VALUE;
+    if (M == 0 || N == 0) return PEAK_OK;
+    rc = check_arch();
+    if (rc != PEAK_OK) return rc;
+    GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, nullptr, lda, ldb, ldc, (cudaStream_t)stream};
+    return launch_xcheck_f64(g, C0, Cref, ldcref);
+}
+
+int peak_query_variant(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                       const void *A, int64_t lda, const void *B, int64_t ldb, float beta, const void *C,
+                       int64_t ldc) {
+    int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
+    if (rc != PEAK_OK) return -rc;
+    GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, const_cast<void *>(C), lda, ldb, ldc, nullptr};
+    return choose_variant(g);
+}
+
+int peak_tile_coord(int64_t tile, int64_t tiles_m, int64_t tiles_n, int64_t group, int64_t *tile_m,
+                    int64_t *tile_n) {
+    if (tiles_m < 1 || tiles_n < 1 || tile < 0 || tile >= tiles_m * tiles_n || !tile_m || !tile_n)
+        return PEAK_ERR_INVALID_VALUE;
+    tile_coord(tile, tiles_m, tiles_n, group, *tile_m, *tile_n);
+    return PEAK_OK;
+}
+
+int peak_check(void *stream, uint32_t *detail) {
+    t_last_cuda_error = 0;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    uint32_t *w = device_status_word();
+    if (!w) return PEAK_ERR_CUDA;
+    uint32_t host = 0, zero = 0;
+    e = cudaMemcpy(&host, w, sizeof(host), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && host != 0) e = cudaMemcpy(w, &zero, sizeof(zero), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (detail) *detail = host;
+    return (host & kStatusTimeout) ? PEAK_ERR_TIMEOUT : PEAK_OK;
+}
+
+int64_t peak_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int peak_last_cuda_error(void) { return t_last_cuda_error; }
+
+const char *peak_status_string(int status) {
+    switch (status) {
+        case PEAK_OK: return "ok";
+        case PEAK_ERR_INVALID_VALUE: return "invalid value";
+        case PEAK_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+        case PEAK_ERR_CUDA: return "CUDA call failed";
+        case PEAK_ERR_UNSUPPORTED: return "variant does not support this problem";
+        case PEAK_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case PEAK_ERR_NO_MEMORY: return "out of device memory for staging";
+    }
+    return "unknown status";
+}
+
+const char *peak_variant_string(int variant) {
+    switch (variant) {
+        case PEAK_VARIANT_AUTO: return "auto";
+        case PEAK_VARIANT_FALLBACK: return "fallback";
+        case PEAK_VARIANT_UMMA_1CTA: return "umma_1cta";
+        case PEAK_VARIANT_UMMA_2CTA: return "umma_2cta";
+        case PEAK_VARIANT_SGEMM: return "sgemm";
+        case PEAK_VARIANT_SCALE: return "scale";
+        case PEAK_VARIANT_NONE: return "none";
+    }
+    return "unknown variant";
+}
+
+int peak_version(void) { return 100; }
+
+}  // extern "C"

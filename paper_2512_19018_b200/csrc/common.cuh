@@ -1,0 +1,81 @@
+// Shared declarations of the CUDA library: storage types, epilogue arithmetic, launch bookkeeping.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/peak_gemm.h"
+
+namespace peak {
+
+// ---- storage types ---------------------------------------------------------------------------
+enum class Elem : int { F16 = 0, BF16 = 1, F32 = 2 };
+
+__host__ __device__ inline Elem in_elem(int dtype) {
+    return (dtype == PEAK_F16_F32 || dtype == PEAK_F16_F16) ? Elem::F16
+           : (dtype == PEAK_F32_F32)                       ? Elem::F32
+                                                           : Elem::BF16;
+}
+__host__ __device__ inline Elem out_elem(int dtype) {
+    return (dtype == PEAK_BF16_BF16) ? Elem::BF16 : (dtype == PEAK_F16_F16) ? Elem::F16 : Elem::F32;
+}
+__host__ __device__ inline int elem_bytes(Elem e) { return e == Elem::F32 ? 4 : 2; }
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// The epilogue's arithmetic, in one place: alpha*acc, plus beta*c_old only when beta != 0.
+__device__ __forceinline__ float epilogue_f32(float alpha, float acc, float beta, float c_old) {
+    float r = alpha * acc;
+    if (beta != 0.0f) r = fmaf(beta, c_old, r);
+    return r;
+}
+
+// ---- host-side bookkeeping (api.cu owns the definitions) ---------------------------------------
+void count_launch(int n = 1);
+void set_cuda_error(cudaError_t e);
+uint32_t *device_status_word();  // address of the per-device status word (nullptr on failure)
+
+struct GemmArgs {
+    int dtype, transA, transB;
+    int64_t M, N, K;
+    float alpha, beta;
+    const void *A, *B;
+    void *C;
+    int64_t lda, ldb, ldc;
+    cudaStream_t stream;
+};
+
+// kernel-family launchers; each returns a peak_status_t
+int launch_fallback(const GemmArgs &g);
+int launch_scale(const GemmArgs &g);
+int launch_xcheck_f64(const GemmArgs &g, const void *C0, double *Cref, int64_t ldcref);
+int launch_sgemm(const GemmArgs &g);
+bool sgemm_supports(const GemmArgs &g);
+int launch_umma(const GemmArgs &g, int cta_group);
+bool umma_supports(const GemmArgs &g, int cta_group);
+
+// status word layout: bit 31 = a bounded wait gave up; bits 0..7 = role, 8..15 = barrier index
+constexpr uint32_t kStatusTimeout = 0x80000000u;
+
+// Tile order of the persistent scheduler (also exported on the host as peak_tile_coord).
+__host__ __device__ inline void tile_coord(int64_t tile, int64_t tiles_m, int64_t tiles_n, int64_t group,
+                                           int64_t &tm, int64_t &tn) {
+    if (group < 1) group = 1;
+    const int64_t per_group = group * tiles_n;
+    const int64_t g = tile / per_group;
+    const int64_t first_m = g * group;
+    const int64_t rows = (tiles_m - first_m < group) ? (tiles_m - first_m) : group;
+    const int64_t r = tile - g * per_group;
+    tm = first_m + r % rows;
+    tn = r / rows;
+}
+
+}  // namespace peak

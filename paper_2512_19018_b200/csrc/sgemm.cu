@@ -1,0 +1,154 @@
+// fp32 GEMM on the CUDA cores (plain fp32 FMA; TF32 is never used).
+//
+// The structure follows the paper's CUDA-core sequence (sections 2.2 and 4.3): thread-block tiling
+// (128 x 128 x 16 tile staged in shared memory), thread tiling (8 x 8 outputs per thread held in
+// registers, operands cached in registers per k), vectorised float4 global and shared accesses,
+// register staging of the next k-block while the current one is multiplied (two shared-memory buffers),
+// a transposing store for the operand whose contiguous index is k, padding against bank conflicts, and a
+// grouped block order for L2 reuse.
+#include "common.cuh"
+
+namespace peak {
+namespace {
+
+constexpr int SG_BM = 128, SG_BN = 128, SG_BK = 16;
+constexpr int SG_THREADS = 256;
+constexpr int SG_PAD = 4;  // floats of padding per shared-memory row
+constexpr int SG_LD = SG_BM + SG_PAD;
+
+// Stage a (128 x 16) operand tile as S[k][mn].  KCONTIG: memory is [mn][k] (k contiguous), so the float4
+// read along k is scattered into four rows; otherwise memory is [k][mn] and the float4 is stored as is.
+template <bool KCONTIG> struct Loader {
+    const float *base;  // tile origin
+    int64_t pitch;
+    int r0, c0;  // this thread's first float4: KCONTIG: row mn=r0 (+64), k=c0 ; else: row k=r0 (+8), mn=c0
+    __device__ __forceinline__ Loader(const float *origin, int64_t pitch_, int tid) : base(origin), pitch(pitch_) {
+        if (KCONTIG) { r0 = tid / 4; c0 = (tid % 4) * 4; } else { r0 = tid / 32; c0 = (tid % 32) * 4; }
+    }
+    __device__ __forceinline__ void load(float4 (&g)[2], int64_t k0) const {
+        if (KCONTIG) {
+            g[0] = *reinterpret_cast<const float4 *>(base + (int64_t)r0 * pitch + k0 + c0);
+            g[1] = *reinterpret_cast<const float4 *>(base + (int64_t)(r0 + 64) * pitch + k0 + c0);
+        } else {
+            g[0] = *reinterpret_cast<const float4 *>(base + (k0 + r0) * pitch + c0);
+            g[1] = *reinterpret_cast<const float4 *>(base + (k0 + r0 + 8) * pitch + c0);
+        }
+    }
+    __device__ __forceinline__ void store(float (*S)[SG_LD], const float4 (&g)[2]) const {
+        if (KCONTIG) {
+            S[c0 + 0][r0] = g[0].x; S[c0 + 1][r0] = g[0].y; S[c0 + 2][r0] = g[0].z; S[c0 + 3][r0] = g[0].w;
+            S[c0 + 0][r0 + 64] = g[1].x; S[c0 + 1][r0 + 64] = g[1].y; S[c0 + 2][r0 + 64] = g[1].z; S[c0 + 3][r0 + 64] = g[1].w;
+        } else {
+            *reinterpret_cast<float4 *>(&S[r0][c0]) = g[0];
+            *reinterpret_cast<float4 *>(&S[r0 + 8][c0]) = g[1];
+        }
+    }
+};
+
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(SG_THREADS, 2)
+sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
+             int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int group) {
+    __shared__ __align__(16) float As[2][SG_BK][SG_LD];
+    __shared__ __align__(16) float Bs[2][SG_BK][SG_LD];
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    int64_t tm, tn;
+    tile_coord(blockIdx.x, tiles_m, tiles_n, group, tm, tn);
+    const int64_t m0 = tm * SG_BM, n0 = tn * SG_BN;
+
+    // A: not transposed -> stored [m][k] (k contiguous); transposed -> stored [k][m]
+    // B: not transposed -> stored [k][n];               transposed -> stored [n][k] (k contiguous)
+    Loader<!TA> la(TA ? A + m0 : A + m0 * lda, lda, tid);
+    Loader<TB> lb(TB ? B + n0 * ldb : B + n0, ldb, tid);
+
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+
+    float4 ga[2], gb[2];
+    la.load(ga, 0);
+    lb.load(gb, 0);
+    la.store(As[0], ga);
+    lb.store(Bs[0], gb);
+    __syncthreads();
+
+    const int nkb = K / SG_BK;
+    for (int kb = 0; kb < nkb; ++kb) {
+        const int cur = kb & 1;
+        if (kb + 1 < nkb) {  // register staging of the next k-block
+            la.load(ga, (int64_t)(kb + 1) * SG_BK);
+            lb.load(gb, (int64_t)(kb + 1) * SG_BK);
+        }
+#pragma unroll
+        for (int k = 0; k < SG_BK; ++k) {
+            float a[8], b[8];
+            *reinterpret_cast<float4 *>(&a[0]) = *reinterpret_cast<const float4 *>(&As[cur][k][ty * 4]);
+            *reinterpret_cast<float4 *>(&a[4]) = *reinterpret_cast<const float4 *>(&As[cur][k][ty * 4 + 64]);
+            *reinterpret_cast<float4 *>(&b[0]) = *reinterpret_cast<const float4 *>(&Bs[cur][k][tx * 4]);
+            *reinterpret_cast<float4 *>(&b[4]) = *reinterpret_cast<const float4 *>(&Bs[cur][k][tx * 4 + 64]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (kb + 1 < nkb) {
+            la.store(As[cur ^ 1], ga);
+            lb.store(Bs[cur ^ 1], gb);
+        }
+        __syncthreads();
+    }
+
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int64_t m = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float4 *dst = reinterpret_cast<float4 *>(C + m * ldc + n0 + tx * 4 + h * 64);
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (beta != 0.0f) o = *dst;
+            float4 r;
+            r.x = epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x);
+            r.y = epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y);
+            r.z = epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z);
+            r.w = epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w);
+            *dst = r;
+        }
+    }
+}
+
+template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
+    const int tiles_m = (int)(g.M / SG_BM), tiles_n = (int)(g.N / SG_BN);
+    sgemm_kernel<TA, TB><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
+        (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
+        (float *)g.C, g.ldc, tiles_m, tiles_n, 8);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+}  // namespace
+
+bool sgemm_supports(const GemmArgs &g) {
+    if (g.dtype != PEAK_F32_F32) return false;
+    if (g.M < SG_BM || g.N < SG_BN || g.K < SG_BK) return false;
+    if (g.M % SG_BM || g.N % SG_BN || g.K % SG_BK) return false;
+    if (g.M >= (1ll << 31) || g.N >= (1ll << 31) || g.K >= (1ll << 31)) return false;
+    if ((g.M / SG_BM) * (g.N / SG_BN) >= (1ll << 31)) return false;
+    if (g.lda % 4 || g.ldb % 4 || g.ldc % 4) return false;
+    if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16 ||
+        reinterpret_cast<uintptr_t>(g.C) % 16)
+        return false;
+    return true;
+}
+
+int launch_sgemm(const GemmArgs &g) {
+    if (!sgemm_supports(g)) return PEAK_ERR_UNSUPPORTED;
+    if (g.transA) return g.transB ? run_sgemm<true, true>(g) : run_sgemm<true, false>(g);
+    return g.transB ? run_sgemm<false, true>(g) : run_sgemm<false, false>(g);
+}
+
+}  // namespace peak

@@ -1,0 +1,210 @@
+"""GPU parity: every kernel family, called through the C ABI, against the CPU oracle on the same seeded
+inputs -- element by element, at sizes that span several tiles, several k-blocks and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_19018_b200 import binding as P
+from paper_2512_19018_b200 import workloads as W
+from tests import parity as R
+
+pytestmark = pytest.mark.gpu
+
+LAYOUTS = [(0, 0), (0, 1), (1, 0), (1, 1)]
+PAIRS_16 = [W.PEAK_F16_F32, W.PEAK_BF16_BF16, W.PEAK_F16_F16, W.PEAK_BF16_F32]
+UMMA = [P.PEAK_VARIANT_UMMA_1CTA, P.PEAK_VARIANT_UMMA_2CTA]
+
+
+def mk(dtype, ta, tb, M, N, K, **kw):
+    return W.GemmCase(f"t{dtype}_{ta}{tb}_{M}x{N}x{K}", dtype, bool(ta), bool(tb), M, N, K, **kw)
+
+
+# ------------------------------------------------------------------ fallback and cross-check kernels
+@pytest.mark.parametrize("dtype", PAIRS_16 + [W.PEAK_F32_F32])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_fallback_any_layout_any_pitch(dtype, ta, tb):
+    for (M, N, K, a, b) in [(1, 1, 1, 1.0, 0.0), (67, 130, 45, 0.5, 2.0), (128, 64, 200, -1.0, 1.0), (5, 300, 17, 2.0, 0.0)]:
+        c = mk(dtype, ta, tb, M, N, K, alpha=a, beta=b, pad_a=1, pad_b=3, pad_c=5, case=M)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_FALLBACK)
+        R.check_full(dc)
+
+
+def test_config0_fp16_512_every_family():
+    c = W.config0()
+    for v in [P.PEAK_VARIANT_FALLBACK] + UMMA + [P.PEAK_VARIANT_AUTO]:
+        dc = R.DeviceCase(c)
+        dc.run(v)
+        R.check_full(dc, what=f"config0/{P.peak_variant_string(v)}")
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_BF16_BF16, W.PEAK_F32_F32, W.PEAK_F16_F32])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_xcheck_f64_matches_oracle(dtype, ta, tb):
+    c = mk(dtype, ta, tb, 70, 90, 150, alpha=0.5, beta=2.0, pad_a=2, pad_b=2, pad_c=2)
+    dc = R.DeviceCase(c)
+    out = torch.full((c.M, c.N + 3), float("nan"), dtype=torch.float64, device="cuda")
+    P.peak_gemm_xcheck_f64(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta,
+                           dc.C, c.ldc, out, c.N + 3)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    ref, S = dc.oracle_full()
+    assert np.isnan(got[:, c.N:]).all()
+    sp = R.s_prime(c, S, c.alpha, c.beta, R.c0_values(dc))
+    assert (np.abs(got[:, :c.N] - ref) <= 4 * c.K * 2.0 ** -53 * sp).all()      # fp64 sum, fma vs mul+add
+    assert np.array_equal(dc.result(), dc.C0_h[:, :c.N])                           # C0 is not written
+
+
+# ------------------------------------------------------------------ tensor-core path: exactness
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("dtype", [W.PEAK_F16_F32, W.PEAK_BF16_BF16, W.PEAK_BF16_F32, W.PEAK_F16_F16])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_umma_exact_small_integers(variant, dtype, ta, tb):
+    """Entries in [-4, 4], K <= 512: every partial sum is an integer below 2^24, so any fp32 summation order
+    is exact and the output must equal the oracle's correctly rounded value bit for bit.  A dropped or
+    repeated k-block, a wrong swizzle or a wrong descriptor stride cannot pass."""
+    for (M, N, K) in [(128, 256, 64), (256, 512, 192), (384, 256, 512), (200, 328, 136)]:
+        c = mk(dtype, ta, tb, M, N, K, dist="smallint", case=K)
+        if c.out_type != "f32":
+            c = c.with_(alpha=0.125)     # keep |C| <= 16*512/8 within the exactly representable integers / eighths
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        ref, _ = dc.oracle_full()
+        want = oracle.round_to(R.OT[c.out_type], ref)
+        got = dc.result()
+        if not np.array_equal(got, want):
+            bad = np.argwhere(got != want)
+            raise AssertionError(f"{c.name} {P.peak_variant_string(variant)}: {len(bad)} of {got.size} wrong, "
+                                 f"first at {bad[0]}, rows {np.unique(bad[:, 0])[:8]}, cols {np.unique(bad[:, 1])[:8]}")
+
+
+@pytest.mark.parametrize("variant", UMMA)
+def test_umma_identity_and_rank1(variant):
+    n = 256
+    rng = np.random.default_rng(5)
+    X = W.encode(rng.standard_normal((n, n)).astype(np.float32), "bf16")
+    eye = W.encode(np.eye(n, dtype=np.float32), "bf16")
+    A, B = R.to_device(eye, "bf16"), R.to_device(X, "bf16")
+    C = torch.zeros((n, n), dtype=torch.bfloat16, device="cuda")
+    P.peak_gemm_variant(variant, W.PEAK_BF16_BF16, 0, 0, n, n, n, 1.0, A, n, B, n, 0.0, C, n)
+    assert P.peak_check()[0] == P.PEAK_OK
+    assert np.array_equal(R.to_host(C, "bf16"), X)          # I * X == X exactly
+    P.peak_gemm_variant(variant, W.PEAK_BF16_BF16, 0, 0, n, n, n, 1.0, B, n, A, n, 0.0, C, n)
+    assert P.peak_check()[0] == P.PEAK_OK
+    assert np.array_equal(R.to_host(C, "bf16"), X)          # X * I == X exactly
+
+
+# ------------------------------------------------------------------ tensor-core path: tolerance parity
+RAGGED = [(1, 8, 8), (7, 16, 24), (127, 255, 63), (129, 257, 65), (128, 256, 64), (300, 520, 200), (17, 1000, 72),
+          (513, 24, 1032)]
+
+
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("dtype", [W.PEAK_F16_F32, W.PEAK_BF16_BF16])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_umma_ragged_shapes_alpha_beta(variant, dtype, ta, tb):
+    for idx, (M, N, K) in enumerate(RAGGED):
+        # pitches must stay multiples of 8 elements for TMA: pad so that they are
+        a_cols = M if ta else K
+        b_cols = K if tb else N
+        alpha, beta = [(1.0, 0.0), (0.5, 2.0), (-1.0, 1.0)][idx % 3]
+        c = mk(dtype, ta, tb, M, N, K, alpha=alpha, beta=beta, pad_a=(-a_cols) % 8 + 8, pad_b=(-b_cols) % 8,
+               pad_c=idx % 4, case=idx)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        R.check_full(dc, what=f"{c.name}/{P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("variant", UMMA)
+def test_umma_run_to_run_bit_identical(variant):
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 640, 768, 1024, dist="normal_rsqrtk")
+    dc = R.DeviceCase(c)
+    outs = []
+    for _ in range(3):
+        dc.reset_c()
+        dc.run(variant)
+        outs.append(dc.result().copy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    R.check_full(dc)
+
+
+@pytest.mark.parametrize("variant", UMMA + [P.PEAK_VARIANT_FALLBACK])
+def test_alpha_beta_invariants_on_gpu(variant):
+    c = mk(W.PEAK_BF16_BF16, 0, 0, 256, 256, 128, beta=1.0)
+    dc = R.DeviceCase(c)
+    c0 = dc.C0_h[:, :c.N].copy()
+    dc.run(variant, alpha=0.0, beta=1.0)                    # C unchanged, bit for bit
+    assert np.array_equal(dc.result(), c0)
+    dc.run(variant, alpha=0.0, beta=0.0)                    # zeros
+    assert not dc.result().any()
+    nan_case = R.DeviceCase(c.with_(beta=0.0), c_init="poison")
+    nan_case.run(variant)                                   # beta == 0: NaN in C does not propagate
+    R.check_full(nan_case)
+    r1 = nan_case.result().copy()
+    nan_case.reset_c()
+    nan_case.run(variant, alpha=4.0)                        # power-of-two scaling is exact
+    assert np.array_equal(W.to_float64(nan_case.result(), "bf16"), 4.0 * W.to_float64(r1, "bf16"))
+
+
+def test_quick_returns_on_gpu():
+    c = mk(W.PEAK_F16_F32, 0, 0, 96, 80, 64, beta=0.5)
+    dc = R.DeviceCase(c)
+    before = dc.result().copy()
+    P.peak_gemm(c.dtype, 0, 0, 0, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb, 0.5, dc.C, c.ldc)       # M == 0
+    P.peak_gemm(c.dtype, 0, 0, c.M, 0, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb, 0.5, dc.C, c.ldc)       # N == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(dc.result(), before)
+    P.peak_gemm(c.dtype, 0, 0, c.M, c.N, 0, 1.0, None, c.lda, None, c.ldb, 0.5, dc.C, c.ldc)        # K == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(dc.result(), (0.5 * before).astype(np.float32))
+    nanA = torch.full_like(dc.A, float("nan"))
+    P.peak_gemm(c.dtype, 0, 0, c.M, c.N, c.K, 0.0, nanA, c.lda, nanA, c.ldb, 2.0, dc.C, c.ldc)      # alpha == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(dc.result(), before)               # 2 * (0.5 * before); A and B were not read
+
+
+# ------------------------------------------------------------------ SGEMM
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_sgemm_parity(ta, tb):
+    for (M, N, K, a, b) in [(128, 128, 16, 1.0, 0.0), (256, 384, 160, 0.5, 2.0), (384, 128, 1024, -1.0, 1.0)]:
+        c = mk(W.PEAK_F32_F32, ta, tb, M, N, K, alpha=a, beta=b, pad_a=4, pad_b=8, pad_c=4, case=K)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_SGEMM)
+        R.check_full(dc)
+    ci = mk(W.PEAK_F32_F32, ta, tb, 256, 256, 512, dist="smallint")
+    dc = R.DeviceCase(ci)
+    dc.run(P.PEAK_VARIANT_SGEMM)
+    ref, _ = dc.oracle_full()
+    assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref))
+
+
+def test_sgemm_unsupported_shape_is_reported_not_faulted():
+    c = mk(W.PEAK_F32_F32, 0, 0, 100, 128, 16)
+    dc = R.DeviceCase(c)
+    rc = P.peak_gemm_variant(P.PEAK_VARIANT_SGEMM, c.dtype, 0, 0, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb, 0.0,
+                             dc.C, c.ldc, check=False)
+    assert rc == P.PEAK_ERR_UNSUPPORTED
+    rc = P.peak_gemm_variant(P.PEAK_VARIANT_UMMA_1CTA, c.dtype, 0, 0, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb,
+                             0.0, dc.C, c.ldc, check=False)
+    assert rc == P.PEAK_ERR_UNSUPPORTED
+    dc.run(P.PEAK_VARIANT_AUTO)                              # the dispatcher falls back
+    R.check_full(dc)
+
+
+def test_host_buffer_entry_point():
+    c = mk(W.PEAK_BF16_BF16, 1, 0, 300, 264, 200, alpha=0.5, beta=2.0, pad_a=4, pad_c=8)
+    A, B, C0 = W.make_inputs(c)
+    C = C0.copy()
+    P.peak_gemm_host(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, A, c.lda, B, c.ldb, c.beta, C, c.ldc)
+    ref, S = oracle.gemm(oracle.BF16, oracle.BF16, 1, 0, c.M, c.N, c.K, c.alpha, A, c.lda, B, c.ldb, c.beta, C0, c.ldc)
+    R.check_values(c, C[:, :c.N], ref, S, W.to_float64(C0[:, :c.N], "bf16"), what="host entry point")
+    assert np.array_equal(C[:, c.N:], C0[:, c.N:])           # pitch padding survives the round trip
+    P.peak_release_staging()
+
+
+def test_launch_counter_moves():
+    n0 = P.peak_kernel_launches()
+    dc = R.DeviceCase(W.config0())
+    dc.run()
+    assert P.peak_kernel_launches() == n0 + 1

@@ -1,0 +1,134 @@
+"""Host-side checks that need no GPU: the library loads and exports what the header declares, arguments
+are validated before any device call, the dispatcher's choices, the tile order, the input generators."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2512_19018_b200 import binding as P
+from paper_2512_19018_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2512_19018_b200 import build
+    build.build()
+    return P.load()
+
+
+def test_exports_match_header(lib):
+    text = open(os.path.join(ROOT, "include", "peak_gemm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(peak_[a-z0-9_]+)\s*\(", text)))
+    assert declared == sorted(P.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} is declared in the header but not exported"
+    assert P.peak_version() >= 100
+    assert P.peak_status_string(P.PEAK_OK) == "ok"
+    assert P.peak_variant_string(P.PEAK_VARIANT_UMMA_2CTA) == "umma_2cta"
+
+
+def test_invalid_arguments_rejected_without_a_device(lib):
+    A = B = C = 0x1000  # never dereferenced: validation comes first
+    ok = dict(dtype=P.PEAK_BF16_BF16, transA=0, transB=0, M=64, N=64, K=64, alpha=1.0, A=A, lda=64, B=B, ldb=64,
+              beta=0.0, C=C, ldc=64)
+    def call(**kw):
+        a = dict(ok, **kw)
+        return P.peak_gemm(a["dtype"], a["transA"], a["transB"], a["M"], a["N"], a["K"], a["alpha"], a["A"], a["lda"],
+                           a["B"], a["ldb"], a["beta"], a["C"], a["ldc"], None, check=False)
+    assert call(dtype=9) == P.PEAK_ERR_INVALID_VALUE
+    assert call(dtype=-1) == P.PEAK_ERR_INVALID_VALUE
+    assert call(transA=2) == P.PEAK_ERR_INVALID_VALUE
+    assert call(transB=-1) == P.PEAK_ERR_INVALID_VALUE
+    assert call(M=-1) == P.PEAK_ERR_INVALID_VALUE
+    assert call(lda=63) == P.PEAK_ERR_INVALID_VALUE
+    assert call(ldb=63) == P.PEAK_ERR_INVALID_VALUE
+    assert call(ldc=63) == P.PEAK_ERR_INVALID_VALUE
+    assert call(transA=1, M=128, lda=64) == P.PEAK_ERR_INVALID_VALUE        # A stored K x M needs lda >= M
+    assert call(transB=1, K=128, lda=128, ldb=64) == P.PEAK_ERR_INVALID_VALUE  # B stored N x K needs ldb >= K
+    assert call(A=None) == P.PEAK_ERR_INVALID_VALUE
+    assert call(C=None) == P.PEAK_ERR_INVALID_VALUE
+    # nothing to do: returns OK without touching a device
+    assert call(M=0) == P.PEAK_OK
+    assert call(N=0) == P.PEAK_OK
+    assert call(alpha=0.0, beta=1.0) == P.PEAK_OK
+    assert call(K=0, beta=1.0, A=None, B=None) == P.PEAK_OK
+    rc = P.peak_gemm_variant(99, P.PEAK_BF16_BF16, 0, 0, 64, 64, 64, 1.0, A, 64, B, 64, 0.0, C, 64, None, check=False)
+    assert rc == P.PEAK_ERR_INVALID_VALUE
+
+
+def test_no_silent_fallback_without_gpu(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    rc = P.peak_gemm(P.PEAK_BF16_BF16, 0, 0, 64, 64, 64, 1.0, 0x1000, 64, 0x1000, 64, 0.0, 0x1000, 64, None,
+                     check=False)
+    assert rc in (P.PEAK_ERR_CUDA, P.PEAK_ERR_ARCH)     # fails loudly: there is no CPU path
+    with pytest.raises(P.PeakError):
+        P.peak_gemm(P.PEAK_BF16_BF16, 0, 0, 64, 64, 64, 1.0, 0x1000, 64, 0x1000, 64, 0.0, 0x1000, 64, None)
+
+
+def test_dispatch_choices(lib):
+    q = P.peak_query_variant
+    al = 0x10000  # a 16-byte aligned fake pointer
+    assert q(P.PEAK_BF16_BF16, 0, 0, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) in (
+        P.PEAK_VARIANT_UMMA_1CTA, P.PEAK_VARIANT_UMMA_2CTA)
+    assert q(P.PEAK_F16_F32, 1, 0, 5000, 3000, 2500, 0.5, al, 5000, al, 3000, 2.0, al, 3000) in (
+        P.PEAK_VARIANT_UMMA_1CTA, P.PEAK_VARIANT_UMMA_2CTA)
+    # a pitch that is not a multiple of 16 bytes, or a misaligned base, cannot use TMA
+    assert q(P.PEAK_BF16_BF16, 0, 0, 100, 100, 100, 1.0, al, 100, al, 100, 0.0, al, 100) == P.PEAK_VARIANT_FALLBACK
+    assert q(P.PEAK_BF16_BF16, 0, 0, 128, 128, 128, 1.0, al + 2, 128, al, 128, 0.0, al, 128) == P.PEAK_VARIANT_FALLBACK
+    assert q(P.PEAK_F32_F32, 0, 0, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_SGEMM
+    assert q(P.PEAK_F32_F32, 0, 0, 100, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
+    assert q(P.PEAK_F32_F32, 0, 0, 0, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_NONE
+    assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 0, 1.0, None, 1, None, 64, 0.5, al, 64) == P.PEAK_VARIANT_SCALE
+    assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 1.0, al, 64) == P.PEAK_VARIANT_NONE
+    assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 0.0, al, 64) == P.PEAK_VARIANT_SCALE
+    assert q(7, 0, 0, 64, 64, 64, 1.0, al, 64, al, 64, 0.0, al, 64) == -P.PEAK_ERR_INVALID_VALUE
+
+
+@pytest.mark.parametrize("tiles_m,tiles_n,group", [(1, 1, 8), (64, 32, 16), (32, 32, 8), (20, 12, 16), (7, 5, 3),
+                                                   (1, 16, 8), (40, 1, 16), (13, 9, 1), (5, 7, 100)])
+def test_tile_order_is_a_bijection_and_grouped(lib, tiles_m, tiles_n, group):
+    seen = set()
+    prev_group = 0
+    for t in range(tiles_m * tiles_n):
+        tm, tn = P.peak_tile_coord(t, tiles_m, tiles_n, group)
+        assert 0 <= tm < tiles_m and 0 <= tn < tiles_n
+        seen.add((tm, tn))
+        g = tm // group
+        assert g >= prev_group          # groups of tile-rows are finished one after the other
+        prev_group = g
+    assert len(seen) == tiles_m * tiles_n
+    # consecutive tiles inside a group walk down the rows first (they share the B panel)
+    if tiles_m >= 2 and group >= 2:
+        a, b = P.peak_tile_coord(0, tiles_m, tiles_n, group), P.peak_tile_coord(1, tiles_m, tiles_n, group)
+        assert b == (a[0] + 1, a[1])
+    with pytest.raises(P.PeakError):
+        P.peak_tile_coord(tiles_m * tiles_n, tiles_m, tiles_n, group)
+
+
+def test_workload_generators_are_seeded_and_shaped():
+    c = W.config0()
+    A1, B1, C1 = W.make_inputs(c)
+    A2, B2, _ = W.make_inputs(c)
+    assert C1 is None and np.array_equal(A1, A2) and np.array_equal(B1, B2)
+    assert A1.shape == (512, 512) and A1.dtype == np.uint16
+    a = W.to_float64(A1, "f16")
+    assert a.min() >= -1.0 and a.max() <= 1.0 and abs(a.mean()) < 0.01
+    r = W.config4_ragged(0)
+    assert (r.layout, r.lda, r.ldb, r.ldc) == ("TN", 5000, 3000, 3000)
+    assert r.a_shape == (2500, 5000) and r.b_shape == (2500, 3000)
+    t = W.config3(1)
+    assert t.layout == "NT" and t.b_shape == (14336, 4096) and t.beta == 1.0
+    small = t.with_(M=64, N=48, K=32)
+    A, B, C0 = W.make_inputs(small)
+    assert B.shape == (48, 32) and C0.shape == (64, 48)
+    assert abs(W.to_float64(B, "bf16").std() - 0.02) < 0.003
+    p = W.GemmCase("pad", W.PEAK_F32_F32, False, False, 5, 6, 7, pad_a=2, pad_c=1, beta=1.0)
+    A, B, C0 = W.make_inputs(p)
+    assert A.shape == (5, 9) and np.isnan(A[:, 7:]).all() and C0.shape == (5, 7)
+    assert W.config1().min_bytes() == 3 * 4096 * 4096 * 2
