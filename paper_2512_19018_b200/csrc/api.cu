@@ -60,6 +60,9 @@ int choose_variant(const GemmArgs &g) {
     if (g.M == 0 || g.N == 0) return PEAK_VARIANT_NONE;
     if (g.K == 0 || g.alpha == 0.0f) return (g.beta == 1.0f) ? PEAK_VARIANT_NONE : PEAK_VARIANT_SCALE;
     if (in_elem(g.dtype) == Elem::F32) return sgemm_supports(g) ? PEAK_VARIANT_SGEMM : PEAK_VARIANT_FALLBACK;
+    // CTA pairs (256-row tiles, B shared between the two SMs) win whenever there is more than one
+    // 128-row block of C; a single block of rows would leave the second CTA of each pair idle.
+    if (umma_supports(g, 2) && g.M > 128) return PEAK_VARIANT_UMMA_2CTA;
     if (umma_supports(g, 1)) return PEAK_VARIANT_UMMA_1CTA;
     return PEAK_VARIANT_FALLBACK;
 }

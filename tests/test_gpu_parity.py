@@ -73,6 +73,8 @@ def test_umma_exact_small_integers(variant, dtype, ta, tb):
         ref, _ = dc.oracle_full()
         want = oracle.round_to(R.OT[c.out_type], ref)
         got = dc.result()
+        if c.out_type == "f32":
+            got = got.view(np.uint32)
         if not np.array_equal(got, want):
             bad = np.argwhere(got != want)
             raise AssertionError(f"{c.name} {P.peak_variant_string(variant)}: {len(bad)} of {got.size} wrong, "
