@@ -74,8 +74,9 @@ typedef enum peak_variant {
     PEAK_VARIANT_AUTO = 0,
     PEAK_VARIANT_FALLBACK = 1, /* plain tiled CUDA-core kernel: any dtype, layout, alignment (the paper's naive
                                   kernel of section 2.2 with thread-block tiling) */
-    PEAK_VARIANT_UMMA_1CTA = 2, /* tcgen05.mma, 128x256 tile per CTA, TMA ring, persistent (16-bit inputs) */
-    PEAK_VARIANT_UMMA_2CTA = 3, /* tcgen05.mma cta_group::2, 256x256 tile per CTA pair (16-bit inputs) */
+    PEAK_VARIANT_UMMA_1CTA = 2, /* tcgen05.mma, 128 x (256|128) tile per CTA, TMA ring, persistent, optional
+                                   split-K (16-bit inputs) */
+    PEAK_VARIANT_UMMA_2CTA = 3, /* tcgen05.mma cta_group::2, 256 x (256|128) tile per CTA pair (16-bit inputs) */
     PEAK_VARIANT_SGEMM = 4,     /* register-tiled fp32 FMA kernel (fp32 inputs) */
     PEAK_VARIANT_SCALE = 5,     /* C = beta*C only (K == 0 or alpha == 0) */
     PEAK_VARIANT_NONE = 6       /* nothing to do (M == 0 or N == 0, or alpha == 0 and beta == 1) */
@@ -153,6 +154,20 @@ int peak_tile_coord(int64_t tile, int64_t tiles_m, int64_t tiles_n, int64_t grou
  * `detail`, if not NULL, receives the raw status word (role and barrier that gave up).
  */
 int peak_check(void *stream, uint32_t *detail);
+
+/*
+ * peak_set_tuning: performance knobs that never change results (the paper's "tuning parameters",
+ * section 3.1).  value 0 restores the library default.  Process-wide; returns PEAK_ERR_INVALID_VALUE for an
+ * unknown key or a negative value.
+ */
+typedef enum peak_tuning_key {
+    PEAK_TUNE_RASTER_GROUP = 0, /* tile-rows per raster group of the persistent scheduler */
+    PEAK_TUNE_TILE_N = 1,       /* tensor-core tile width: 128 or 256 */
+    PEAK_TUNE_SPLIT_K = 2,      /* k-slices per tile (1 = never split; capped by the number of k-blocks) */
+    PEAK_TUNE_EPILOGUE = 3,     /* 1 = direct global stores, 2 = shared-memory staging + TMA stores */
+    PEAK_TUNE_COUNT_ = 4
+} peak_tuning_key_t;
+int peak_set_tuning(int key, int value);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t peak_kernel_launches(void);

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libpeak_gemm.so")
 _lib = None
 
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
-           "peak_query_variant", "peak_tile_coord", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
+           "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
            "peak_status_string", "peak_variant_string", "peak_version"]
 
 
@@ -60,6 +60,8 @@ def load():
     lib.peak_query_variant.argtypes = [i, i, i, i64, i64, i64, f, vp, i64, vp, i64, f, vp, i64]
     lib.peak_tile_coord.restype = i
     lib.peak_tile_coord.argtypes = [i64, i64, i64, i64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.peak_set_tuning.restype = i
+    lib.peak_set_tuning.argtypes = [i, i]
     lib.peak_check.restype = i
     lib.peak_check.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.peak_kernel_launches.restype = i64
@@ -143,6 +145,13 @@ def peak_tile_coord(tile, tiles_m, tiles_n, group):
     if rc != PEAK_OK:
         raise PeakError(rc, "peak_tile_coord")
     return tm.value, tn.value
+
+
+PEAK_TUNE_RASTER_GROUP, PEAK_TUNE_TILE_N, PEAK_TUNE_SPLIT_K, PEAK_TUNE_EPILOGUE = 0, 1, 2, 3
+
+
+def peak_set_tuning(key: int, value: int) -> int:
+    return _raise(load().peak_set_tuning(key, value), "peak_set_tuning")
 
 
 def peak_check(stream=None):

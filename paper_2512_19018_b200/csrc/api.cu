@@ -20,6 +20,11 @@ uint32_t *g_status_ptr[kMaxDevices] = {};
 std::mutex g_status_mutex;
 }  // namespace
 
+namespace {
+std::atomic<int> g_tuning[PEAK_TUNE_COUNT_];
+}
+int tuning(int key) { return (key >= 0 && key < PEAK_TUNE_COUNT_) ? g_tuning[key].load(std::memory_order_relaxed) : 0; }
+
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 void set_cuda_error(cudaError_t e) { t_last_cuda_error = (int)e; }
 
@@ -245,6 +250,12 @@ int peak_check(void *stream, uint32_t *detail) {
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     if (detail) *detail = host;
     return (host & kStatusTimeout) ? PEAK_ERR_TIMEOUT : PEAK_OK;
+}
+
+int peak_set_tuning(int key, int value) {
+    if (key < 0 || key >= PEAK_TUNE_COUNT_ || value < 0) return PEAK_ERR_INVALID_VALUE;
+    g_tuning[key].store(value, std::memory_order_relaxed);
+    return PEAK_OK;
 }
 
 int64_t peak_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }

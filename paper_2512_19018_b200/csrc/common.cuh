@@ -42,6 +42,7 @@ __device__ __forceinline__ float epilogue_f32(float alpha, float acc, float beta
 void count_launch(int n = 1);
 void set_cuda_error(cudaError_t e);
 uint32_t *device_status_word();  // address of the per-device status word (nullptr on failure)
+int tuning(int key);             // value set through peak_set_tuning (0 = library default)
 
 struct GemmArgs {
     int dtype, transA, transB;

@@ -1,17 +1,25 @@
 // Tensor-core GEMM for 16-bit inputs on sm_100a.
 //
-// One persistent CTA (or CTA pair) per SM walks output tiles in a grouped order (the paper's block
-// swizzle).  Inside a CTA three roles run concurrently (warp specialisation):
+// One persistent CTA (or CTA pair) per SM walks work items -- output tiles, or (tile, k-slice) pairs when
+// K is split -- in a grouped order (the paper's block swizzle).  Inside a CTA three roles run concurrently
+// (warp specialisation):
 //   warp 0      producer: TMA tile loads of A and B into a ring of 128-byte-swizzled shared-memory stages
 //               (the paper's thread-block tiling + pipelining + bank-conflict offset, section 2.2),
 //   warp 1      one thread issues tcgen05.mma; fp32 accumulators live in tensor memory (the paper's
 //               warp tiling / tensor-core steps), two accumulator buffers so that the next tile's main
 //               loop overlaps this tile's epilogue,
-//   warps 2..5  epilogue: tcgen05.ld -> alpha/beta in fp32 -> one rounding -> vectorised global stores.
+//   warps 2..5  epilogue: tcgen05.ld -> alpha/beta in fp32 -> one rounding -> swizzled shared-memory
+//               staging -> TMA store (coalesced, clipped at the matrix edge); a direct vector / scalar
+//               store path serves outputs whose base or pitch is not 16-byte aligned.
 // mbarriers connect the roles (full/empty per stage, full/empty per accumulator).  Every wait is bounded.
 //
-// Tile: 128 x 256 x 64 per CTA (CTA_GROUP 1) or 256 x 256 x 64 per CTA pair (CTA_GROUP 2, each CTA stages
-// its 128 rows of A and its 128-column half of B; the leader CTA issues MMAs for both).
+// Tile: 128 x BN x 64 per CTA (CTA_GROUP 1) or 256 x BN x 64 per CTA pair (CTA_GROUP 2: each CTA stages its
+// 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 256 or 128.
+//
+// Split-K (the paper's Split-K transformation, section 4.1): for shapes with too few tiles to fill the GPU,
+// each tile's k-blocks are divided among `splits` work items; every item stores its fp32 partial tile to
+// a workspace slice and a second kernel adds the slices in a fixed order and applies alpha/beta, so the
+// result does not depend on scheduling.
 #include <cuda.h>
 
 #include <mutex>
@@ -23,33 +31,45 @@ namespace peak {
 namespace {
 
 constexpr int BM = 128;   // rows of C per CTA
-constexpr int BN = 256;   // columns of C per tile
 constexpr int BK = 64;    // k-block: 64 16-bit elements = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KiB
 constexpr int ATOM_BYTES = 64 * BK * 2;     // one 64-wide MN-major box: 64 k-rows of 128 bytes = 8 KiB
 constexpr int NUM_THREADS = 192;
-constexpr int TMEM_COLS = 512;              // two 256-column fp32 accumulators
+constexpr int EPI_BUF_BYTES = 32 * 128;               // one staging buffer: 32 rows x 128 bytes
+constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;      // 4 epilogue warps x 2 buffers = 32 KiB
+constexpr int SMEM_LIMIT = 232448;                    // 227 KiB of dynamic shared memory per CTA
 
-template <int CG> struct Cfg {
+template <int CG, int BN> struct Cfg {
     static constexpr int B_ROWS = BN / CG;                 // rows of op(B)^T this CTA stages
-    static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;  // 32 KiB or 16 KiB
+    static constexpr int B_BOX_ROWS = B_ROWS < 128 ? B_ROWS : 128;
+    static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = (CG == 1) ? 4 : 6;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int AUX_BYTES = 256;
+    static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - EPI_BYTES - AUX_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + AUX_BYTES;
+    static constexpr int TMEM_COLS = 2 * BN;               // two fp32 accumulators
+    static_assert(STAGES >= 3, "pipeline too shallow");
+    static_assert(8 * (2 * STAGES + 4) + 8 <= AUX_BYTES, "barrier area too small");
 };
 
 struct UmmaParams {
     int M, N, K;
     int num_kb;            // ceil(K / BK)
-    int tiles_m, tiles_n;  // in units of (128*CG) x 256
+    int tiles_m, tiles_n;  // in units of (128*CG) x BN
     int group;             // tile-rows per raster group
+    int splits;            // k-slices per tile (1 = no split)
+    int kb_per_split;
     int a_mn, b_mn;        // 1: operand is MN-major in memory (transA == 1 / transB == 0)
     uint32_t idesc;
     float alpha, beta;
-    void *C;
+    void *C;               // output (or fp32 workspace when splits > 1)
     int64_t ldc;
+    int64_t slice_stride;  // elements between workspace slices (splits > 1)
+    int slice_rows;        // rows per workspace slice in the TMA store map (splits > 1)
     int vec_ok;            // C base and pitch allow 16-byte vector access
+    int tma_store;         // epilogue stores through TMA
     uint32_t *status;
 };
 
@@ -66,8 +86,14 @@ __device__ __forceinline__ void report_timeout(const UmmaParams &p, volatile uin
     *abort_flag = 1;
 }
 
+template <typename TOut> __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    TOut a = from_f32<TOut>(lo), b = from_f32<TOut>(hi);
+    return (uint32_t)(*reinterpret_cast<uint16_t *>(&a)) | ((uint32_t)(*reinterpret_cast<uint16_t *>(&b)) << 16);
+}
+
+// 32 consecutive outputs of one row -> global memory (vector path when aligned and whole)
 template <typename TOut>
-__device__ __forceinline__ void store_row_chunk(TOut *dst, const float (&v)[32], int valid, bool vec) {
+__device__ __forceinline__ void store_row32(TOut *dst, const float (&v)[32], int valid, bool vec) {
     if (vec && valid == 32) {
         if constexpr (sizeof(TOut) == 4) {
 #pragma unroll
@@ -75,16 +101,10 @@ __device__ __forceinline__ void store_row_chunk(TOut *dst, const float (&v)[32],
                 reinterpret_cast<float4 *>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t w[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    TOut lo = from_f32<TOut>(v[8 * i + 2 * j]), hi = from_f32<TOut>(v[8 * i + 2 * j + 1]);
-                    w[j] = (uint32_t)(*reinterpret_cast<uint16_t *>(&lo)) |
-                           ((uint32_t)(*reinterpret_cast<uint16_t *>(&hi)) << 16);
-                }
-                reinterpret_cast<uint4 *>(dst)[i] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+            for (int i = 0; i < 4; ++i)
+                reinterpret_cast<uint4 *>(dst)[i] =
+                    make_uint4(pack2<TOut>(v[8 * i], v[8 * i + 1]), pack2<TOut>(v[8 * i + 2], v[8 * i + 3]),
+                               pack2<TOut>(v[8 * i + 4], v[8 * i + 5]), pack2<TOut>(v[8 * i + 6], v[8 * i + 7]));
         }
     } else {
 #pragma unroll
@@ -93,8 +113,9 @@ __device__ __forceinline__ void store_row_chunk(TOut *dst, const float (&v)[32],
     }
 }
 
+// 32 consecutive old values of one row <- global memory
 template <typename TOut>
-__device__ __forceinline__ void load_row_chunk(const TOut *src, float (&c)[32], int valid, bool vec) {
+__device__ __forceinline__ void load_row32(const TOut *src, float (&c)[32], int valid, bool vec) {
     if (vec && valid == 32) {
         if constexpr (sizeof(TOut) == 4) {
 #pragma unroll
@@ -121,17 +142,43 @@ __device__ __forceinline__ void load_row_chunk(const TOut *src, float (&c)[32], 
     }
 }
 
-template <int CG, typename TOut>
+// 32 consecutive outputs of row `lane` -> staging buffer laid out as the 128-byte-swizzled box a TMA
+// store expects: 16-byte piece j of row r sits at piece (j ^ (r & 7)).  `h` selects which 32-column
+// half of a 64-column (16-bit) chunk is written; fp32 chunks are 32 columns wide and use h = 0.
+template <typename TOut>
+__device__ __forceinline__ void stage_row32(uint32_t buf, int lane, int h, const float (&v)[32]) {
+    constexpr int PIECES = 32 * (int)sizeof(TOut) / 16;  // 8 (fp32) or 4 (16-bit)
+    const uint32_t row = buf + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int j = 0; j < PIECES; ++j) {
+        uint32_t w0, w1, w2, w3;
+        if constexpr (sizeof(TOut) == 4) {
+            w0 = __float_as_uint(v[4 * j]); w1 = __float_as_uint(v[4 * j + 1]);
+            w2 = __float_as_uint(v[4 * j + 2]); w3 = __float_as_uint(v[4 * j + 3]);
+        } else {
+            w0 = pack2<TOut>(v[8 * j], v[8 * j + 1]); w1 = pack2<TOut>(v[8 * j + 2], v[8 * j + 3]);
+            w2 = pack2<TOut>(v[8 * j + 4], v[8 * j + 5]); w3 = pack2<TOut>(v[8 * j + 6], v[8 * j + 7]);
+        }
+        const uint32_t piece = (uint32_t)((h * PIECES + j) ^ (lane & 7));
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + piece * 16u), "r"(w0), "r"(w1), "r"(w2),
+                     "r"(w3)
+                     : "memory");
+    }
+}
+
+template <int CG, int BN, typename TOut>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const UmmaParams p) {
-    using C_ = Cfg<CG>;
+                 const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+    using C_ = Cfg<CG, BN>;
     constexpr int STAGES = C_::STAGES;
+    constexpr int CHUNK_COLS = 128 / (int)sizeof(TOut);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
     extern __shared__ uint8_t smem_raw[];
 
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t stage_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-    uint8_t *aux = smem_raw + (stage_base - raw) + STAGES * C_::STAGE_BYTES;
+    const uint32_t epi_base = stage_base + STAGES * C_::STAGE_BYTES;
+    uint8_t *aux = smem_raw + (epi_base - raw) + EPI_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * (2 * STAGES + 4));
     volatile uint32_t *abort_flag = tmem_slot + 1;
@@ -147,7 +194,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool leader = (rank == 0);
     const int unit = blockIdx.x / CG;          // CTA (or CTA pair) index
     const int num_units = gridDim.x / CG;
-    const int total_tiles = p.tiles_m * p.tiles_n;
+    const int total_items = p.tiles_m * p.tiles_n * p.splits;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -165,9 +212,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (warp == 0 && lane == 0) {
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB);
+        if (p.tma_store) ptx::prefetch_tensormap(&tmC);
     }
     if (warp == 1) {
-        ptx::tmem_alloc<CG>(ptx::smem_u32(tmem_slot), TMEM_COLS);
+        ptx::tmem_alloc<CG>(ptx::smem_u32(tmem_slot), C_::TMEM_COLS);
         ptx::tmem_relinquish<CG>();
     }
     ptx::tc_fence_before_sync();
@@ -181,12 +229,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
+            for (int item = unit; item < total_items && ok; item += num_units) {
+                const int tile = item / p.splits, slice = item - tile * p.splits;
                 int64_t tm, tn;
                 tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CG) + (int)rank * BM;
                 const int n_cta = (int)tn * BN + (int)rank * C_::B_ROWS;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                const int kb0 = slice * p.kb_per_split;
+                const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
                         report_timeout(p, abort_flag, 1, s);
@@ -211,9 +262,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     if (!p.b_mn) {
 #pragma unroll
-                        for (int h = 0; h < C_::B_ROWS / 128; ++h) {
-                            if (CG == 1) ptx::tma_load_2d(b_dst + h * 128 * 128, &tmB, k0, n_cta + 128 * h, bar);
-                            else ptx::tma_load_2d_pair(b_dst + h * 128 * 128, &tmB, k0, n_cta + 128 * h, bar);
+                        for (int h = 0; h < C_::B_ROWS / C_::B_BOX_ROWS; ++h) {
+                            const uint32_t d = b_dst + h * C_::B_BOX_ROWS * 128;
+                            if (CG == 1) ptx::tma_load_2d(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
+                            else ptx::tma_load_2d_pair(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
                         }
                     } else {
 #pragma unroll
@@ -241,7 +293,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             const uint32_t a_lbo = p.a_mn ? (uint32_t)ATOM_BYTES : 16u, b_lbo = p.b_mn ? (uint32_t)ATOM_BYTES : 16u;
             const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
-            for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tl) {
+            for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
+                const int slice = item % p.splits;
+                const int kb0 = slice * p.kb_per_split;
+                const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);
                 const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
                 if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag)) {
                     report_timeout(p, abort_flag, 3, b);
@@ -250,7 +305,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + b * BN;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag)) {
                         report_timeout(p, abort_flag, 4, s);
@@ -264,7 +319,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
                         const uint64_t bd = smem_desc(b_base + k * b_kstep, b_lbo, 1024u);
-                        ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb | k) != 0));
+                        ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
                     }
                     // release the stage (in both CTAs of a pair) once these MMAs have read it
                     if (CG == 1) ptx::umma_commit_1cta(empty0 + 8 * s);
@@ -279,14 +334,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else {
         // ------------------------------------------------------------------ epilogue (4 warps)
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
-        TOut *Cout = reinterpret_cast<TOut *>(p.C);
-        uint32_t tl = 0;
+        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
+        const bool vec = p.vec_ok != 0;
+        uint32_t tl = 0, chunk_no = 0;
         bool ok = true;
-        for (int tile = unit; tile < total_tiles && ok; tile += num_units, ++tl) {
+        for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
+            const int tile = item / p.splits, slice = item - tile * p.splits;
             int64_t tm, tn;
             tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-            const int row = (int)tm * (BM * CG) + (int)rank * BM + q * 32 + lane;
+            const int row0 = (int)tm * (BM * CG) + (int)rank * BM + q * 32;  // first row of this warp
+            const int row = row0 + lane;
             const int n0 = (int)tn * BN;
+            TOut *Cout = reinterpret_cast<TOut *>(p.C) + (int64_t)slice * p.slice_stride;
+            const int store_row0 = row0 + slice * p.slice_rows;  // row coordinate in the TMA store map
             const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
             // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
             const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag);
@@ -298,26 +358,49 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::tc_fence_after_sync();
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                const int col = n0 + c * 32;
-                if (col >= p.N) break;  // warp-uniform
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(t_addr + c * 32, r);
-                ptx::tmem_ld_wait();
-                if (row < p.M) {
-                    const int valid = (p.N - col < 32) ? (p.N - col) : 32;
+            for (int c = 0; c < BN / CHUNK_COLS; ++c) {
+                const int col0 = n0 + c * CHUNK_COLS;
+                if (col0 >= p.N) break;  // warp-uniform
+                uint32_t buf = 0;
+                if (p.tma_store) {
+                    // the store that last read this buffer (two chunks ago) must have drained it
+                    buf = my_stage + (chunk_no & 1u) * EPI_BUF_BYTES;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int h = 0; h < CHUNK_COLS / 32; ++h) {
+                    const int col = col0 + h * 32;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r);
+                    ptx::tmem_ld_wait();
+                    const int valid = (p.N - col >= 32) ? 32 : (p.N - col > 0 ? p.N - col : 0);
                     TOut *dst = Cout + (int64_t)row * p.ldc + col;
                     float v[32];
                     if (p.beta != 0.0f) {
                         float cold[32];
-                        load_row_chunk<TOut>(dst, cold, valid, p.vec_ok != 0);
+                        if (row < p.M && valid > 0) load_row32<TOut>(dst, cold, valid, vec);
+                        else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = fmaf(p.beta, cold[i], p.alpha * __uint_as_float(r[i]));
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
                     }
-                    store_row_chunk<TOut>(dst, v, valid, p.vec_ok != 0);
+                    if (p.tma_store) stage_row32<TOut>(buf, lane, h, v);
+                    else if (row < p.M && valid > 0) store_row32<TOut>(dst, v, valid, vec);
+                }
+                if (p.tma_store) {
+                    ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M) {
+                        ptx::tma_store_2d(&tmC, col0, store_row0, buf);
+                        ptx::tma_store_commit();
+                    }
+                    ++chunk_no;
                 }
             }
             // hand the accumulator buffer back to the MMA issuer
@@ -328,6 +411,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, 0));
             }
         }
+        if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();  // staging memory must outlive the stores
+        __syncwarp();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -341,7 +426,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (CG == 2) ptx::cluster_sync();  // the peer may still signal this CTA's barriers or read its tiles
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc<CG>(tmem_base, TMEM_COLS);
+        ptx::tmem_dealloc<CG>(tmem_base, C_::TMEM_COLS);
+    }
+}
+
+// Adds the k-slices of a split GEMM in slice order and applies the epilogue:
+// C = alpha * (ws[0] + ws[1] + ... ) + beta * C, one rounding.
+template <typename TOut>
+__global__ void splitk_reduce_kernel(const float *__restrict__ ws, int64_t slice_stride, int64_t ldws, int splits,
+                                     int64_t M, int64_t N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc) {
+    const int64_t total = M * N;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = e / N, j = e - i * N;
+        const float *src = ws + i * ldws + j;
+        float acc = src[0];
+        for (int s = 1; s < splits; ++s) acc += src[(int64_t)s * slice_stride];
+        TOut *dst = C + i * ldc + j;
+        const float c_old = (beta != 0.0f) ? to_f32(*dst) : 0.0f;
+        *dst = from_f32<TOut>(epilogue_f32(alpha, acc, beta, c_old));
     }
 }
 
@@ -364,25 +466,77 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Tensor map over a row-major 2-D array of 16-bit elements: `inner` contiguous elements per row,
-// `outer` rows, `pitch` elements between rows; box = box_inner x box_outer, 128-byte swizzle, zero fill.
+// Tensor map over a row-major 2-D array: `inner` contiguous elements per row, `outer` rows, `pitch`
+// elements between rows; box = box_inner x box_outer, 128-byte swizzle, zero fill.
 bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
               int box_outer) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                   : e == Elem::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                     : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch * (cuuint64_t)elem_bytes(e)};
     cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, e == Elem::F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                    const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    CUresult r = fn(tm, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
-template <int CG, typename TOut> int run_umma(const GemmArgs &g) {
-    using C_ = Cfg<CG>;
-    auto kernel = umma_gemm_kernel<CG, TOut>;
+int sm_count() {
+    static int sms[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return 148;
+    if (sms[dev] == 0) {
+        int n = 0;
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        sms[dev] = n > 0 ? n : 148;
+    }
+    return sms[dev];
+}
+
+constexpr double kL2BytesPerClk = 64.0;  // assumed L2 -> shared-memory bandwidth per SM
+
+struct Plan {
+    int bn;      // 256 or 128
+    int splits;  // k-slices per tile
+};
+
+// Tile width and k-split from a small cost model (cycles): an item costs its k-blocks times the slower of
+// the tensor pipe (2*BN cycles per k-block per SM) and the operand stream (bytes per k-block over an
+// assumed 64 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread
+// over the units in waves.  A split additionally pays for writing and re-reading fp32 partials.
+Plan choose_plan(const GemmArgs &g, int cg, int units) {
+    const int64_t num_kb = (g.K + BK - 1) / BK;
+    Plan best{256, 1};
+    double best_cost = 1e300;
+    const int force_bn = tuning(PEAK_TUNE_TILE_N), force_split = tuning(PEAK_TUNE_SPLIT_K);
+    for (int bn : {256, 128}) {
+        if (force_bn && bn != force_bn) continue;
+        const int64_t tiles = ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn);
+        const double kb_cycles = fmax(2.0 * bn, (128.0 + bn / cg) * 128.0 / kL2BytesPerClk);
+        for (int s = 1; s <= 16; ++s) {
+            if (force_split && s != force_split) continue;
+            if (s > 1 && !force_split && (s > num_kb || tiles * s > 2 * units)) break;
+            if (s > num_kb) break;
+            const int64_t kbps = (num_kb + s - 1) / s;
+            if (s > 1 && (kbps * (s - 1) >= num_kb)) continue;  // an empty last slice
+            const int64_t waves = (tiles * s + units - 1) / units;
+            double cost = (double)waves * (kbps * kb_cycles + 1500.0);
+            if (s > 1) cost += 2.0 * (double)g.M * g.N * s * 4.0 / (units * 24.0) + 6000.0;  // partials + 2nd launch
+            if (cost < best_cost) { best_cost = cost; best = Plan{bn, s}; }
+        }
+    }
+    return best;
+}
+
+template <int CG, int BN, typename TOut>
+int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, void *out, int64_t ldo, Elem eout,
+                  int64_t slice_stride, int slice_rows, float alpha, float beta) {
+    using C_ = Cfg<CG, BN>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -393,9 +547,10 @@ template <int CG, typename TOut> int run_umma(const GemmArgs &g) {
     const Elem ein = in_elem(g.dtype);
     const int a_mn = g.transA ? 1 : 0;  // A stored K x M: M is the contiguous index
     const int b_mn = g.transB ? 0 : 1;  // B stored K x N: N is the contiguous index
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmC;
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK) : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BK, 128);
-    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK) : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, 128));
+    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK)
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, C_::B_BOX_ROWS));
     if (!ok) return PEAK_ERR_CUDA;
 
     UmmaParams p;
@@ -403,23 +558,36 @@ template <int CG, typename TOut> int run_umma(const GemmArgs &g) {
     p.num_kb = (int)((g.K + BK - 1) / BK);
     p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((g.N + BN - 1) / BN);
-    p.group = (CG == 1) ? 16 : 8;
+    p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : ((CG == 1) ? 16 : 8);
+    p.splits = plan.splits;
+    p.kb_per_split = (p.num_kb + plan.splits - 1) / plan.splits;
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
-    p.alpha = g.alpha; p.beta = g.beta;
-    p.C = g.C; p.ldc = g.ldc;
-    const int ob = elem_bytes(out_elem(g.dtype));
-    p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0) ? 1 : 0;
+    p.alpha = alpha; p.beta = beta;
+    p.C = out; p.ldc = ldo;
+    p.slice_stride = slice_stride; p.slice_rows = slice_rows;
+    const int ob = elem_bytes(eout);
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(out) % 16) == 0 && (ldo * ob) % 16 == 0) ? 1 : 0;
+    const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
+    // TMA stores clip rows exactly but clip the contiguous index only at 16-byte granularity, so they are
+    // used when a row of C is a whole number of 16-byte pieces; other widths take the direct-store path
+    const int64_t out_cols = plan.splits > 1 ? ldo : g.N;
+    p.tma_store = (p.vec_ok && (out_cols * ob) % 16 == 0 && epi != 1) ? 1 : 0;
+    if (p.tma_store) {
+        // rows of the map: the matrix itself, or all workspace slices stacked (each slice_rows high)
+        const int64_t rows = plan.splits > 1 ? (int64_t)plan.splits * slice_rows : g.M;
+        const int64_t cols = plan.splits > 1 ? ldo : g.N;
+        if (!make_map(&tmC, eout, out, cols, rows, ldo, 128 / ob, 32)) return PEAK_ERR_CUDA;
+    } else {
+        tmC = tmA;  // unused
+    }
     p.status = device_status_word();
     if (!p.status) return PEAK_ERR_CUDA;
 
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
-    int units = sms / CG;
+    const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.splits;
+    int units = units_max;
     if (total < units) units = (int)total;
 
     cudaLaunchConfig_t cfg = {};
@@ -432,19 +600,83 @@ template <int CG, typename TOut> int run_umma(const GemmArgs &g) {
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
 
-template <int CG> int dispatch_out(const GemmArgs &g) {
-    switch (out_elem(g.dtype)) {
-        case Elem::F32: return run_umma<CG, float>(g);
-        case Elem::F16: return run_umma<CG, __half>(g);
-        case Elem::BF16: return run_umma<CG, __nv_bfloat16>(g);
+template <typename TOut>
+int launch_reduce(const GemmArgs &g, const float *ws, int64_t slice_stride, int64_t ldws, int splits) {
+    const int64_t total = g.M * g.N;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<TOut><<<(unsigned)blocks, 256, 0, g.stream>>>(ws, slice_stride, ldws, splits, g.M, g.N, g.alpha,
+                                                                     g.beta, (TOut *)g.C, g.ldc);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+// Stream-ordered workspace for split-K partials: one memory pool per device that keeps what it has been
+// given (release threshold = max), so that steady-state calls neither touch the OS allocator nor share a
+// buffer between streams.
+cudaMemPool_t workspace_pool() {
+    static cudaMemPool_t pools[64] = {};
+    static std::mutex m;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(m);
+    if (!pools[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t pool = nullptr;
+        cudaError_t e = cudaMemPoolCreate(&pool, &props);
+        if (e != cudaSuccess) { set_cuda_error(e); return nullptr; }
+        uint64_t keep = UINT64_MAX;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        pools[dev] = pool;
     }
-    return PEAK_ERR_INVALID_VALUE;
+    return pools[dev];
+}
+
+template <int CG, int BN> int run_umma(const GemmArgs &g, const Plan &plan, int units) {
+    const Elem eout = out_elem(g.dtype);
+    if (plan.splits == 1) {
+        switch (eout) {
+            case Elem::F32: return launch_kernel<CG, BN, float>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
+            case Elem::F16: return launch_kernel<CG, BN, __half>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
+            case Elem::BF16:
+                return launch_kernel<CG, BN, __nv_bfloat16>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
+        }
+        return PEAK_ERR_INVALID_VALUE;
+    }
+    // split-K: fp32 partial tiles in a stream-ordered workspace, padded to whole tiles so that no store clips
+    const int64_t rows_pad = ((g.M + BM * CG - 1) / (BM * CG)) * (BM * CG);
+    const int64_t cols_pad = ((g.N + BN - 1) / BN) * BN;
+    const int64_t slice_stride = rows_pad * cols_pad;
+    float *ws = nullptr;
+    cudaMemPool_t pool = workspace_pool();
+    if (!pool) return PEAK_ERR_CUDA;
+    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&ws),
+                                            (size_t)slice_stride * plan.splits * sizeof(float), pool, g.stream);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_NO_MEMORY; }
+    int rc = launch_kernel<CG, BN, float>(g, plan, units, ws, cols_pad, Elem::F32, slice_stride, (int)rows_pad, 1.0f,
+                                          0.0f);
+    if (rc == PEAK_OK) {
+        switch (eout) {
+            case Elem::F32: rc = launch_reduce<float>(g, ws, slice_stride, cols_pad, plan.splits); break;
+            case Elem::F16: rc = launch_reduce<__half>(g, ws, slice_stride, cols_pad, plan.splits); break;
+            case Elem::BF16: rc = launch_reduce<__nv_bfloat16>(g, ws, slice_stride, cols_pad, plan.splits); break;
+        }
+    }
+    e = cudaFreeAsync(ws, g.stream);
+    if (e != cudaSuccess && rc == PEAK_OK) { set_cuda_error(e); rc = PEAK_ERR_CUDA; }
+    return rc;
 }
 
 }  // namespace
@@ -456,15 +688,18 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
     if (g.M >= (1ll << 31) - 512 || g.N >= (1ll << 31) - 512 || g.K >= (1ll << 31) - 512) return false;
     if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16) return false;
     if (g.lda % 8 || g.ldb % 8) return false;  // TMA: row pitch must be a multiple of 16 bytes
-    if (g.lda >= (1ll << 38) || g.ldb >= (1ll << 38)) return false;
-    const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 255) / 256);
-    if (tiles >= (1ll << 31)) return false;
+    if (g.lda >= (1ll << 38) || g.ldb >= (1ll << 38) || g.ldc >= (1ll << 38)) return false;
+    const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 127) / 128);
+    if (tiles * 16 >= (1ll << 31)) return false;
     return true;
 }
 
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
-    return cta_group == 2 ? dispatch_out<2>(g) : dispatch_out<1>(g);
+    const int units = sm_count() / cta_group;
+    const Plan plan = choose_plan(g, cta_group, units);
+    if (cta_group == 2) return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);
+    return plan.bn == 256 ? run_umma<1, 256>(g, plan, units) : run_umma<1, 128>(g, plan, units);
 }
 
 }  // namespace peak

@@ -210,3 +210,61 @@ def test_launch_counter_moves():
     dc = R.DeviceCase(W.config0())
     dc.run()
     assert P.peak_kernel_launches() == n0 + 1
+
+
+# ------------------------------------------------------------------ tuning knobs never change results
+@pytest.fixture
+def reset_tuning():
+    yield
+    for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE):
+        P.peak_set_tuning(key, 0)
+
+
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("epilogue", [1, 2])
+def test_umma_tile_width_epilogue_and_split_k(variant, tile_n, epilogue, reset_tuning):
+    """Tile width, epilogue store path and k-split are performance knobs: with integer inputs every
+    combination must give the oracle's correctly rounded result bit for bit (which also shows that a split
+    neither drops nor repeats a k-block), and with real inputs the tolerance checks must hold."""
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, tile_n)
+    P.peak_set_tuning(P.PEAK_TUNE_EPILOGUE, epilogue)
+    for split in (1, 2, 3, 5):
+        P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+        for idx, (dtype, ta, tb, M, N, K) in enumerate([(W.PEAK_BF16_BF16, 1, 0, 200, 328, 456),
+                                                       (W.PEAK_F16_F32, 0, 1, 300, 136, 520),
+                                                       (W.PEAK_BF16_F32, 0, 0, 16, 520, 640),
+                                                       (W.PEAK_F16_F16, 1, 1, 264, 256, 320)]):
+            ci = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.125, beta=-2.0, case=idx)
+            dc = R.DeviceCase(ci)
+            dc.run(variant)
+            ref, _ = dc.oracle_full()
+            want = oracle.round_to(R.OT[ci.out_type], ref)
+            got = dc.result()
+            got = got.view(np.uint32) if ci.out_type == "f32" else got
+            assert np.array_equal(got, want), f"{ci.name} tile_n={tile_n} epilogue={epilogue} split={split}"
+            cr = mk(dtype, ta, tb, M, N, K, alpha=0.5, beta=2.0, pad_c=8, case=idx)
+            dr = R.DeviceCase(cr)
+            dr.run(variant)
+            R.check_full(dr, what=f"{cr.name} tile_n={tile_n} epilogue={epilogue} split={split}")
+
+
+def test_auto_dispatch_skinny_shapes(reset_tuning):
+    """Shapes with few output tiles (the dispatcher may split K): results against the oracle, run twice
+    for bit-identical output (the split reduction is in a fixed order)."""
+    for (M, N, K) in [(16, 1024, 4096), (128, 1792, 2048), (40, 264, 8192)]:
+        c = mk(W.PEAK_BF16_BF16, 1, 0, M, N, K, alpha=0.5, beta=2.0, case=M)
+        dc = R.DeviceCase(c)
+        dc.run()
+        first = dc.result().copy()
+        R.check_full(dc)
+        dc.reset_c()
+        dc.run()
+        assert np.array_equal(first, dc.result())
+
+
+def test_set_tuning_rejects_bad_arguments():
+    with pytest.raises(P.PeakError):
+        P.peak_set_tuning(99, 1)
+    with pytest.raises(P.PeakError):
+        P.peak_set_tuning(P.PEAK_TUNE_TILE_N, -1)
