@@ -44,6 +44,7 @@
 #ifndef PEAK_GEMM_H
 #define PEAK_GEMM_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -66,7 +67,8 @@ typedef enum peak_status {
     PEAK_ERR_CUDA = 3,          /* a CUDA runtime / driver call failed; see peak_last_cuda_error() */
     PEAK_ERR_UNSUPPORTED = 4,   /* the forced variant cannot run this problem */
     PEAK_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up; reported by peak_check() */
-    PEAK_ERR_NO_MEMORY = 6      /* staging memory for the host-buffer call could not be allocated */
+    PEAK_ERR_NO_MEMORY = 6,     /* staging or workspace memory could not be allocated */
+    PEAK_ERR_WORKSPACE_TOO_SMALL = 7 /* peak_gemm_static_ws: the partial tiles do not fit the fixed workspace */
 } peak_status_t;
 
 /* Kernel families.  PEAK_VARIANT_AUTO lets the dispatcher choose. */
@@ -129,6 +131,39 @@ int peak_release_staging(void);
 int peak_gemm_xcheck_f64(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
                          const void *A, int64_t lda, const void *B, int64_t ldb, float beta, const void *C0,
                          int64_t ldc, double *Cref, int64_t ldcref, void *stream);
+
+/*
+ * peak_gemm_static_ws: split-K GEMM that allocates nothing.  (The paper has no counterpart: this entry
+ * point exists for callers, not for the method.)
+ *
+ * Who needs it: code that must not, or cannot, allocate device memory when it calls a GEMM -- a serving loop
+ * that has handed all free HBM to its own pools, a process whose memory is accounted for up front, a
+ * latency-critical path where an allocator call (which may take a lock or synchronise) is not acceptable.
+ * The ordinary split-K path of peak_gemm takes its fp32 partial tiles from a stream-ordered memory pool;
+ * this one keeps them in a fixed array that is part of the library image: peak_static_ws_bytes() bytes
+ * (32 MiB), held by every GPU that loads the library for as long as the process lives.
+ *
+ * Same operation, arguments, layout rules and epilogue as peak_gemm, for 16-bit inputs only, with K cut
+ * into `splits` slices (2 <= splits <= 64; every slice must get at least one 64-wide k-block) computed by
+ * 128 x 128 tensor-core tiles; the slices are added in slice order by a second kernel, so results are
+ * reproducible run to run.  A, B, C are device pointers; A and B need 16-byte aligned bases and pitches
+ * that are multiples of 8 elements (else PEAK_ERR_UNSUPPORTED).  Enqueues two kernels on `stream` and
+ * returns without synchronising.
+ *
+ * Limit: roundup(M,128) * roundup(N,128) * splits * 4 bytes must not exceed peak_static_ws_bytes();
+ * otherwise PEAK_ERR_WORKSPACE_TOO_SMALL is returned and nothing is launched.
+ *
+ * Makes no cudaMalloc / cudaFree / pool call and calls no allocating library routine.  The first call on
+ * each device looks up the array's device address (cudaGetSymbolAddress, cached per device); make that first
+ * call outside any stream capture.  All calls share the one array, and it keeps whatever the previous call
+ * left there; nothing in it needs clearing, because every cell the reduction reads is written by the
+ * tile kernel of the same call first.  Two calls that overlap on the GPU (different streams, no ordering
+ * between them) would overwrite each other's partial tiles: order them.
+ */
+int peak_gemm_static_ws(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                        const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc,
+                        int splits, void *stream);
+size_t peak_static_ws_bytes(void);
 
 /*
  * peak_query_variant: which kernel family peak_gemm would run for these arguments (a peak_variant_t),

@@ -12,7 +12,7 @@ import os
 
 PEAK_F16_F32, PEAK_BF16_BF16, PEAK_F32_F32, PEAK_F16_F16, PEAK_BF16_F32 = 0, 1, 2, 3, 4
 PEAK_OK, PEAK_ERR_INVALID_VALUE, PEAK_ERR_ARCH, PEAK_ERR_CUDA, PEAK_ERR_UNSUPPORTED, PEAK_ERR_TIMEOUT, \
-    PEAK_ERR_NO_MEMORY = range(7)
+    PEAK_ERR_NO_MEMORY, PEAK_ERR_WORKSPACE_TOO_SMALL = range(8)
 PEAK_VARIANT_AUTO, PEAK_VARIANT_FALLBACK, PEAK_VARIANT_UMMA_1CTA, PEAK_VARIANT_UMMA_2CTA, PEAK_VARIANT_SGEMM, \
     PEAK_VARIANT_SCALE, PEAK_VARIANT_NONE = range(7)
 
@@ -22,7 +22,7 @@ _lib = None
 
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
-           "peak_status_string", "peak_variant_string", "peak_version"]
+           "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes"]
 
 
 class PeakError(RuntimeError):
@@ -52,6 +52,10 @@ def load():
     lib.peak_gemm_variant.argtypes = [i] + gemm_args
     lib.peak_gemm_host.restype = i
     lib.peak_gemm_host.argtypes = gemm_args
+    lib.peak_gemm_static_ws.restype = i
+    lib.peak_gemm_static_ws.argtypes = gemm_args[:-1] + [i, vp]
+    lib.peak_static_ws_bytes.restype = ctypes.c_size_t
+    lib.peak_static_ws_bytes.argtypes = []
     lib.peak_release_staging.restype = i
     lib.peak_release_staging.argtypes = []
     lib.peak_gemm_xcheck_f64.restype = i
@@ -121,6 +125,18 @@ def peak_gemm_host(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, 
     rc = load().peak_gemm_host(dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda, _ptr(B), ldb, beta,
                                _ptr(C), ldc, _stream(stream))
     return _raise(rc, "peak_gemm_host") if check else rc
+
+
+def peak_gemm_static_ws(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, splits, stream=None,
+                        check=True):
+    """Split-K GEMM whose partial tiles live in the library's fixed 32 MiB array: no allocation at call time."""
+    rc = load().peak_gemm_static_ws(dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda, _ptr(B), ldb, beta,
+                                    _ptr(C), ldc, int(splits), _stream(stream))
+    return _raise(rc, "peak_gemm_static_ws") if check else rc
+
+
+def peak_static_ws_bytes() -> int:
+    return load().peak_static_ws_bytes()
 
 
 def peak_release_staging():

@@ -270,7 +270,8 @@ const char *peak_status_string(int status) {
         case PEAK_ERR_CUDA: return "CUDA call failed";
         case PEAK_ERR_UNSUPPORTED: return "variant does not support this problem";
         case PEAK_ERR_TIMEOUT: return "a bounded device-side wait gave up";
-        case PEAK_ERR_NO_MEMORY: return "out of device memory for staging";
+        case PEAK_ERR_NO_MEMORY: return "out of device memory for staging or workspace";
+        case PEAK_ERR_WORKSPACE_TOO_SMALL: return "partial tiles exceed the fixed workspace of peak_gemm_static_ws";
     }
     return "unknown status";
 }

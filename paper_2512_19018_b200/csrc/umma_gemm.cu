@@ -679,6 +679,52 @@ template <int CG, int BN> int run_umma(const GemmArgs &g, const Plan &plan, int 
     return rc;
 }
 
+
+// ---- split-K with a fixed, library-owned workspace (no allocation at call time) --------------------------
+// The partial tiles of peak_gemm_static_ws live in this array instead of in pool memory.  It is part of
+// the loaded module, so every GPU that loads the library holds these bytes until the process exits.
+constexpr size_t kStaticWsBytes = 32u << 20;  // 32 MiB
+static __device__ __align__(256) float g_static_ws[kStaticWsBytes / sizeof(float)];
+
+// Device address of g_static_ws on the current device.  In host code the array's name is only a handle
+// for the runtime, not a device address, so the address is asked for once per device (with that device
+// current) and cached.
+float *static_ws_address() {
+    static float *addr[64] = {};
+    static std::mutex m;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e); return nullptr; }
+    if (dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(m);
+    if (!addr[dev]) {
+        float *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_static_ws);
+        if (e != cudaSuccess) { set_cuda_error(e); return nullptr; }
+        addr[dev] = ptr;
+    }
+    return addr[dev];
+}
+
+// The split-K path of run_umma with the workspace passed in; 128 x 128 tiles, one CTA per tile slice.
+int run_umma_static_ws(const GemmArgs &g, int splits, float *ws) {
+    constexpr int CG = 1, BN = 128;
+    const Plan plan{BN, splits};
+    const int units = sm_count();
+    const int64_t rows_pad = ((g.M + BM * CG - 1) / (BM * CG)) * (BM * CG);
+    const int64_t cols_pad = ((g.N + BN - 1) / BN) * BN;
+    const int64_t slice_stride = rows_pad * cols_pad;
+    int rc = launch_kernel<CG, BN, float>(g, plan, units, ws, cols_pad, Elem::F32, slice_stride, (int)rows_pad, 1.0f,
+                                          0.0f);
+    if (rc != PEAK_OK) return rc;
+    switch (out_elem(g.dtype)) {
+        case Elem::F32: return launch_reduce<float>(g, ws, slice_stride, cols_pad, splits);
+        case Elem::F16: return launch_reduce<__half>(g, ws, slice_stride, cols_pad, splits);
+        case Elem::BF16: return launch_reduce<__nv_bfloat16>(g, ws, slice_stride, cols_pad, splits);
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
 }  // namespace
 
 bool umma_supports(const GemmArgs &g, int cta_group) {
@@ -703,3 +749,39 @@ int launch_umma(const GemmArgs &g, int cta_group) {
 }
 
 }  // namespace peak
+
+extern "C" {
+
+size_t peak_static_ws_bytes(void) { return peak::kStaticWsBytes; }
+
+int peak_gemm_static_ws(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+                        int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, int splits,
+                        void *stream) {
+    using namespace peak;
+    set_cuda_error(cudaSuccess);
+    // arguments first: nothing is launched or written on an error
+    if (dtype != PEAK_F16_F32 && dtype != PEAK_BF16_BF16 && dtype != PEAK_F16_F16 && dtype != PEAK_BF16_F32)
+        return PEAK_ERR_INVALID_VALUE;  // 16-bit inputs only: this is the tensor-core path
+    if ((transA != 0 && transA != 1) || (transB != 0 && transB != 1)) return PEAK_ERR_INVALID_VALUE;
+    if (M < 1 || N < 1 || K < 1 || !A || !B || !C) return PEAK_ERR_INVALID_VALUE;
+    if (lda < (transA ? M : K) || ldb < (transB ? K : N) || ldc < N) return PEAK_ERR_INVALID_VALUE;
+    const int64_t num_kb = (K + BK - 1) / BK;
+    if (splits < 2 || splits > 64) return PEAK_ERR_INVALID_VALUE;
+    const int64_t kbps = (num_kb + splits - 1) / splits;
+    if (splits > num_kb || kbps * (splits - 1) >= num_kb) return PEAK_ERR_INVALID_VALUE;  // a slice would be empty
+    GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, C, lda, ldb, ldc, (cudaStream_t)stream};
+    if (!umma_supports(g, 1)) return PEAK_ERR_UNSUPPORTED;
+    const int64_t rows_pad = ((M + 127) / 128) * 128, cols_pad = ((N + 127) / 128) * 128;
+    if ((double)rows_pad * (double)cols_pad * (double)splits * sizeof(float) > (double)kStaticWsBytes)
+        return PEAK_ERR_WORKSPACE_TOO_SMALL;
+    int major = 0, dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (major != 10) return PEAK_ERR_ARCH;
+    float *ws = static_ws_address();
+    if (!ws) return PEAK_ERR_CUDA;
+    return run_umma_static_ws(g, splits, ws);
+}
+
+}  // extern "C"
