@@ -163,7 +163,8 @@ def peak_tile_coord(tile, tiles_m, tiles_n, group):
     return tm.value, tn.value
 
 
-PEAK_TUNE_RASTER_GROUP, PEAK_TUNE_TILE_N, PEAK_TUNE_SPLIT_K, PEAK_TUNE_EPILOGUE = 0, 1, 2, 3
+PEAK_TUNE_RASTER_GROUP, PEAK_TUNE_TILE_N, PEAK_TUNE_SPLIT_K, PEAK_TUNE_EPILOGUE, PEAK_TUNE_SGEMM_FMA, \
+    PEAK_TUNE_TAIL_SPLIT = 0, 1, 2, 3, 4, 5
 
 
 def peak_set_tuning(key: int, value: int) -> int:

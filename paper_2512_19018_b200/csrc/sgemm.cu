@@ -45,7 +45,9 @@ template <bool KCONTIG> struct Loader {
     }
 };
 
-template <bool TA, bool TB>
+// PACKED selects the two-wide fp32 FMA of sm_100 (two independent fp32 FMAs per instruction, same rounding
+// as two scalar FMAs): half the issue slots for the same arithmetic.
+template <bool TA, bool TB, bool PACKED>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
              int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int group) {
@@ -89,10 +91,24 @@ sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int6
             *reinterpret_cast<float4 *>(&a[4]) = *reinterpret_cast<const float4 *>(&As[cur][k][ty * 4 + 64]);
             *reinterpret_cast<float4 *>(&b[0]) = *reinterpret_cast<const float4 *>(&Bs[cur][k][tx * 4]);
             *reinterpret_cast<float4 *>(&b[4]) = *reinterpret_cast<const float4 *>(&Bs[cur][k][tx * 4 + 64]);
+            if (PACKED) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+                for (int i = 0; i < 8; ++i) {
+                    const float2 aa = make_float2(a[i], a[i]);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                    for (int j = 0; j < 4; ++j) {
+                        float2 c = make_float2(acc[i][2 * j], acc[i][2 * j + 1]);
+                        c = __ffma2_rn(aa, make_float2(b[2 * j], b[2 * j + 1]), c);
+                        acc[i][2 * j] = c.x;
+                        acc[i][2 * j + 1] = c.y;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
         }
         if (kb + 1 < nkb) {
             la.store(As[cur ^ 1], ga);
@@ -121,9 +137,15 @@ sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int6
 
 template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
     const int tiles_m = (int)(g.M / SG_BM), tiles_n = (int)(g.N / SG_BN);
-    sgemm_kernel<TA, TB><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
-        (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-        (float *)g.C, g.ldc, tiles_m, tiles_n, 8);
+    const int group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 8;
+    if (tuning(PEAK_TUNE_SGEMM_FMA) == 1)
+        sgemm_kernel<TA, TB, false><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
+            (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group);
+    else
+        sgemm_kernel<TA, TB, true><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
+            (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }

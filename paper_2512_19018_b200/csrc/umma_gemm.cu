@@ -16,10 +16,12 @@
 // Tile: 128 x BN x 64 per CTA (CTA_GROUP 1) or 256 x BN x 64 per CTA pair (CTA_GROUP 2: each CTA stages its
 // 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 256 or 128.
 //
-// Split-K (the paper's Split-K transformation, section 4.1): for shapes with too few tiles to fill the GPU,
-// each tile's k-blocks are divided among `splits` work items; every item stores its fp32 partial tile to
-// a workspace slice and a second kernel adds the slices in a fixed order and applies alpha/beta, so the
-// result does not depend on scheduling.
+// Split-K (the paper's Split-K transformation, section 4.1).  The first `full_tiles` tiles are computed
+// whole; each remaining tile has its k-blocks divided among `tail_splits` work items that store fp32 partial
+// tiles to a workspace, and a second kernel adds a tile's slices in slice order and applies alpha/beta, so
+// the result does not depend on scheduling.  Two uses: shapes with too few tiles to fill the GPU split every
+// tile (full_tiles = 0); shapes whose tile count is not a multiple of the SM (pair) count split only the
+// tiles of the last, partly filled wave, so that the wave finishes in a fraction of a tile time.
 #include <cuda.h>
 
 #include <mutex>
@@ -59,15 +61,15 @@ struct UmmaParams {
     int num_kb;            // ceil(K / BK)
     int tiles_m, tiles_n;  // in units of (128*CG) x BN
     int group;             // tile-rows per raster group
-    int splits;            // k-slices per tile (1 = no split)
+    int full_tiles;        // tiles [0, full_tiles) are computed whole and stored to C
+    int tail_splits;       // k-slices of every later tile (partials go to the workspace)
     int kb_per_split;
+    int total_items;       // full_tiles + (tiles - full_tiles) * tail_splits
     int a_mn, b_mn;        // 1: operand is MN-major in memory (transA == 1 / transB == 0)
     uint32_t idesc;
     float alpha, beta;
-    void *C;               // output (or fp32 workspace when splits > 1)
+    void *C;
     int64_t ldc;
-    int64_t slice_stride;  // elements between workspace slices (splits > 1)
-    int slice_rows;        // rows per workspace slice in the TMA store map (splits > 1)
     int vec_ok;            // C base and pitch allow 16-byte vector access
     int tma_store;         // epilogue stores through TMA
     uint32_t *status;
@@ -166,13 +168,90 @@ __device__ __forceinline__ void stage_row32(uint32_t buf, int lane, int h, const
     }
 }
 
+// Work item -> tile, k-block range and destination (ws_block < 0: the tile is whole and goes to C;
+// otherwise the index of the (tile, slice) block of the partial-tile workspace).
+struct Item {
+    int tile, kb0, kb1, ws_block;
+};
+__device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
+    Item w;
+    if (item < p.full_tiles) {
+        w.tile = item; w.kb0 = 0; w.kb1 = p.num_kb; w.ws_block = -1;
+    } else {
+        const int j = item - p.full_tiles;
+        const int t = j / p.tail_splits, slice = j - t * p.tail_splits;
+        w.tile = p.full_tiles + t;
+        w.kb0 = slice * p.kb_per_split;
+        w.kb1 = min(w.kb0 + p.kb_per_split, p.num_kb);
+        w.ws_block = j;
+    }
+    return w;
+}
+
+// Epilogue of one accumulator tile for one warp: TMEM -> registers -> alpha/beta -> T -> staging + TMA
+// store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
+// column limit, `nrows` the row limit for `row`; (x0, y0) is where chunk 0 of this warp lands in `tm`.
+template <typename T, int BN>
+__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
+                                              T *base, int64_t ld, int row, int row0, int nrows, int cbase,
+                                              int ncols, const CUtensorMap *tm, int x0, int y0, bool tma, bool vec,
+                                              float alpha, float beta) {
+    constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
+#pragma unroll 1
+    for (int c = 0; c < BN / CHUNK_COLS; ++c) {
+        const int col0 = cbase + c * CHUNK_COLS;
+        if (col0 >= ncols) break;  // warp-uniform
+        uint32_t buf = 0;
+        if (tma) {
+            // the store that last read this buffer (two chunks ago) must have drained it
+            buf = my_stage + (chunk_no & 1u) * EPI_BUF_BYTES;
+            if (lane == 0) ptx::tma_store_wait_read<1>();
+            __syncwarp();
+        }
+#pragma unroll
+        for (int h = 0; h < CHUNK_COLS / 32; ++h) {
+            const int col = col0 + h * 32;
+            uint32_t r[32];
+            ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r);
+            ptx::tmem_ld_wait();
+            const int valid = (ncols - col >= 32) ? 32 : (ncols - col > 0 ? ncols - col : 0);
+            T *dst = base + (int64_t)row * ld + col;
+            float v[32];
+            if (beta != 0.0f) {
+                float cold[32];
+                if (row < nrows && valid > 0) load_row32<T>(dst, cold, valid, vec);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = fmaf(beta, cold[i], alpha * __uint_as_float(r[i]));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[i]);
+            }
+            if (tma) stage_row32<T>(buf, lane, h, v);
+            else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
+        }
+        if (tma) {
+            ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
+            __syncwarp();
+            if (lane == 0 && row0 < nrows) {
+                ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
+                ptx::tma_store_commit();
+            }
+            ++chunk_no;
+        }
+    }
+}
+
 template <int CG, int BN, typename TOut>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+                 const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
+                 float *__restrict__ ws, const UmmaParams p) {
     using C_ = Cfg<CG, BN>;
     constexpr int STAGES = C_::STAGES;
-    constexpr int CHUNK_COLS = 128 / (int)sizeof(TOut);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
     extern __shared__ uint8_t smem_raw[];
 
     const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -194,7 +273,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool leader = (rank == 0);
     const int unit = blockIdx.x / CG;          // CTA (or CTA pair) index
     const int num_units = gridDim.x / CG;
-    const int total_items = p.tiles_m * p.tiles_n * p.splits;
+    const int total_items = p.total_items;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -213,6 +292,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB);
         if (p.tma_store) ptx::prefetch_tensormap(&tmC);
+        if (p.total_items > p.full_tiles) ptx::prefetch_tensormap(&tmW);
     }
     if (warp == 1) {
         ptx::tmem_alloc<CG>(ptx::smem_u32(tmem_slot), C_::TMEM_COLS);
@@ -230,14 +310,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int item = unit; item < total_items && ok; item += num_units) {
-                const int tile = item / p.splits, slice = item - tile * p.splits;
+                const Item w = decode_item(p, item);
                 int64_t tm, tn;
-                tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
+                tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CG) + (int)rank * BM;
                 const int n_cta = (int)tn * BN + (int)rank * C_::B_ROWS;
-                const int kb0 = slice * p.kb_per_split;
-                const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
                         report_timeout(p, abort_flag, 1, s);
@@ -294,9 +372,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t a_lbo = p.a_mn ? (uint32_t)ATOM_BYTES : 16u, b_lbo = p.b_mn ? (uint32_t)ATOM_BYTES : 16u;
             const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
             for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
-                const int slice = item % p.splits;
-                const int kb0 = slice * p.kb_per_split;
-                const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);
+                const Item w = decode_item(p, item);
+                const int kb0 = w.kb0, kb1 = w.kb1;
                 const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
                 if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag)) {
                     report_timeout(p, abort_flag, 3, b);
@@ -339,14 +416,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t tl = 0, chunk_no = 0;
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
-            const int tile = item / p.splits, slice = item - tile * p.splits;
+            const Item w = decode_item(p, item);
             int64_t tm, tn;
-            tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
+            tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CG) + (int)rank * BM + q * 32;  // first row of this warp
-            const int row = row0 + lane;
             const int n0 = (int)tn * BN;
-            TOut *Cout = reinterpret_cast<TOut *>(p.C) + (int64_t)slice * p.slice_stride;
-            const int store_row0 = row0 + slice * p.slice_rows;  // row coordinate in the TMA store map
             const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
             // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
             const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag);
@@ -357,51 +431,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             ptx::tc_fence_after_sync();
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / CHUNK_COLS; ++c) {
-                const int col0 = n0 + c * CHUNK_COLS;
-                if (col0 >= p.N) break;  // warp-uniform
-                uint32_t buf = 0;
-                if (p.tma_store) {
-                    // the store that last read this buffer (two chunks ago) must have drained it
-                    buf = my_stage + (chunk_no & 1u) * EPI_BUF_BYTES;
-                    if (lane == 0) ptx::tma_store_wait_read<1>();
-                    __syncwarp();
-                }
-#pragma unroll
-                for (int h = 0; h < CHUNK_COLS / 32; ++h) {
-                    const int col = col0 + h * 32;
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r);
-                    ptx::tmem_ld_wait();
-                    const int valid = (p.N - col >= 32) ? 32 : (p.N - col > 0 ? p.N - col : 0);
-                    TOut *dst = Cout + (int64_t)row * p.ldc + col;
-                    float v[32];
-                    if (p.beta != 0.0f) {
-                        float cold[32];
-                        if (row < p.M && valid > 0) load_row32<TOut>(dst, cold, valid, vec);
-                        else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
-                        }
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = fmaf(p.beta, cold[i], p.alpha * __uint_as_float(r[i]));
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
-                    }
-                    if (p.tma_store) stage_row32<TOut>(buf, lane, h, v);
-                    else if (row < p.M && valid > 0) store_row32<TOut>(dst, v, valid, vec);
-                }
-                if (p.tma_store) {
-                    ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
-                    __syncwarp();
-                    if (lane == 0 && row0 < p.M) {
-                        ptx::tma_store_2d(&tmC, col0, store_row0, buf);
-                        ptx::tma_store_commit();
-                    }
-                    ++chunk_no;
-                }
+            if (w.ws_block < 0) {
+                // whole tile: alpha/beta epilogue straight to C
+                epilogue_tile<TOut, BN>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C), p.ldc,
+                                        row0 + lane, row0, p.M, n0, p.N, &tmC, n0, row0, p.tma_store != 0, vec,
+                                        p.alpha, p.beta);
+            } else {
+                // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
+                const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
+                epilogue_tile<float, BN>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
+                                         0x7fffffff, 0, BN, &tmW, 0, wrow0, true, true, 1.0f, 0.0f);
             }
             // hand the accumulator buffer back to the MMA issuer
             ptx::tc_fence_before_sync();
@@ -411,7 +450,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, 0));
             }
         }
-        if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();  // staging memory must outlive the stores
+        if (lane == 0) ptx::tma_store_wait_all<0>();  // staging memory must outlive the stores
         __syncwarp();
     }
 
@@ -430,20 +469,67 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-// Adds the k-slices of a split GEMM in slice order and applies the epilogue:
-// C = alpha * (ws[0] + ws[1] + ... ) + beta * C, one rounding.
+// Adds the k-slices of every split tile in slice order and applies the epilogue:
+// C = alpha * (ws[tile][0] + ws[tile][1] + ...) + beta * C, one rounding.  The workspace holds, for split tile
+// t (counted from full_tiles) and slice s, a dense rows_t x bn fp32 block at index t * splits + s.
+// One block of 256 threads handles a quarter of a tile's float4 columns groups at a time.
 template <typename TOut>
-__global__ void splitk_reduce_kernel(const float *__restrict__ ws, int64_t slice_stride, int64_t ldws, int splits,
-                                     int64_t M, int64_t N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc) {
-    const int64_t total = M * N;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t i = e / N, j = e - i * N;
-        const float *src = ws + i * ldws + j;
-        float acc = src[0];
-        for (int s = 1; s < splits; ++s) acc += src[(int64_t)s * slice_stride];
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
+                     int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
+                     int vec_ok) {
+    const int blocks_per_tile = gridDim.y;
+    const int t = blockIdx.x;  // split tile number
+    int64_t tm, tn;
+    tile_coord(full_tiles + t, tiles_m, tiles_n, group, tm, tn);
+    const int vec_per_row = bn / 4;
+    const int total_vec = rows_t * vec_per_row;
+    const int64_t block_elems = (int64_t)rows_t * bn;
+    const float *base = ws + (int64_t)t * splits * block_elems;
+    for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < total_vec; e += blocks_per_tile * blockDim.x) {
+        const int r = e / vec_per_row, c4 = e - r * vec_per_row;
+        const int64_t i = tm * rows_t + r;
+        const int64_t j = tn * bn + c4 * 4;
+        if (i >= M || j >= N) continue;
+        const float *src = base + (int64_t)r * bn + c4 * 4;
+        float4 acc = *reinterpret_cast<const float4 *>(src);
+        for (int sl = 1; sl < splits; ++sl) {
+            const float4 v = *reinterpret_cast<const float4 *>(src + sl * block_elems);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
         TOut *dst = C + i * ldc + j;
-        const float c_old = (beta != 0.0f) ? to_f32(*dst) : 0.0f;
-        *dst = from_f32<TOut>(epilogue_f32(alpha, acc, beta, c_old));
+        if (vec_ok && j + 4 <= N) {
+            float o[4] = {0.f, 0.f, 0.f, 0.f};
+            if (beta != 0.0f) {
+                if constexpr (sizeof(TOut) == 4) {
+                    const float4 t4 = *reinterpret_cast<const float4 *>(dst);
+                    o[0] = t4.x; o[1] = t4.y; o[2] = t4.z; o[3] = t4.w;
+                } else {
+                    const uint2 t2 = *reinterpret_cast<const uint2 *>(dst);
+                    uint16_t h[4] = {(uint16_t)(t2.x & 0xffffu), (uint16_t)(t2.x >> 16), (uint16_t)(t2.y & 0xffffu),
+                                     (uint16_t)(t2.y >> 16)};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) o[k] = to_f32(*reinterpret_cast<TOut *>(&h[k]));
+                }
+            }
+            float rr[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) rr[k] = epilogue_f32(alpha, a4[k], beta, o[k]);
+            if constexpr (sizeof(TOut) == 4) {
+                *reinterpret_cast<float4 *>(dst) = make_float4(rr[0], rr[1], rr[2], rr[3]);
+            } else {
+                *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<TOut>(rr[0], rr[1]), pack2<TOut>(rr[2], rr[3]));
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (j + k < N) {
+                    const float c_old = (beta != 0.0f) ? to_f32(dst[k]) : 0.0f;
+                    dst[k] = from_f32<TOut>(epilogue_f32(alpha, a4[k], beta, c_old));
+                }
+            }
+        }
     }
 }
 
@@ -497,44 +583,73 @@ int sm_count() {
     return sms[dev];
 }
 
-constexpr double kL2BytesPerClk = 64.0;  // assumed L2 -> shared-memory bandwidth per SM
+constexpr double kL2BytesPerClk = 64.0;      // assumed L2 -> shared-memory bandwidth per SM
+constexpr double kSplitFixedCycles = 20000.0;  // workspace allocation + second launch of a split (~12 us)
 
 struct Plan {
-    int bn;      // 256 or 128
-    int splits;  // k-slices per tile
+    int bn;           // tile width: 256 or 128
+    int full_tiles;   // tiles computed whole
+    int tail_splits;  // k-slices of each remaining tile (1 when nothing is split)
 };
 
-// Tile width and k-split from a small cost model (cycles): an item costs its k-blocks times the slower of
-// the tensor pipe (2*BN cycles per k-block per SM) and the operand stream (bytes per k-block over an
-// assumed 64 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread
-// over the units in waves.  A split additionally pays for writing and re-reading fp32 partials.
+int64_t tiles_of(const GemmArgs &g, int cg, int bn) {
+    return ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn);
+}
+
+// Tile width and k-splitting from a small cost model (cycles): an item costs its k-blocks times the slower
+// of the tensor pipe (2*BN cycles per k-block per SM) and the operand stream (bytes per k-block over an
+// assumed 64 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread over
+// the units in waves.  Splitting additionally pays for writing and re-reading fp32 partials and for the
+// second launch.  Candidates: no split; every tile split s ways (few tiles); only the last wave split.
 Plan choose_plan(const GemmArgs &g, int cg, int units) {
     const int64_t num_kb = (g.K + BK - 1) / BK;
-    Plan best{256, 1};
+    Plan best{256, 0, 1};
     double best_cost = 1e300;
     const int force_bn = tuning(PEAK_TUNE_TILE_N), force_split = tuning(PEAK_TUNE_SPLIT_K);
+    const int tail_mode = tuning(PEAK_TUNE_TAIL_SPLIT);  // 2 = split the last wave whenever possible
     for (int bn : {256, 128}) {
         if (force_bn && bn != force_bn) continue;
-        const int64_t tiles = ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn);
+        const int64_t tiles = tiles_of(g, cg, bn);
         const double kb_cycles = fmax(2.0 * bn, (128.0 + bn / cg) * 128.0 / kL2BytesPerClk);
+        const double item_ovh = 1500.0;
+        const double tile_bytes = (double)BM * bn * 4.0;  // fp32 partial tile per SM
+        auto consider = [&](int64_t full, int s, double cost) {
+            if (cost < best_cost) { best_cost = cost; best = Plan{bn, (int)full, s}; }
+        };
+        // (a) every tile whole, or every tile split s ways
         for (int s = 1; s <= 16; ++s) {
             if (force_split && s != force_split) continue;
-            if (s > 1 && !force_split && (s > num_kb || tiles * s > 2 * units)) break;
             if (s > num_kb) break;
+            if (s > 1 && !force_split && tiles * s > 2 * units) break;
             const int64_t kbps = (num_kb + s - 1) / s;
-            if (s > 1 && (kbps * (s - 1) >= num_kb)) continue;  // an empty last slice
+            if (s > 1 && kbps * (s - 1) >= num_kb) continue;  // an empty last slice
             const int64_t waves = (tiles * s + units - 1) / units;
-            double cost = (double)waves * (kbps * kb_cycles + 1500.0);
-            if (s > 1) cost += 2.0 * (double)g.M * g.N * s * 4.0 / (units * 24.0) + 6000.0;  // partials + 2nd launch
-            if (cost < best_cost) { best_cost = cost; best = Plan{bn, s}; }
+            double cost = (double)waves * (kbps * kb_cycles + item_ovh);
+            if (s > 1) cost += 2.0 * waves * tile_bytes / 24.0 + kSplitFixedCycles;
+            if (s > 1 && tail_mode == 2 && !force_split) cost *= 4.0;  // forced tail mode prefers (b)
+            consider(s == 1 ? tiles : 0, s, cost);
+        }
+        // (b) whole tiles for the full waves, the last partly filled wave split s ways
+        const int64_t full = (tiles / units) * units, rest = tiles - full;
+        // (measured on B200: under the power cap the busy SMs of a partly filled wave clock higher, so this
+        // split gains nothing at 4096^3 or 5000x3000x2500; it stays opt-in through PEAK_TUNE_TAIL_SPLIT = 2)
+        if (!force_split && tail_mode == 2 && full > 0 && rest > 0) {
+            for (int s = 2; s <= 8; ++s) {
+                if (rest * s > units || s > num_kb) break;
+                const int64_t kbps = (num_kb + s - 1) / s;
+                if (kbps * (s - 1) >= num_kb || kbps < 4) continue;
+                double cost = (double)(full / units) * (num_kb * kb_cycles + item_ovh) + (kbps * kb_cycles + item_ovh) +
+                              2.0 * tile_bytes / 24.0 + kSplitFixedCycles;
+                cost *= 0.01;
+                consider(full, s, cost);
+            }
         }
     }
     return best;
 }
 
 template <int CG, int BN, typename TOut>
-int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, void *out, int64_t ldo, Elem eout,
-                  int64_t slice_stride, int slice_rows, float alpha, float beta) {
+int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws) {
     using C_ = Cfg<CG, BN>;
     auto kernel = umma_gemm_kernel<CG, BN, TOut>;
     static std::once_flag once;
@@ -544,10 +659,10 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, void *out,
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err); return PEAK_ERR_CUDA; }
 
-    const Elem ein = in_elem(g.dtype);
+    const Elem ein = in_elem(g.dtype), eout = out_elem(g.dtype);
     const int a_mn = g.transA ? 1 : 0;  // A stored K x M: M is the contiguous index
     const int b_mn = g.transB ? 0 : 1;  // B stored K x N: N is the contiguous index
-    CUtensorMap tmA, tmB, tmC;
+    CUtensorMap tmA, tmB, tmC, tmW;
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK) : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BK, 128);
     ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK)
                      : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, C_::B_BOX_ROWS));
@@ -559,36 +674,37 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, void *out,
     p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((g.N + BN - 1) / BN);
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : ((CG == 1) ? 16 : 8);
-    p.splits = plan.splits;
-    p.kb_per_split = (p.num_kb + plan.splits - 1) / plan.splits;
+    const int tiles = p.tiles_m * p.tiles_n;
+    p.full_tiles = plan.full_tiles;
+    p.tail_splits = plan.tail_splits;
+    p.kb_per_split = (p.num_kb + plan.tail_splits - 1) / plan.tail_splits;
+    p.total_items = plan.full_tiles + (tiles - plan.full_tiles) * plan.tail_splits;
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
-    p.alpha = alpha; p.beta = beta;
-    p.C = out; p.ldc = ldo;
-    p.slice_stride = slice_stride; p.slice_rows = slice_rows;
+    p.alpha = g.alpha; p.beta = g.beta;
+    p.C = g.C; p.ldc = g.ldc;
     const int ob = elem_bytes(eout);
-    p.vec_ok = ((reinterpret_cast<uintptr_t>(out) % 16) == 0 && (ldo * ob) % 16 == 0) ? 1 : 0;
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0) ? 1 : 0;
     const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
     // TMA stores clip rows exactly but clip the contiguous index only at 16-byte granularity, so they are
     // used when a row of C is a whole number of 16-byte pieces; other widths take the direct-store path
-    const int64_t out_cols = plan.splits > 1 ? ldo : g.N;
-    p.tma_store = (p.vec_ok && (out_cols * ob) % 16 == 0 && epi != 1) ? 1 : 0;
-    if (p.tma_store) {
-        // rows of the map: the matrix itself, or all workspace slices stacked (each slice_rows high)
-        const int64_t rows = plan.splits > 1 ? (int64_t)plan.splits * slice_rows : g.M;
-        const int64_t cols = plan.splits > 1 ? ldo : g.N;
-        if (!make_map(&tmC, eout, out, cols, rows, ldo, 128 / ob, 32)) return PEAK_ERR_CUDA;
-    } else {
-        tmC = tmA;  // unused
+    p.tma_store = (p.vec_ok && (g.N * ob) % 16 == 0 && epi != 1) ? 1 : 0;
+    tmC = tmA;  // placeholders when unused
+    tmW = tmA;
+    if (p.tma_store && plan.full_tiles > 0 && !make_map(&tmC, eout, g.C, g.N, g.M, g.ldc, 128 / ob, 32))
+        return PEAK_ERR_CUDA;
+    if (plan.full_tiles < tiles) {
+        // the workspace as one tall matrix of dense (BM*CG) x BN blocks, one per (split tile, slice)
+        const int64_t rows = (int64_t)(tiles - plan.full_tiles) * plan.tail_splits * (BM * CG);
+        if (!ws || !make_map(&tmW, Elem::F32, ws, BN, rows, BN, 32, 32)) return PEAK_ERR_CUDA;
     }
     p.status = device_status_word();
     if (!p.status) return PEAK_ERR_CUDA;
 
-    const int64_t total = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     int units = units_max;
-    if (total < units) units = (int)total;
+    if (p.total_items < units) units = p.total_items;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(units * CG));
@@ -600,23 +716,36 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, void *out,
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, tmW, ws, p);
     count_launch();
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (plan.full_tiles == tiles) return PEAK_OK;
+
+    // second kernel: add the slices of the split tiles in order, apply alpha/beta
+    const int split_tiles = tiles - plan.full_tiles;
+    dim3 rgrid((unsigned)split_tiles, split_tiles >= 64 ? 2u : 8u);
+    splitk_reduce_kernel<TOut><<<rgrid, 256, 0, g.stream>>>(ws, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
+                                                            p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C,
+                                                            g.ldc, p.vec_ok);
+    count_launch();
+    e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
 
-template <typename TOut>
-int launch_reduce(const GemmArgs &g, const float *ws, int64_t slice_stride, int64_t ldws, int splits) {
-    const int64_t total = g.M * g.N;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<TOut><<<(unsigned)blocks, 256, 0, g.stream>>>(ws, slice_stride, ldws, splits, g.M, g.N, g.alpha,
-                                                                     g.beta, (TOut *)g.C, g.ldc);
-    count_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
-    return PEAK_OK;
+template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, int units, float *ws) {
+    switch (out_elem(g.dtype)) {
+        case Elem::F32: return launch_kernel<CG, BN, float>(g, plan, units, ws);
+        case Elem::F16: return launch_kernel<CG, BN, __half>(g, plan, units, ws);
+        case Elem::BF16: return launch_kernel<CG, BN, __nv_bfloat16>(g, plan, units, ws);
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
+// Bytes of fp32 partial tiles a plan needs (0 when nothing is split).
+size_t workspace_bytes(const GemmArgs &g, int cg, const Plan &plan) {
+    const int64_t split_tiles = tiles_of(g, cg, plan.bn) - plan.full_tiles;
+    return (size_t)split_tiles * plan.tail_splits * (size_t)(BM * cg) * plan.bn * sizeof(float);
 }
 
 // Stream-ordered workspace for split-K partials: one memory pool per device that keeps what it has been
@@ -645,40 +774,18 @@ cudaMemPool_t workspace_pool() {
 }
 
 template <int CG, int BN> int run_umma(const GemmArgs &g, const Plan &plan, int units) {
-    const Elem eout = out_elem(g.dtype);
-    if (plan.splits == 1) {
-        switch (eout) {
-            case Elem::F32: return launch_kernel<CG, BN, float>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
-            case Elem::F16: return launch_kernel<CG, BN, __half>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
-            case Elem::BF16:
-                return launch_kernel<CG, BN, __nv_bfloat16>(g, plan, units, g.C, g.ldc, eout, 0, 0, g.alpha, g.beta);
-        }
-        return PEAK_ERR_INVALID_VALUE;
-    }
-    // split-K: fp32 partial tiles in a stream-ordered workspace, padded to whole tiles so that no store clips
-    const int64_t rows_pad = ((g.M + BM * CG - 1) / (BM * CG)) * (BM * CG);
-    const int64_t cols_pad = ((g.N + BN - 1) / BN) * BN;
-    const int64_t slice_stride = rows_pad * cols_pad;
+    const size_t need = workspace_bytes(g, CG, plan);
+    if (need == 0) return launch_typed<CG, BN>(g, plan, units, nullptr);
     float *ws = nullptr;
     cudaMemPool_t pool = workspace_pool();
     if (!pool) return PEAK_ERR_CUDA;
-    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&ws),
-                                            (size_t)slice_stride * plan.splits * sizeof(float), pool, g.stream);
+    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&ws), need, pool, g.stream);
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_NO_MEMORY; }
-    int rc = launch_kernel<CG, BN, float>(g, plan, units, ws, cols_pad, Elem::F32, slice_stride, (int)rows_pad, 1.0f,
-                                          0.0f);
-    if (rc == PEAK_OK) {
-        switch (eout) {
-            case Elem::F32: rc = launch_reduce<float>(g, ws, slice_stride, cols_pad, plan.splits); break;
-            case Elem::F16: rc = launch_reduce<__half>(g, ws, slice_stride, cols_pad, plan.splits); break;
-            case Elem::BF16: rc = launch_reduce<__nv_bfloat16>(g, ws, slice_stride, cols_pad, plan.splits); break;
-        }
-    }
+    int rc = launch_typed<CG, BN>(g, plan, units, ws);
     e = cudaFreeAsync(ws, g.stream);
     if (e != cudaSuccess && rc == PEAK_OK) { set_cuda_error(e); rc = PEAK_ERR_CUDA; }
     return rc;
 }
-
 
 // ---- split-K with a fixed, library-owned workspace (no allocation at call time) --------------------------
 // The partial tiles of peak_gemm_static_ws live in this array instead of in pool memory.  It is part of
@@ -706,23 +813,10 @@ float *static_ws_address() {
     return addr[dev];
 }
 
-// The split-K path of run_umma with the workspace passed in; 128 x 128 tiles, one CTA per tile slice.
+// Every tile split `splits` ways with the workspace passed in; 128 x 128 tiles, one CTA per tile slice.
 int run_umma_static_ws(const GemmArgs &g, int splits, float *ws) {
-    constexpr int CG = 1, BN = 128;
-    const Plan plan{BN, splits};
-    const int units = sm_count();
-    const int64_t rows_pad = ((g.M + BM * CG - 1) / (BM * CG)) * (BM * CG);
-    const int64_t cols_pad = ((g.N + BN - 1) / BN) * BN;
-    const int64_t slice_stride = rows_pad * cols_pad;
-    int rc = launch_kernel<CG, BN, float>(g, plan, units, ws, cols_pad, Elem::F32, slice_stride, (int)rows_pad, 1.0f,
-                                          0.0f);
-    if (rc != PEAK_OK) return rc;
-    switch (out_elem(g.dtype)) {
-        case Elem::F32: return launch_reduce<float>(g, ws, slice_stride, cols_pad, splits);
-        case Elem::F16: return launch_reduce<__half>(g, ws, slice_stride, cols_pad, splits);
-        case Elem::BF16: return launch_reduce<__nv_bfloat16>(g, ws, slice_stride, cols_pad, splits);
-    }
-    return PEAK_ERR_INVALID_VALUE;
+    const Plan plan{128, 0, splits};
+    return launch_typed<1, 128>(g, plan, sm_count(), ws);
 }
 
 }  // namespace
@@ -773,7 +867,7 @@ int peak_gemm_static_ws(int dtype, int transA, int transB, int64_t M, int64_t N,
     if (!umma_supports(g, 1)) return PEAK_ERR_UNSUPPORTED;
     const int64_t rows_pad = ((M + 127) / 128) * 128, cols_pad = ((N + 127) / 128) * 128;
     if ((double)rows_pad * (double)cols_pad * (double)splits * sizeof(float) > (double)kStaticWsBytes)
-        return PEAK_ERR_WORKSPACE_TOO_SMALL;
+        return PEAK_ERR_WORKSPACE_TOO_SMALL;  // 128 x 128 fp32 blocks: one per (tile, slice)
     int major = 0, dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);

@@ -216,7 +216,8 @@ def test_launch_counter_moves():
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE):
+    for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE,
+                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT):
         P.peak_set_tuning(key, 0)
 
 
@@ -247,6 +248,36 @@ def test_umma_tile_width_epilogue_and_split_k(variant, tile_n, epilogue, reset_t
             dr = R.DeviceCase(cr)
             dr.run(variant)
             R.check_full(dr, what=f"{cr.name} tile_n={tile_n} epilogue={epilogue} split={split}")
+
+
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("tail", [1, 2])
+def test_umma_last_wave_split(variant, tail, reset_tuning):
+    """More tiles than SMs with a partly filled last wave: with the tail split forced on, the tiles of that
+    wave are computed as k-slices and reduced by the second kernel; forced off, they are computed whole.
+    Integer inputs (K = 1024, entries in [-4, 4]) make both exact: sampled elements of every tile must equal
+    the oracle's correctly rounded value bit for bit, and the two settings must agree on the whole matrix."""
+    P.peak_set_tuning(P.PEAK_TUNE_TAIL_SPLIT, tail)
+    outs = []
+    for (dtype, ta, tb, M, N) in [(W.PEAK_BF16_BF16, 0, 1, 2560, 2304), (W.PEAK_F16_F32, 1, 0, 3000, 3336)]:
+        c = mk(dtype, ta, tb, M, N, 1024, dist="smallint", alpha=0.125, beta=-1.0, pad_c=8)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        rows, cols = R.sample_grid(c, 128, 128, budget_macs=6e8)
+        ref, _ = dc.oracle_sub(rows, cols)
+        want = oracle.round_to(R.OT[c.out_type], ref)
+        got = dc.result()[np.ix_(rows, cols)]
+        got = got.view(np.uint32) if c.out_type == "f32" else got
+        assert np.array_equal(got, want), f"{c.name} tail={tail}"
+        outs.append(dc.result().copy())
+    key = ("tail_outs", variant)
+    prev = _TAIL_CACHE.get(key)
+    if prev is not None:
+        assert all(np.array_equal(a, b) for a, b in zip(prev, outs)), "tail split on / off disagree"
+    _TAIL_CACHE[key] = outs
+
+
+_TAIL_CACHE = {}
 
 
 def test_auto_dispatch_skinny_shapes(reset_tuning):
