@@ -217,6 +217,7 @@ def main():
     ap.add_argument("--workload", default="bf16_4096_nn")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    ap.add_argument("--tune", default="", help="comma-separated key=value pairs passed to peak_set_tuning")
     ap.add_argument("--list", action="store_true")
     args = ap.parse_args()
 
@@ -247,6 +248,9 @@ def main():
                 "sgemm": P.PEAK_VARIANT_SGEMM, "fallback": P.PEAK_VARIANT_FALLBACK}
     variant = variants[args.variant]
     P.load()
+    for kv in filter(None, args.tune.split(",")):
+        k, v = kv.split("=")
+        P.peak_set_tuning(int(k), int(v))
 
     def barrier():
         if distributed:

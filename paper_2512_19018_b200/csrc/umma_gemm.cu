@@ -303,6 +303,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (CG == 2) ptx::cluster_sync();  // the peer's barriers must be initialised before anything signals them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: everything above touched only this CTA's shared and tensor memory, so
+    // it may overlap the tail of the previous kernel in the stream; global memory is touched only after
+    // that kernel has completed.  The next kernel in the stream may start its own prologue as soon as
+    // SMs free up.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -711,11 +717,13 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = g.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, tmW, ws, p);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }

@@ -217,7 +217,7 @@ def test_launch_counter_moves():
 def reset_tuning():
     yield
     for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE,
-                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT):
+                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT, P.PEAK_TUNE_DEPENDENT_LAUNCH):
         P.peak_set_tuning(key, 0)
 
 
