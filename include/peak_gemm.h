@@ -203,7 +203,8 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_SGEMM_FMA = 4,    /* SGEMM inner product: 1 = scalar fp32 FMA, 2 = two-wide fp32 FMA (default) */
     PEAK_TUNE_TAIL_SPLIT = 5,   /* 2 = split the tiles of the last, partly filled wave whenever possible (off by default) */
     PEAK_TUNE_DEPENDENT_LAUNCH = 6, /* 1 = launch the tensor-core kernel without programmatic dependent launch */
-    PEAK_TUNE_COUNT_ = 7
+    PEAK_TUNE_SGEMM_COPY = 7,   /* SGEMM tile loads: 1 = staged through registers, 2 = asynchronous copies */
+    PEAK_TUNE_COUNT_ = 8
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

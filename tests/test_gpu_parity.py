@@ -181,6 +181,25 @@ def test_sgemm_parity(ta, tb):
     assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref))
 
 
+@pytest.mark.parametrize("copy", [1, 2])
+@pytest.mark.parametrize("fma", [1, 2])
+def test_sgemm_kernel_variants_agree_with_oracle(copy, fma, reset_tuning):
+    """Register-staged vs asynchronous-copy tile loads, scalar vs two-wide FMA: every combination exact on
+    integer inputs and within the fp32 bounds on real inputs, for all four layouts."""
+    P.peak_set_tuning(P.PEAK_TUNE_SGEMM_COPY, copy)
+    P.peak_set_tuning(P.PEAK_TUNE_SGEMM_FMA, fma)
+    for ta, tb in LAYOUTS:
+        ci = mk(W.PEAK_F32_F32, ta, tb, 384, 256, 528, dist="smallint", alpha=2.0, beta=-1.0, pad_a=4, pad_b=4, pad_c=4)
+        dc = R.DeviceCase(ci)
+        dc.run(P.PEAK_VARIANT_SGEMM)
+        ref, _ = dc.oracle_full()
+        assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref))
+        cr = mk(W.PEAK_F32_F32, ta, tb, 256, 384, 1040, alpha=0.5, beta=2.0)
+        dr = R.DeviceCase(cr)
+        dr.run(P.PEAK_VARIANT_SGEMM)
+        R.check_full(dr)
+
+
 def test_sgemm_unsupported_shape_is_reported_not_faulted():
     c = mk(W.PEAK_F32_F32, 0, 0, 100, 128, 16)
     dc = R.DeviceCase(c)
@@ -217,7 +236,8 @@ def test_launch_counter_moves():
 def reset_tuning():
     yield
     for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE,
-                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT, P.PEAK_TUNE_DEPENDENT_LAUNCH):
+                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT, P.PEAK_TUNE_DEPENDENT_LAUNCH,
+                P.PEAK_TUNE_SGEMM_COPY):
         P.peak_set_tuning(key, 0)
 
 
