@@ -66,10 +66,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 
-// Bounded wait: polls until the phase with the given parity completes or `budget` clock cycles pass.
-constexpr long long kWaitBudgetCycles = 4000000000LL;  // about two seconds at B200 clocks
+// Bounded wait: polls until the phase with the given parity completes, the CTA's abort flag is raised, or
+// `budget` clock cycles pass (the default is about two seconds at B200 clocks).
+constexpr long long kWaitBudgetCycles = 4000000000LL;
 template <bool kCluster = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile uint32_t *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile uint32_t *abort_flag,
+                                          long long budget = kWaitBudgetCycles) {
     if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -77,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
         if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0x3f) == 0) {
             if (*abort_flag != 0) return false;
-            if (clock64() - t0 > kWaitBudgetCycles) return false;
+            if (clock64() - t0 > budget) return false;
         }
     }
 }

@@ -72,6 +72,8 @@ struct UmmaParams {
     int64_t ldc;
     int vec_ok;            // C base and pitch allow 16-byte vector access
     int tma_store;         // epilogue stores through TMA
+    long long wait_cycles; // budget of every mbarrier wait
+    int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;
 };
 
@@ -323,11 +325,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n_cta = (int)tn * BN + (int)rank * C_::B_ROWS;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
+                    if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
                         report_timeout(p, abort_flag, 1, s);
                         ok = false;
                         break;
                     }
+                    if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && kb == w.kb1 - 1)
+                        continue;  // test hook: leave this stage empty so that the waits downstream run out
                     uint32_t bar = full0 + 8 * s;
                     if (leader) ptx::mbar_arrive_expect_tx(bar, (uint32_t)(C_::STAGE_BYTES * CG));
                     if (CG == 2) bar = ptx::map_to_cta(bar, 0);
@@ -363,7 +367,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // tail: every stage this CTA filled must have been released before the CTA may exit
             for (int j = 0; j < STAGES && ok; ++j, ++it) {
                 const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
+                if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
                     report_timeout(p, abort_flag, 2, s);
                     ok = false;
                 }
@@ -381,7 +385,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const Item w = decode_item(p, item);
                 const int kb0 = w.kb0, kb1 = w.kb1;
                 const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
-                if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag)) {
+                if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag, p.wait_cycles)) {
                     report_timeout(p, abort_flag, 3, b);
                     ok = false;
                     break;
@@ -390,7 +394,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t d_tmem = tmem_base + b * BN;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag)) {
+                    if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
                         report_timeout(p, abort_flag, 4, s);
                         ok = false;
                         break;
@@ -429,7 +433,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int n0 = (int)tn * BN;
             const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
             // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
-            const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag);
+            const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag, p.wait_cycles);
             if (!__all_sync(0xffffffffu, got)) {
                 if (lane == 0) report_timeout(p, abort_flag, 5, b);
                 ok = false;
@@ -708,6 +712,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     }
     p.status = device_status_word();
     if (!p.status) return PEAK_ERR_CUDA;
+    const int wait_ms = tuning(PEAK_TUNE_WAIT_MS);
+    p.wait_cycles = wait_ms > 0 ? (long long)wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
+    p.inject_stall = tuning(PEAK_TUNE_INJECT_STALL) == 1 ? 1 : 0;
 
     int units = units_max;
     if (p.total_items < units) units = p.total_items;

@@ -235,9 +235,7 @@ def test_launch_counter_moves():
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in (P.PEAK_TUNE_RASTER_GROUP, P.PEAK_TUNE_TILE_N, P.PEAK_TUNE_SPLIT_K, P.PEAK_TUNE_EPILOGUE,
-                P.PEAK_TUNE_SGEMM_FMA, P.PEAK_TUNE_TAIL_SPLIT, P.PEAK_TUNE_DEPENDENT_LAUNCH,
-                P.PEAK_TUNE_SGEMM_COPY):
+    for key in range(10):
         P.peak_set_tuning(key, 0)
 
 
@@ -312,6 +310,28 @@ def test_auto_dispatch_skinny_shapes(reset_tuning):
         dc.reset_c()
         dc.run()
         assert np.array_equal(first, dc.result())
+
+
+@pytest.mark.parametrize("variant", UMMA)
+def test_bounded_wait_reports_timeout_and_context_survives(variant, reset_tuning):
+    """Failure detection without a GPU fault: a test hook makes one CTA leave a pipeline stage unfilled (a
+    barrier that nothing completes).  The waits downstream give up after their budget (set to 20 ms here),
+    the kernel unwinds and frees its tensor memory, peak_check() reports PEAK_ERR_TIMEOUT once, and the next
+    call on the same context computes correct results."""
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 512, 512, 256)
+    dc = R.DeviceCase(c)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 20)
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 1)
+    P.peak_gemm_variant(variant, c.dtype, c.transA, c.transB, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb, 0.0, dc.C,
+                        c.ldc)
+    rc, detail = P.peak_check()
+    assert rc == P.PEAK_ERR_TIMEOUT and (detail & 0x80000000)
+    assert P.peak_check()[0] == P.PEAK_OK                      # the status word was cleared
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 0)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 0)
+    dc.reset_c()
+    dc.run(variant)                                            # same context, same buffers: correct again
+    R.check_full(dc)
 
 
 def test_set_tuning_rejects_bad_arguments():
