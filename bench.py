@@ -38,7 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SM_COUNT, SM_MAX_MHZ = 148, 1965.0
 # DRAM bytes per launch (read + write) of the dominant kernel from the ncu capture summarised under
 # profiles/; None where no capture exists for the workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "bf16_4096_nn": 103.7e6,    # profiles/umma_gemm_2cta_bf16_4096_nn.md (88.3 MB read + 15.4 MB written)
+    "bf16_8192_nn": 1.242e9,    # profiles/umma_gemm_2cta_bf16_8192_nn.md (1.115 GB read + 0.127 GB written)
+    "fp32_8192_nn": 3.553e9,    # profiles/sgemm_async_fp32_8192_nn.md (3.281 GB read + 0.272 GB written)
+}
 
 
 def workloads_table():
@@ -198,6 +202,27 @@ def run_reference(args, case):
     return 0
 
 
+def rank_case(case, rank: int):
+    """The problem rank `rank` runs: same shape and recipe, its own seed (independent problems, no collective
+    on the data path)."""
+    return case.with_(case=case.case + 17 * rank)
+
+
+def reduce_max(x: float, dist=None, device="cpu") -> float:
+    """Max over ranks of a per-rank time (the slowest rank defines the step time)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return x
+    import torch
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(case, world: int, steps: int, max_ms: float) -> float:
+    """Whole-job TFLOP/s: every rank did `steps` GEMMs of `case.flops`; time is the slowest rank's."""
+    return world * case.flops * steps / (max_ms * 1e-3) / 1e12
+
+
 def workload_config(case, l2_note):
     cfg = {"workload": case.name, "M": case.M, "N": case.N, "K": case.K, "layout": case.layout,
            "in": case.in_type, "out": case.out_type, "alpha": case.alpha, "beta": case.beta,
@@ -258,11 +283,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if not distributed:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max(x, dist if distributed else None, "cuda")
 
     def time_device(case, steps, warmup, sets, clocks_index=None):
         """W warm-up steps, then exactly `steps` back-to-back calls timed with CUDA events on the launching
@@ -322,17 +343,20 @@ def main():
             return torch.from_numpy(arr.view(np.int16)).cuda().view(torch.float16 if t == "f16" else torch.bfloat16)
 
     def measure(case, steps, warmup, with_clocks):
-        seeded = case.with_(case=case.case + 17 * rank)           # every rank its own problem
+        seeded = rank_case(case, rank)                            # every rank its own problem
         dc = Resident(seeded)
         sets, note = make_sets(seeded, dc)
         ms, launches, clocks = time_device(seeded, steps, warmup, sets, local_rank if with_clocks else None)
         return dc, sets, ms, launches, clocks, note
 
-    steps = args.steps if args.steps is not None else max(20, min(1000, int(2e14 / case.flops)))
+    # default K: about one second of timed work, long enough for the NVML clock samples to mean something
+    # (the driver updates them every ~100 ms) and for the power cap to settle -- a sustained figure
+    expected_tflops = 55.0 if case.in_type == "f32" else 1200.0
+    steps = args.steps if args.steps is not None else max(20, min(20000, int(1.0 * expected_tflops * 1e12 / case.flops)))
     warmup = args.warmup if args.warmup is not None else 10
     warmup = max(warmup, 3)
     dc, sets, ms, launches, clocks, l2_note = measure(case, steps, warmup, True)
-    value = world * case.flops * steps / (ms * 1e-3) / 1e12
+    value = aggregate_value(case, world, steps, ms)
     peaks, peak_kind = measured_peaks()
 
     # ---- roofline of the dominant kernel (the only kernel of a step) ----------------------------------
@@ -342,9 +366,16 @@ def main():
         roof = {"bound": "alu", "achieved": case.flops / (kernel_ms * 1e-3) / 1e12, "peak": alu_peak,
                 "unit": "TFLOP/s", "peak_kind": "derived: 148 SMs x 128 FMA lanes x 2 x 1.965 GHz"}
     else:
+        # a timed region of a second or more runs under the power cap: the sustained cuBLAS figure is the
+        # denominator there, the burst figure for short runs
+        long_run = ms >= 500.0
+        burst, sustained = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
         roof = {"bound": "tensor", "achieved": case.flops / (kernel_ms * 1e-3) / 1e12,
-                "peak": float(peaks["bf16_tflops"]), "unit": "TFLOP/s",
-                "peak_kind": f"{peak_kind} cuBLAS bf16 burst; sustained {peaks.get('bf16_tflops_sustained')}"}
+                "peak": sustained if long_run else burst, "unit": "TFLOP/s",
+                "peak_kind": f"{peak_kind} cuBLAS bf16 8192^3, " + ("sustained (timed region >= 0.5 s)" if long_run
+                                                                     else "burst (timed region < 0.5 s)"),
+                "frac_of_burst_peak": case.flops / (kernel_ms * 1e-3) / 1e12 / burst,
+                "frac_of_sustained_peak": case.flops / (kernel_ms * 1e-3) / 1e12 / sustained}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(case.name)
     roof["algorithmic_flops_per_launch"] = case.flops
@@ -392,12 +423,36 @@ def main():
             if name == case.name:
                 continue
             c2 = table[name]
-            s2 = max(10, min(200, int(5e13 / c2.flops)))
+            s2 = max(10, min(400, int(0.3 * (55.0 if c2.in_type == "f32" else 1200.0) * 1e12 / c2.flops)))
             _, _, ms2, l2, _, _ = measure(c2, s2, 5, False)
             tf = c2.flops * s2 / (ms2 * 1e-3) / 1e12
             pk = float(peaks["bf16_tflops"]) if c2.in_type != "f32" else SM_COUNT * 128 * 2 * SM_MAX_MHZ * 1e6 / 1e12
-            extra[name] = {"tflops": tf, "ms_per_step": ms2 / s2, "steps": s2, "frac_of_peak": tf / pk, "peak": pk}
+            extra[name] = {"tflops": tf, "ms_per_step": ms2 / s2, "steps": s2, "frac_of_peak": tf / pk, "peak": pk,
+                           "peak_kind": "burst" if c2.in_type != "f32" else "derived fp32 FMA peak"}
             torch.cuda.empty_cache()
+        # cuBLAS (torch.matmul) on the headline workload with the same protocol: a context point only
+        try:
+            torch.backends.cuda.matmul.allow_tf32 = False
+            dcc = Resident(case)
+            csets, _ = make_sets(case, dcc)
+            opA = [(a.t() if case.transA else a)[:case.M, :case.K] for a, _, _ in csets]
+            opB = [(b.t() if case.transB else b)[:case.K, :case.N] for _, b, _ in csets]
+            def mm(i):
+                torch.matmul(opA[i % len(csets)], opB[i % len(csets)])
+            for i in range(10):
+                mm(i)
+            torch.cuda.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            for i in range(steps):
+                mm(i)
+            c1.record()
+            torch.cuda.synchronize()
+            extra["cublas_context"] = {"workload": case.name, "tflops": case.flops * steps / (c0.elapsed_time(c1) * 1e-3) / 1e12,
+                                       "steps": steps, "note": "torch.matmul, same rotation and step count; not this library"}
+            del dcc, csets, opA, opB
+        except Exception as exc:  # context only: never fail the bench for it
+            extra["cublas_context"] = {"error": str(exc)[:200]}
         run, desc, threads = oracle_sampler(dc.case, dc.A_h, dc.B_h, dc.C0_h if dc.case.beta != 0 else None, 15.0)
         tf, dt = run()
         cpu = {"value": tf, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": desc, "seconds": dt}
