@@ -208,9 +208,18 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_INJECT_STALL = 9, /* test hook, 1 = one CTA leaves one pipeline stage unfilled so that the bounded
                                    waits run out: the call's result is then wrong by design and peak_check()
                                    reports PEAK_ERR_TIMEOUT; nothing hangs and the context stays usable */
-    PEAK_TUNE_COUNT_ = 10
+    PEAK_TUNE_MULTICAST = 10,   /* cluster-multicast plug-in: 1 = never use it, 2 = use it whenever it can run */
+    PEAK_TUNE_COUNT_ = 11
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
+
+/*
+ * peak_multicast_available: 1 when the optional single-GPU plug-in (libpeak_gemm_mc.so, beside the main
+ * library) is present and loaded.  It runs large 16-bit GEMMs with clusters of four CTAs that share B tiles
+ * through TMA multicast (the paper's thread-block tiling taken one level up: a cluster-level tile); results
+ * and the call contract are the same with and without it.
+ */
+int peak_multicast_available(void);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t peak_kernel_launches(void);

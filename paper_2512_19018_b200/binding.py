@@ -22,7 +22,7 @@ _lib = None
 
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
-           "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes"]
+           "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available"]
 
 
 class PeakError(RuntimeError):
@@ -56,6 +56,8 @@ def load():
     lib.peak_gemm_static_ws.argtypes = gemm_args[:-1] + [i, vp]
     lib.peak_static_ws_bytes.restype = ctypes.c_size_t
     lib.peak_static_ws_bytes.argtypes = []
+    lib.peak_multicast_available.restype = i
+    lib.peak_multicast_available.argtypes = []
     lib.peak_release_staging.restype = i
     lib.peak_release_staging.argtypes = []
     lib.peak_gemm_xcheck_f64.restype = i
@@ -139,6 +141,10 @@ def peak_static_ws_bytes() -> int:
     return load().peak_static_ws_bytes()
 
 
+def peak_multicast_available() -> bool:
+    return bool(load().peak_multicast_available())
+
+
 def peak_release_staging():
     return load().peak_release_staging()
 
@@ -165,7 +171,7 @@ def peak_tile_coord(tile, tiles_m, tiles_n, group):
 
 PEAK_TUNE_RASTER_GROUP, PEAK_TUNE_TILE_N, PEAK_TUNE_SPLIT_K, PEAK_TUNE_EPILOGUE, PEAK_TUNE_SGEMM_FMA, \
     PEAK_TUNE_TAIL_SPLIT, PEAK_TUNE_DEPENDENT_LAUNCH, PEAK_TUNE_SGEMM_COPY, PEAK_TUNE_WAIT_MS, \
-    PEAK_TUNE_INJECT_STALL = 0, 1, 2, 3, 4, 5, 6, 7, 8, 9
+    PEAK_TUNE_INJECT_STALL, PEAK_TUNE_MULTICAST = 0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10
 
 
 def peak_set_tuning(key: int, value: int) -> int:

@@ -12,8 +12,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libpeak_gemm.so")
+# optional single-GPU plug-in (cluster-multicast loads): built only where its source is present
+MC_SOURCE = os.path.join(CSRC, "umma_gemm_mc.cu")
+MC_LIB = os.path.join(HERE, "libpeak_gemm_mc.so")
 SOURCES = ["api.cu", "fallback_gemm.cu", "sgemm.cu", "umma_gemm.cu"]
-HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "ptx.cuh")] + [
+HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "ptx.cuh", "umma_device.cuh", "umma_host.cuh", "mc_plugin.h")] + [
     os.path.join(os.path.dirname(HERE), "include", "peak_gemm.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
@@ -53,9 +56,18 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
     if force or procs or _stale(LIB, objs):
         tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs
+        cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-ldl"]
         subprocess.run(cmd, check=True)
         os.replace(tmp, LIB)
+    if os.path.exists(MC_SOURCE) and (force or _stale(MC_LIB, [MC_SOURCE] + HEADERS)):
+        tmp = MC_LIB + f".tmp{os.getpid()}"
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-shared", MC_SOURCE, "-o", tmp]
+        r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+        if verbose or r.returncode:
+            sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + "\n")
+        if r.returncode:
+            raise RuntimeError("nvcc failed: " + " ".join(cmd))
+        os.replace(tmp, MC_LIB)
     return LIB
 
 

@@ -258,6 +258,8 @@ int peak_set_tuning(int key, int value) {
     return PEAK_OK;
 }
 
+int peak_multicast_available(void) { return umma_multicast_available() ? 1 : 0; }
+
 int64_t peak_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int peak_last_cuda_error(void) { return t_last_cuda_error; }

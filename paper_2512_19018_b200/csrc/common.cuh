@@ -62,6 +62,7 @@ int launch_sgemm(const GemmArgs &g);
 bool sgemm_supports(const GemmArgs &g);
 int launch_umma(const GemmArgs &g, int cta_group);
 bool umma_supports(const GemmArgs &g, int cta_group);
+bool umma_multicast_available();
 
 // status word layout: bit 31 = a bounded wait gave up; bits 0..7 = role, 8..15 = barrier index
 constexpr uint32_t kStatusTimeout = 0x80000000u;

@@ -1,0 +1,31 @@
+// Interface between the main library and its optional single-GPU accelerator plug-in
+// (libpeak_gemm_mc.so): the tensor-core GEMM run by clusters of four CTAs that share B tiles.
+// Plain C structs and one entry point, so that the two shared objects need nothing else from each other.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+extern "C" {
+
+struct peak_mc_request {
+    int dtype, transA, transB;
+    int64_t M, N, K;
+    float alpha, beta;
+    const void *A, *B;
+    void *C;
+    int64_t lda, ldb, ldc;
+    cudaStream_t stream;
+    uint32_t *status;       // the main library's per-device status word
+    int raster_group;       // 0 = default
+    int epilogue;           // PEAK_TUNE_EPILOGUE value
+    int wait_ms;            // PEAK_TUNE_WAIT_MS value
+    int dependent_launch;   // PEAK_TUNE_DEPENDENT_LAUNCH value
+    int inject_stall;       // PEAK_TUNE_INJECT_STALL value
+    int cuda_error;         // out: cudaError_t of a failing CUDA call
+};
+
+// Returns a peak_status_t.  PEAK_ERR_UNSUPPORTED: the caller should run its own kernel instead.
+typedef int (*peak_mc_gemm_fn)(peak_mc_request *req);
+int peak_mc_gemm(peak_mc_request *req);
+
+}  // extern "C"

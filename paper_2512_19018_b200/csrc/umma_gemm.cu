@@ -1,600 +1,40 @@
-// Tensor-core GEMM for 16-bit inputs on sm_100a.
-//
-// One persistent CTA (or CTA pair) per SM walks work items -- output tiles, or (tile, k-slice) pairs when
-// K is split -- in a grouped order (the paper's block swizzle).  Inside a CTA three roles run concurrently
-// (warp specialisation):
-//   warp 0      producer: TMA tile loads of A and B into a ring of 128-byte-swizzled shared-memory stages
-//               (the paper's thread-block tiling + pipelining + bank-conflict offset, section 2.2),
-//   warp 1      one thread issues tcgen05.mma; fp32 accumulators live in tensor memory (the paper's
-//               warp tiling / tensor-core steps), two accumulator buffers so that the next tile's main
-//               loop overlaps this tile's epilogue,
-//   warps 2..5  epilogue: tcgen05.ld -> alpha/beta in fp32 -> one rounding -> swizzled shared-memory
-//               staging -> TMA store (coalesced, clipped at the matrix edge); a direct vector / scalar
-//               store path serves outputs whose base or pitch is not 16-byte aligned.
-// mbarriers connect the roles (full/empty per stage, full/empty per accumulator).  Every wait is bounded.
-//
-// Tile: 128 x BN x 64 per CTA (CTA_GROUP 1) or 256 x BN x 64 per CTA pair (CTA_GROUP 2: each CTA stages its
-// 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 256 or 128.
-//
-// Split-K (the paper's Split-K transformation, section 4.1).  The first `full_tiles` tiles are computed
-// whole; each remaining tile has its k-blocks divided among `tail_splits` work items that store fp32 partial
-// tiles to a workspace, and a second kernel adds a tile's slices in slice order and applies alpha/beta, so
-// the result does not depend on scheduling.  Two uses: shapes with too few tiles to fill the GPU split every
-// tile (full_tiles = 0); shapes whose tile count is not a multiple of the SM (pair) count split only the
-// tiles of the last, partly filled wave, so that the wave finishes in a fraction of a tile time.
+// Tensor-core GEMM for 16-bit inputs on sm_100a: host side (plan, launch, workspace, entry points).
+// The kernels are in umma_device.cuh.
 #include <cuda.h>
 
 #include <mutex>
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "umma_device.cuh"
+#include "umma_host.cuh"
+#include "mc_plugin.h"
+
+#include <dlfcn.h>
+
+#include <string>
 
 namespace peak {
 namespace {
 
-constexpr int BM = 128;   // rows of C per CTA
-constexpr int BK = 64;    // k-block: 64 16-bit elements = one 128-byte swizzle row
-constexpr int UMMA_K = 16;
-constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KiB
-constexpr int ATOM_BYTES = 64 * BK * 2;     // one 64-wide MN-major box: 64 k-rows of 128 bytes = 8 KiB
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_BUF_BYTES = 32 * 128;               // one staging buffer: 32 rows x 128 bytes
-constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;      // 4 epilogue warps x 2 buffers = 32 KiB
-constexpr int SMEM_LIMIT = 232448;                    // 227 KiB of dynamic shared memory per CTA
+using namespace umma;
 
-template <int CG, int BN> struct Cfg {
-    static constexpr int B_ROWS = BN / CG;                 // rows of op(B)^T this CTA stages
-    static constexpr int B_BOX_ROWS = B_ROWS < 128 ? B_ROWS : 128;
-    static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;
-    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int AUX_BYTES = 256;
-    static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - EPI_BYTES - AUX_BYTES) / STAGE_BYTES;
-    static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + AUX_BYTES;
-    static constexpr int TMEM_COLS = 2 * BN;               // two fp32 accumulators
-    static_assert(STAGES >= 3, "pipeline too shallow");
-    static_assert(8 * (2 * STAGES + 4) + 8 <= AUX_BYTES, "barrier area too small");
-};
-
-struct UmmaParams {
-    int M, N, K;
-    int num_kb;            // ceil(K / BK)
-    int tiles_m, tiles_n;  // in units of (128*CG) x BN
-    int group;             // tile-rows per raster group
-    int full_tiles;        // tiles [0, full_tiles) are computed whole and stored to C
-    int tail_splits;       // k-slices of every later tile (partials go to the workspace)
-    int kb_per_split;
-    int total_items;       // full_tiles + (tiles - full_tiles) * tail_splits
-    int a_mn, b_mn;        // 1: operand is MN-major in memory (transA == 1 / transB == 0)
-    uint32_t idesc;
-    float alpha, beta;
-    void *C;
-    int64_t ldc;
-    int vec_ok;            // C base and pitch allow 16-byte vector access
-    int tma_store;         // epilogue stores through TMA
-    long long wait_cycles; // budget of every mbarrier wait
-    int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
-    uint32_t *status;
-};
-
-// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4),
-// descriptor version 1 (sm_100), 128-byte swizzle.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-__device__ __forceinline__ void report_timeout(const UmmaParams &p, volatile uint32_t *abort_flag, uint32_t role,
-                                               uint32_t which) {
-    if (*abort_flag == 0) atomicOr(p.status, kStatusTimeout | (which << 8) | role);
-    *abort_flag = 1;
-}
-
-template <typename TOut> __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-    TOut a = from_f32<TOut>(lo), b = from_f32<TOut>(hi);
-    return (uint32_t)(*reinterpret_cast<uint16_t *>(&a)) | ((uint32_t)(*reinterpret_cast<uint16_t *>(&b)) << 16);
-}
-
-// 32 consecutive outputs of one row -> global memory (vector path when aligned and whole)
-template <typename TOut>
-__device__ __forceinline__ void store_row32(TOut *dst, const float (&v)[32], int valid, bool vec) {
-    if (vec && valid == 32) {
-        if constexpr (sizeof(TOut) == 4) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                reinterpret_cast<float4 *>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                reinterpret_cast<uint4 *>(dst)[i] =
-                    make_uint4(pack2<TOut>(v[8 * i], v[8 * i + 1]), pack2<TOut>(v[8 * i + 2], v[8 * i + 3]),
-                               pack2<TOut>(v[8 * i + 4], v[8 * i + 5]), pack2<TOut>(v[8 * i + 6], v[8 * i + 7]));
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-            if (i < valid) dst[i] = from_f32<TOut>(v[i]);
-    }
-}
-
-// 32 consecutive old values of one row <- global memory
-template <typename TOut>
-__device__ __forceinline__ void load_row32(const TOut *src, float (&c)[32], int valid, bool vec) {
-    if (vec && valid == 32) {
-        if constexpr (sizeof(TOut) == 4) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float4 t = reinterpret_cast<const float4 *>(src)[i];
-                c[4 * i] = t.x; c[4 * i + 1] = t.y; c[4 * i + 2] = t.z; c[4 * i + 3] = t.w;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint4 t = reinterpret_cast<const uint4 *>(src)[i];
-                uint32_t w[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint16_t lo = (uint16_t)(w[j] & 0xffffu), hi = (uint16_t)(w[j] >> 16);
-                    c[8 * i + 2 * j] = to_f32(*reinterpret_cast<TOut *>(&lo));
-                    c[8 * i + 2 * j + 1] = to_f32(*reinterpret_cast<TOut *>(&hi));
-                }
-            }
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) c[i] = (i < valid) ? to_f32(src[i]) : 0.0f;
-    }
-}
-
-// 32 consecutive outputs of row `lane` -> staging buffer laid out as the 128-byte-swizzled box a TMA
-// store expects: 16-byte piece j of row r sits at piece (j ^ (r & 7)).  `h` selects which 32-column
-// half of a 64-column (16-bit) chunk is written; fp32 chunks are 32 columns wide and use h = 0.
-template <typename TOut>
-__device__ __forceinline__ void stage_row32(uint32_t buf, int lane, int h, const float (&v)[32]) {
-    constexpr int PIECES = 32 * (int)sizeof(TOut) / 16;  // 8 (fp32) or 4 (16-bit)
-    const uint32_t row = buf + (uint32_t)lane * 128u;
-#pragma unroll
-    for (int j = 0; j < PIECES; ++j) {
-        uint32_t w0, w1, w2, w3;
-        if constexpr (sizeof(TOut) == 4) {
-            w0 = __float_as_uint(v[4 * j]); w1 = __float_as_uint(v[4 * j + 1]);
-            w2 = __float_as_uint(v[4 * j + 2]); w3 = __float_as_uint(v[4 * j + 3]);
-        } else {
-            w0 = pack2<TOut>(v[8 * j], v[8 * j + 1]); w1 = pack2<TOut>(v[8 * j + 2], v[8 * j + 3]);
-            w2 = pack2<TOut>(v[8 * j + 4], v[8 * j + 5]); w3 = pack2<TOut>(v[8 * j + 6], v[8 * j + 7]);
-        }
-        const uint32_t piece = (uint32_t)((h * PIECES + j) ^ (lane & 7));
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + piece * 16u), "r"(w0), "r"(w1), "r"(w2),
-                     "r"(w3)
-                     : "memory");
-    }
-}
-
-// Work item -> tile, k-block range and destination (ws_block < 0: the tile is whole and goes to C;
-// otherwise the index of the (tile, slice) block of the partial-tile workspace).
-struct Item {
-    int tile, kb0, kb1, ws_block;
-};
-__device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
-    Item w;
-    if (item < p.full_tiles) {
-        w.tile = item; w.kb0 = 0; w.kb1 = p.num_kb; w.ws_block = -1;
-    } else {
-        const int j = item - p.full_tiles;
-        const int t = j / p.tail_splits, slice = j - t * p.tail_splits;
-        w.tile = p.full_tiles + t;
-        w.kb0 = slice * p.kb_per_split;
-        w.kb1 = min(w.kb0 + p.kb_per_split, p.num_kb);
-        w.ws_block = j;
-    }
-    return w;
-}
-
-// Epilogue of one accumulator tile for one warp: TMEM -> registers -> alpha/beta -> T -> staging + TMA
-// store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
-// column limit, `nrows` the row limit for `row`; (x0, y0) is where chunk 0 of this warp lands in `tm`.
-template <typename T, int BN>
-__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
-                                              T *base, int64_t ld, int row, int row0, int nrows, int cbase,
-                                              int ncols, const CUtensorMap *tm, int x0, int y0, bool tma, bool vec,
-                                              float alpha, float beta) {
-    constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
-#pragma unroll 1
-    for (int c = 0; c < BN / CHUNK_COLS; ++c) {
-        const int col0 = cbase + c * CHUNK_COLS;
-        if (col0 >= ncols) break;  // warp-uniform
-        uint32_t buf = 0;
-        if (tma) {
-            // the store that last read this buffer (two chunks ago) must have drained it
-            buf = my_stage + (chunk_no & 1u) * EPI_BUF_BYTES;
-            if (lane == 0) ptx::tma_store_wait_read<1>();
-            __syncwarp();
-        }
-#pragma unroll
-        for (int h = 0; h < CHUNK_COLS / 32; ++h) {
-            const int col = col0 + h * 32;
-            uint32_t r[32];
-            ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r);
-            ptx::tmem_ld_wait();
-            const int valid = (ncols - col >= 32) ? 32 : (ncols - col > 0 ? ncols - col : 0);
-            T *dst = base + (int64_t)row * ld + col;
-            float v[32];
-            if (beta != 0.0f) {
-                float cold[32];
-                if (row < nrows && valid > 0) load_row32<T>(dst, cold, valid, vec);
-                else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = fmaf(beta, cold[i], alpha * __uint_as_float(r[i]));
-            } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[i]);
-            }
-            if (tma) stage_row32<T>(buf, lane, h, v);
-            else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
-        }
-        if (tma) {
-            ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
-            __syncwarp();
-            if (lane == 0 && row0 < nrows) {
-                ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
-                ptx::tma_store_commit();
-            }
-            ++chunk_no;
-        }
-    }
-}
-
-template <int CG, int BN, typename TOut>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
-                 float *__restrict__ ws, const UmmaParams p) {
-    using C_ = Cfg<CG, BN>;
-    constexpr int STAGES = C_::STAGES;
-    extern __shared__ uint8_t smem_raw[];
-
-    const uint32_t raw = ptx::smem_u32(smem_raw);
-    const uint32_t stage_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-    const uint32_t epi_base = stage_base + STAGES * C_::STAGE_BYTES;
-    uint8_t *aux = smem_raw + (epi_base - raw) + EPI_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * (2 * STAGES + 4));
-    volatile uint32_t *abort_flag = tmem_slot + 1;
-
-    const uint32_t full0 = ptx::smem_u32(bars);
-    const uint32_t empty0 = full0 + 8 * STAGES;
-    const uint32_t accfull0 = empty0 + 8 * STAGES;
-    const uint32_t accempty0 = accfull0 + 16;
-
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
-    const bool leader = (rank == 0);
-    const int unit = blockIdx.x / CG;          // CTA (or CTA pair) index
-    const int num_units = gridDim.x / CG;
-    const int total_items = p.total_items;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(full0 + 8 * s, 1);
-            ptx::mbar_init(empty0 + 8 * s, 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(accfull0 + 8 * b, 1);
-            ptx::mbar_init(accempty0 + 8 * b, 4 * CG);  // one arrival per epilogue warp of every CTA
-        }
-        *abort_flag = 0;
-        ptx::fence_mbar_init();
-        ptx::fence_proxy_async_smem();
-    }
-    if (warp == 0 && lane == 0) {
-        ptx::prefetch_tensormap(&tmA);
-        ptx::prefetch_tensormap(&tmB);
-        if (p.tma_store) ptx::prefetch_tensormap(&tmC);
-        if (p.total_items > p.full_tiles) ptx::prefetch_tensormap(&tmW);
-    }
-    if (warp == 1) {
-        ptx::tmem_alloc<CG>(ptx::smem_u32(tmem_slot), C_::TMEM_COLS);
-        ptx::tmem_relinquish<CG>();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (CG == 2) ptx::cluster_sync();  // the peer's barriers must be initialised before anything signals them
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-    // Programmatic dependent launch: everything above touched only this CTA's shared and tensor memory, so
-    // it may overlap the tail of the previous kernel in the stream; global memory is touched only after
-    // that kernel has completed.  The next kernel in the stream may start its own prologue as soon as
-    // SMs free up.
-    ptx::grid_dependency_wait();
-    ptx::grid_launch_dependents();
-
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int item = unit; item < total_items && ok; item += num_units) {
-                const Item w = decode_item(p, item);
-                int64_t tm, tn;
-                tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-                const int m_cta = (int)tm * (BM * CG) + (int)rank * BM;
-                const int n_cta = (int)tn * BN + (int)rank * C_::B_ROWS;
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
-                        report_timeout(p, abort_flag, 1, s);
-                        ok = false;
-                        break;
-                    }
-                    if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && kb == w.kb1 - 1)
-                        continue;  // test hook: leave this stage empty so that the waits downstream run out
-                    uint32_t bar = full0 + 8 * s;
-                    if (leader) ptx::mbar_arrive_expect_tx(bar, (uint32_t)(C_::STAGE_BYTES * CG));
-                    if (CG == 2) bar = ptx::map_to_cta(bar, 0);
-                    const uint32_t a_dst = stage_base + s * C_::STAGE_BYTES;
-                    const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                    const int k0 = kb * BK;
-                    if (!p.a_mn) {
-                        if (CG == 1) ptx::tma_load_2d(a_dst, &tmA, k0, m_cta, bar);
-                        else ptx::tma_load_2d_pair(a_dst, &tmA, k0, m_cta, bar);
-                    } else {
-#pragma unroll
-                        for (int h = 0; h < BM / 64; ++h) {
-                            if (CG == 1) ptx::tma_load_2d(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bar);
-                            else ptx::tma_load_2d_pair(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bar);
-                        }
-                    }
-                    if (!p.b_mn) {
-#pragma unroll
-                        for (int h = 0; h < C_::B_ROWS / C_::B_BOX_ROWS; ++h) {
-                            const uint32_t d = b_dst + h * C_::B_BOX_ROWS * 128;
-                            if (CG == 1) ptx::tma_load_2d(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
-                            else ptx::tma_load_2d_pair(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
-                        }
-                    } else {
-#pragma unroll
-                        for (int h = 0; h < C_::B_ROWS / 64; ++h) {
-                            if (CG == 1) ptx::tma_load_2d(b_dst + h * ATOM_BYTES, &tmB, n_cta + 64 * h, k0, bar);
-                            else ptx::tma_load_2d_pair(b_dst + h * ATOM_BYTES, &tmB, n_cta + 64 * h, k0, bar);
-                        }
-                    }
-                }
-            }
-            // tail: every stage this CTA filled must have been released before the CTA may exit
-            for (int j = 0; j < STAGES && ok; ++j, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
-                    report_timeout(p, abort_flag, 2, s);
-                    ok = false;
-                }
-            }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && leader) {
-            uint32_t it = 0, tl = 0;
-            bool ok = true;
-            const uint32_t a_lbo = p.a_mn ? (uint32_t)ATOM_BYTES : 16u, b_lbo = p.b_mn ? (uint32_t)ATOM_BYTES : 16u;
-            const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
-            for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
-                const Item w = decode_item(p, item);
-                const int kb0 = w.kb0, kb1 = w.kb1;
-                const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
-                if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag, p.wait_cycles)) {
-                    report_timeout(p, abort_flag, 3, b);
-                    ok = false;
-                    break;
-                }
-                ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + b * BN;
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
-                        report_timeout(p, abort_flag, 4, s);
-                        ok = false;
-                        break;
-                    }
-                    ptx::tc_fence_after_sync();
-                    const uint32_t a_base = stage_base + s * C_::STAGE_BYTES;
-                    const uint32_t b_base = a_base + A_STAGE_BYTES;
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
-                        const uint64_t bd = smem_desc(b_base + k * b_kstep, b_lbo, 1024u);
-                        ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
-                    }
-                    // release the stage (in both CTAs of a pair) once these MMAs have read it
-                    if (CG == 1) ptx::umma_commit_1cta(empty0 + 8 * s);
-                    else ptx::umma_commit_pair(empty0 + 8 * s, 3);
-                }
-                if (!ok) break;
-                if (CG == 1) ptx::umma_commit_1cta(accfull0 + 8 * b);
-                else ptx::umma_commit_pair(accfull0 + 8 * b, 3);
-            }
-        }
-        __syncwarp();
-    } else {
-        // ------------------------------------------------------------------ epilogue (4 warps)
-        const int q = warp & 3;  // TMEM lane quadrant this warp may read
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
-        const bool vec = p.vec_ok != 0;
-        uint32_t tl = 0, chunk_no = 0;
-        bool ok = true;
-        for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
-            const Item w = decode_item(p, item);
-            int64_t tm, tn;
-            tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-            const int row0 = (int)tm * (BM * CG) + (int)rank * BM + q * 32;  // first row of this warp
-            const int n0 = (int)tn * BN;
-            const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
-            // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
-            const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag, p.wait_cycles);
-            if (!__all_sync(0xffffffffu, got)) {
-                if (lane == 0) report_timeout(p, abort_flag, 5, b);
-                ok = false;
-                break;
-            }
-            ptx::tc_fence_after_sync();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
-            if (w.ws_block < 0) {
-                // whole tile: alpha/beta epilogue straight to C
-                epilogue_tile<TOut, BN>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C), p.ldc,
-                                        row0 + lane, row0, p.M, n0, p.N, &tmC, n0, row0, p.tma_store != 0, vec,
-                                        p.alpha, p.beta);
-            } else {
-                // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
-                const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
-                epilogue_tile<float, BN>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
-                                         0x7fffffff, 0, BN, &tmW, 0, wrow0, true, true, 1.0f, 0.0f);
-            }
-            // hand the accumulator buffer back to the MMA issuer
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-                if (CG == 1) ptx::mbar_arrive(accempty0 + 8 * b);
-                else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, 0));
-            }
-        }
-        if (lane == 0) ptx::tma_store_wait_all<0>();  // staging memory must outlive the stores
-        __syncwarp();
-    }
-
-    // ---------------------------------------------------------------------- teardown
-    if (*abort_flag != 0) {
-        // a wait gave up: give copies that may still be in flight time to land before shared memory goes away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (CG == 2) ptx::cluster_sync();  // the peer may still signal this CTA's barriers or read its tiles
-    if (warp == 1) {
-        ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc<CG>(tmem_base, C_::TMEM_COLS);
-    }
-}
-
-// Adds the k-slices of every split tile in slice order and applies the epilogue:
-// C = alpha * (ws[tile][0] + ws[tile][1] + ...) + beta * C, one rounding.  The workspace holds, for split tile
-// t (counted from full_tiles) and slice s, a dense rows_t x bn fp32 block at index t * splits + s.
-// One block of 256 threads handles a quarter of a tile's float4 columns groups at a time.
-template <typename TOut>
-__global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
-                     int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
-                     int vec_ok) {
-    const int blocks_per_tile = gridDim.y;
-    const int t = blockIdx.x;  // split tile number
-    int64_t tm, tn;
-    tile_coord(full_tiles + t, tiles_m, tiles_n, group, tm, tn);
-    const int vec_per_row = bn / 4;
-    const int total_vec = rows_t * vec_per_row;
-    const int64_t block_elems = (int64_t)rows_t * bn;
-    const float *base = ws + (int64_t)t * splits * block_elems;
-    for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < total_vec; e += blocks_per_tile * blockDim.x) {
-        const int r = e / vec_per_row, c4 = e - r * vec_per_row;
-        const int64_t i = tm * rows_t + r;
-        const int64_t j = tn * bn + c4 * 4;
-        if (i >= M || j >= N) continue;
-        const float *src = base + (int64_t)r * bn + c4 * 4;
-        float4 acc = *reinterpret_cast<const float4 *>(src);
-        for (int sl = 1; sl < splits; ++sl) {
-            const float4 v = *reinterpret_cast<const float4 *>(src + sl * block_elems);
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
-        TOut *dst = C + i * ldc + j;
-        if (vec_ok && j + 4 <= N) {
-            float o[4] = {0.f, 0.f, 0.f, 0.f};
-            if (beta != 0.0f) {
-                if constexpr (sizeof(TOut) == 4) {
-                    const float4 t4 = *reinterpret_cast<const float4 *>(dst);
-                    o[0] = t4.x; o[1] = t4.y; o[2] = t4.z; o[3] = t4.w;
-                } else {
-                    const uint2 t2 = *reinterpret_cast<const uint2 *>(dst);
-                    uint16_t h[4] = {(uint16_t)(t2.x & 0xffffu), (uint16_t)(t2.x >> 16), (uint16_t)(t2.y & 0xffffu),
-                                     (uint16_t)(t2.y >> 16)};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) o[k] = to_f32(*reinterpret_cast<TOut *>(&h[k]));
-                }
-            }
-            float rr[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) rr[k] = epilogue_f32(alpha, a4[k], beta, o[k]);
-            if constexpr (sizeof(TOut) == 4) {
-                *reinterpret_cast<float4 *>(dst) = make_float4(rr[0], rr[1], rr[2], rr[3]);
-            } else {
-                *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<TOut>(rr[0], rr[1]), pack2<TOut>(rr[2], rr[3]));
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                if (j + k < N) {
-                    const float c_old = (beta != 0.0f) ? to_f32(dst[k]) : 0.0f;
-                    dst[k] = from_f32<TOut>(epilogue_f32(alpha, a4[k], beta, c_old));
-                }
-            }
-        }
-    }
-}
-
-// ---- host side -------------------------------------------------------------------------------------------
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
+// ---- optional single-GPU plug-in (cluster-multicast B loads), loaded from beside this library ------------
+peak_mc_gemm_fn mc_entry() {
+    static peak_mc_gemm_fn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
-        void *f = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
+        Dl_info info;
+        if (!dladdr(reinterpret_cast<void *>(&mc_entry), &info) || !info.dli_fname) return;
+        std::string path(info.dli_fname);
+        const size_t slash = path.find_last_of('/');
+        path = (slash == std::string::npos ? std::string(".") : path.substr(0, slash)) + "/libpeak_gemm_mc.so";
+        void *h = dlopen(path.c_str(), RTLD_NOW | RTLD_LOCAL);
+        if (!h) return;
+        fn = reinterpret_cast<peak_mc_gemm_fn>(dlsym(h, "peak_mc_gemm"));
     });
     return fn;
 }
-
-// Tensor map over a row-major 2-D array: `inner` contiguous elements per row, `outer` rows, `pitch`
-// elements between rows; box = box_inner x box_outer, 128-byte swizzle, zero fill.
-bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
-              int box_outer) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
-                                   : e == Elem::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
-                                                     : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)pitch * (cuuint64_t)elem_bytes(e)};
-    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
-int sm_count() {
-    static int sms[64];
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) return 148;
-    if (sms[dev] == 0) {
-        int n = 0;
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        sms[dev] = n > 0 ? n : 148;
-    }
-    return sms[dev];
-}
-
-constexpr double kL2BytesPerClk = 64.0;      // assumed L2 -> shared-memory bandwidth per SM
-constexpr double kSplitFixedCycles = 20000.0;  // workspace allocation + second launch of a split (~12 us)
 
 struct Plan {
     int bn;           // tile width: 256 or 128
@@ -849,10 +289,28 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
     return true;
 }
 
+bool umma_multicast_available() { return mc_entry() != nullptr; }
+
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
     const int units = sm_count() / cta_group;
     const Plan plan = choose_plan(g, cta_group, units);
+    // whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there
+    const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
+    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && mc_entry()) {
+        const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
+        if (mc_mode == 2 || super_tiles >= 32) {
+            peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
+                              g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
+                              tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
+                              tuning(PEAK_TUNE_INJECT_STALL), 0};
+            if (!r.status) return PEAK_ERR_CUDA;
+            const int rc = mc_entry()(&r);
+            if (rc == PEAK_OK) { count_launch(); return rc; }
+            if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
+            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+        }
+    }
     if (cta_group == 2) return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);
     return plan.bn == 256 ? run_umma<1, 256>(g, plan, units) : run_umma<1, 128>(g, plan, units);
 }

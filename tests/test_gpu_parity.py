@@ -235,7 +235,7 @@ def test_launch_counter_moves():
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(10):
+    for key in range(11):
         P.peak_set_tuning(key, 0)
 
 
@@ -332,6 +332,36 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant, reset_tuning
     dc.reset_c()
     dc.run(variant)                                            # same context, same buffers: correct again
     R.check_full(dc)
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_BF16_BF16, W.PEAK_F16_F32])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_multicast_plugin_matches_oracle(dtype, ta, tb, reset_tuning):
+    """The optional cluster-multicast plug-in (four-CTA clusters sharing B tiles), forced on: exact on integer
+    inputs for every layout, within the bounds on real inputs with alpha/beta and ragged edges, and identical
+    to the plain kernel's output bit for bit on the integer cases."""
+    if not P.peak_multicast_available():
+        pytest.skip("libpeak_gemm_mc.so is not present (multi-GPU runs leave it out)")
+    for idx, (M, N, K) in enumerate([(512, 256, 64), (1024, 512, 448), (700, 328, 264), (1536, 1280, 1024)]):
+        pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8     # TMA needs pitches that are multiples of 8
+        ci = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.125, beta=-1.0, case=idx, pad_a=pa, pad_b=pb, pad_c=8)
+        outs = []
+        for mode in (2, 1):
+            P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, mode)
+            dc = R.DeviceCase(ci)
+            dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+            outs.append(dc.result().copy())
+            if mode == 2:
+                ref, _ = dc.oracle_full()
+                want = oracle.round_to(R.OT[ci.out_type], ref)
+                got = outs[0].view(np.uint32) if ci.out_type == "f32" else outs[0]
+                assert np.array_equal(got, want), f"{ci.name}: multicast result differs from the oracle"
+        assert np.array_equal(outs[0], outs[1]), f"{ci.name}: multicast and plain kernels disagree"
+        P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, 2)
+        cr = mk(dtype, ta, tb, M, N, K, alpha=0.5, beta=2.0, case=idx, pad_a=pa, pad_b=pb)
+        dr = R.DeviceCase(cr)
+        dr.run(P.PEAK_VARIANT_UMMA_2CTA)
+        R.check_full(dr, what=f"{cr.name} multicast")
 
 
 def test_set_tuning_rejects_bad_arguments():
