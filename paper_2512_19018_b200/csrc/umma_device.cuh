@@ -14,7 +14,10 @@
 // mbarriers connect the roles (full/empty per stage, full/empty per accumulator).  Every wait is bounded.
 //
 // Tile: 128 x BN x 64 per CTA (CTA_GROUP 1) or 256 x BN x 64 per CTA pair (CTA_GROUP 2: each CTA stages its
-// 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 256 or 128.
+// 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 128, 256, or --
+// CTA pairs only -- 512: a 256 x 512 tile is computed as two 256-column halves that occupy both accumulator
+// slots, so a quarter fewer operand bytes reach each SM per flop (what limits the sustained rate under the
+// power cap) at the price of an epilogue that overlaps the next main loop only half by half.
 //
 // Split-K (the paper's Split-K transformation, section 4.1).  The first `full_tiles` tiles are computed
 // whole; each remaining tile has its k-blocks divided among `tail_splits` work items that store fp32 partial
@@ -42,15 +45,20 @@ constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;      // 4 epilogue warps x 2 bu
 constexpr int SMEM_LIMIT = 232448;                    // 227 KiB of dynamic shared memory per CTA
 
 template <int CG, int BN> struct Cfg {
-    static constexpr int B_ROWS = BN / CG;                 // rows of op(B)^T this CTA stages
-    static constexpr int B_BOX_ROWS = B_ROWS < 128 ? B_ROWS : 128;
+    // A tile wider than one MMA (BN = 512) is computed as two 256-column halves, one per accumulator slot.
+    static constexpr int SLOT_N = BN > 256 ? 256 : BN;     // MMA N = width of one accumulator slot
+    static constexpr int HALVES = BN / SLOT_N;
+    static constexpr int HROWS = SLOT_N / CG;              // rows of op(B)^T this CTA stages per half
+    static constexpr int B_ROWS = HALVES * HROWS;
+    static constexpr int B_BOX_ROWS = HROWS < 128 ? HROWS : 128;
     static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
     static constexpr int AUX_BYTES = 256;
     static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - EPI_BYTES - AUX_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + AUX_BYTES;
-    static constexpr int TMEM_COLS = 2 * BN;               // two fp32 accumulators
+    static constexpr int TMEM_COLS = 2 * SLOT_N;           // two fp32 accumulator slots
+    static_assert(HALVES == 1 || CG == 2, "512-wide tiles are for CTA pairs");
     static_assert(STAGES >= 3, "pipeline too shallow");
     static_assert(8 * (2 * STAGES + 4) + 8 <= AUX_BYTES, "barrier area too small");
 };
@@ -335,7 +343,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 int64_t tm, tn;
                 tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
-                const int n_cta = (int)tn * BN + (int)rank * C_::B_ROWS;
+                const int n_cta = (int)tn * BN + (int)rank * C_::HROWS;  // first B row of this CTA (half 0)
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
@@ -370,16 +378,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                   bar, mask);
                     } else if (!p.b_mn) {
 #pragma unroll
-                        for (int h = 0; h < C_::B_ROWS / C_::B_BOX_ROWS; ++h) {
-                            const uint32_t d = b_dst + h * C_::B_BOX_ROWS * 128;
-                            if (CG == 1) ptx::tma_load_2d(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
-                            else ptx::tma_load_2d_pair(d, &tmB, k0, n_cta + C_::B_BOX_ROWS * h, bar);
+                        for (int hf = 0; hf < C_::HALVES; ++hf) {
+#pragma unroll
+                            for (int h = 0; h < C_::HROWS / C_::B_BOX_ROWS; ++h) {
+                                const uint32_t d = b_dst + (hf * C_::HROWS + h * C_::B_BOX_ROWS) * 128;
+                                const int n = n_cta + hf * C_::SLOT_N + C_::B_BOX_ROWS * h;
+                                if (CG == 1) ptx::tma_load_2d(d, &tmB, k0, n, bar);
+                                else ptx::tma_load_2d_pair(d, &tmB, k0, n, bar);
+                            }
                         }
                     } else {
 #pragma unroll
-                        for (int h = 0; h < C_::B_ROWS / 64; ++h) {
-                            if (CG == 1) ptx::tma_load_2d(b_dst + h * ATOM_BYTES, &tmB, n_cta + 64 * h, k0, bar);
-                            else ptx::tma_load_2d_pair(b_dst + h * ATOM_BYTES, &tmB, n_cta + 64 * h, k0, bar);
+                        for (int hf = 0; hf < C_::HALVES; ++hf) {
+#pragma unroll
+                            for (int h = 0; h < C_::HROWS / 64; ++h) {
+                                const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * ATOM_BYTES;
+                                const int n = n_cta + hf * C_::SLOT_N + 64 * h;
+                                if (CG == 1) ptx::tma_load_2d(d, &tmB, n, k0, bar);
+                                else ptx::tma_load_2d_pair(d, &tmB, n, k0, bar);
+                            }
                         }
                     }
                 }
@@ -404,14 +421,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
                 const Item w = decode_item(p, item);
                 const int kb0 = w.kb0, kb1 = w.kb1;
-                const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
-                if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag, p.wait_cycles)) {
-                    report_timeout(p, abort_flag, 3, b);
-                    ok = false;
-                    break;
+                // one-slot tiles alternate between the two accumulator slots; a two-half tile uses both
+                const uint32_t b = (C_::HALVES == 1) ? (tl & 1u) : 0u;
+                const uint32_t aph = (C_::HALVES == 1) ? ((tl >> 1) & 1u) : (tl & 1u);
+                if (C_::HALVES == 1) {
+                    if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * b, aph ^ 1u, abort_flag, p.wait_cycles)) {
+                        report_timeout(p, abort_flag, 3, b);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
                 }
-                ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + b * BN;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
@@ -423,18 +443,38 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t a_base = stage_base + s * C_::STAGE_BYTES;
                     const uint32_t b_base = a_base + A_STAGE_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
-                        const uint64_t bd = smem_desc(b_base + k * b_kstep, b_lbo, 1024u);
-                        ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
+                    for (int hf = 0; hf < C_::HALVES; ++hf) {
+                        const uint32_t slot = (C_::HALVES == 1) ? b : (uint32_t)hf;
+                        if (C_::HALVES == 2 && kb == kb0) {
+                            // the epilogue hands the halves of the previous tile back one after the other
+                            if (!ptx::mbar_wait<CG == 2>(accempty0 + 8 * slot, aph ^ 1u, abort_flag, p.wait_cycles)) {
+                                report_timeout(p, abort_flag, 3, slot);
+                                ok = false;
+                                break;
+                            }
+                            ptx::tc_fence_after_sync();
+                        }
+                        const uint32_t d_tmem = tmem_base + slot * C_::SLOT_N;
+                        const uint32_t bh_base = b_base + hf * C_::HROWS * 128;
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
+                            const uint64_t bd = smem_desc(bh_base + k * b_kstep, b_lbo, 1024u);
+                            ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
+                        }
                     }
+                    if (!ok) break;
                     // release the stage (in both CTAs of a pair) once these MMAs have read it
                     if (CG == 1) ptx::umma_commit_1cta(empty0 + 8 * s);
                     else ptx::umma_commit_pair(empty0 + 8 * s, MC ? 0xF : 3);
                 }
                 if (!ok) break;
-                if (CG == 1) ptx::umma_commit_1cta(accfull0 + 8 * b);
-                else ptx::umma_commit_pair(accfull0 + 8 * b, (uint16_t)(3u << leader_crank));
+#pragma unroll
+                for (int hf = 0; hf < C_::HALVES; ++hf) {
+                    const uint32_t slot = (C_::HALVES == 1) ? b : (uint32_t)hf;
+                    if (CG == 1) ptx::umma_commit_1cta(accfull0 + 8 * slot);
+                    else ptx::umma_commit_pair(accfull0 + 8 * slot, (uint16_t)(3u << leader_crank));
+                }
             }
         }
         __syncwarp();
@@ -451,33 +491,38 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
             const int n0 = (int)tn * BN;
-            const uint32_t b = tl & 1u, aph = (tl >> 1) & 1u;
-            // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
-            const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag, p.wait_cycles);
-            if (!__all_sync(0xffffffffu, got)) {
-                if (lane == 0) report_timeout(p, abort_flag, 5, b);
-                ok = false;
-                break;
-            }
-            ptx::tc_fence_after_sync();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN;
-            if (w.ws_block < 0) {
-                // whole tile: alpha/beta epilogue straight to C
-                epilogue_tile<TOut, BN>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C), p.ldc,
-                                        row0 + lane, row0, p.M, n0, p.N, &tmC, n0, row0, p.tma_store != 0, vec,
-                                        p.alpha, p.beta);
-            } else {
-                // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
-                const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
-                epilogue_tile<float, BN>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
-                                         0x7fffffff, 0, BN, &tmW, 0, wrow0, true, true, 1.0f, 0.0f);
-            }
-            // hand the accumulator buffer back to the MMA issuer
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-                if (CG == 1) ptx::mbar_arrive(accempty0 + 8 * b);
-                else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, leader_crank));
+#pragma unroll 1
+            for (int hf = 0; hf < C_::HALVES && ok; ++hf) {
+                const uint32_t b = (C_::HALVES == 1) ? (tl & 1u) : (uint32_t)hf;
+                const uint32_t aph = (C_::HALVES == 1) ? ((tl >> 1) & 1u) : (tl & 1u);
+                // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
+                const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag, p.wait_cycles);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (lane == 0) report_timeout(p, abort_flag, 5, b);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * C_::SLOT_N;
+                const int nh = n0 + hf * C_::SLOT_N;  // first column of this half
+                if (w.ws_block < 0) {
+                    // whole tile: alpha/beta epilogue straight to C
+                    epilogue_tile<TOut, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C),
+                                                    p.ldc, row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0,
+                                                    p.tma_store != 0, vec, p.alpha, p.beta);
+                } else {
+                    // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
+                    const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
+                    epilogue_tile<float, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane,
+                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, true, true, 1.0f, 0.0f);
+                }
+                // hand the accumulator slot back to the MMA issuer
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 1) ptx::mbar_arrive(accempty0 + 8 * b);
+                    else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, leader_crank));
+                }
             }
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();  // staging memory must outlive the stores

@@ -57,8 +57,9 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     double best_cost = 1e300;
     const int force_bn = tuning(PEAK_TUNE_TILE_N), force_split = tuning(PEAK_TUNE_SPLIT_K);
     const int tail_mode = tuning(PEAK_TUNE_TAIL_SPLIT);  // 2 = split the last wave whenever possible
-    for (int bn : {256, 128}) {
-        if (force_bn && bn != force_bn) continue;
+    for (int bn : {512, 256, 128}) {
+        if (force_bn ? bn != force_bn : bn == 512) continue;  // 512-wide tiles only on request (see launch_umma)
+        if (bn == 512 && cg != 2) continue;
         const int64_t tiles = tiles_of(g, cg, bn);
         const double kb_cycles = fmax(2.0 * bn, (128.0 + bn / cg) * 128.0 / kL2BytesPerClk);
         const double item_ovh = 1500.0;
@@ -69,7 +70,7 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
         // (a) every tile whole, or every tile split s ways
         for (int s = 1; s <= 16; ++s) {
             if (force_split && s != force_split) continue;
-            if (s > num_kb) break;
+            if (s > num_kb || (bn == 512 && s > 1)) break;
             if (s > 1 && !force_split && tiles * s > 2 * units) break;
             const int64_t kbps = (num_kb + s - 1) / s;
             if (s > 1 && kbps * (s - 1) >= num_kb) continue;  // an empty last slice
@@ -83,7 +84,7 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
         const int64_t full = (tiles / units) * units, rest = tiles - full;
         // (measured on B200: under the power cap the busy SMs of a partly filled wave clock higher, so this
         // split gains nothing at 4096^3 or 5000x3000x2500; it stays opt-in through PEAK_TUNE_TAIL_SPLIT = 2)
-        if (!force_split && tail_mode == 2 && full > 0 && rest > 0) {
+        if (!force_split && tail_mode == 2 && full > 0 && rest > 0 && bn != 512) {
             for (int s = 2; s <= 8; ++s) {
                 if (rest * s > units || s > num_kb) break;
                 const int64_t kbps = (num_kb + s - 1) / s;
@@ -132,7 +133,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
+              ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.ldc = g.ldc;
     const int ob = elem_bytes(eout);
@@ -294,12 +295,20 @@ bool umma_multicast_available() { return mc_entry() != nullptr; }
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
     const int units = sm_count() / cta_group;
-    const Plan plan = choose_plan(g, cta_group, units);
-    // whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there
+    Plan plan = choose_plan(g, cta_group, units);
+    // Measured on B200 under the power cap (sustained, random inputs): 256 x 512 pair tiles are 4-12 % faster
+    // than 256 x 256 ones when the main loop is long (K >= 8192) and there are at least two waves of them, and
+    // up to 13 % slower at K = 4096 where their half-overlapped epilogue shows.
+    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && !tuning(PEAK_TUNE_TILE_N) &&
+        g.K >= 8192 && tiles_of(g, 2, 512) >= 2 * units)
+        plan = Plan{512, (int)tiles_of(g, 2, 512), 1};
+    // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
+    // Measured: +3 % at 4096^3, +12 % at 5000x3000x2500, but -2..-4 % on problems of 5e11 flop and more.
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
     if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && mc_entry()) {
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
-        if (mc_mode == 2 || super_tiles >= 32) {
+        const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
+        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 3e11)) {
             peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
@@ -311,7 +320,10 @@ int launch_umma(const GemmArgs &g, int cta_group) {
             if (rc != PEAK_ERR_UNSUPPORTED) return rc;
         }
     }
-    if (cta_group == 2) return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);
+    if (cta_group == 2) {
+        if (plan.bn == 512) return run_umma<2, 512>(g, plan, units);
+        return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);
+    }
     return plan.bn == 256 ? run_umma<1, 256>(g, plan, units) : run_umma<1, 128>(g, plan, units);
 }
 

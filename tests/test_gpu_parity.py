@@ -298,6 +298,35 @@ def test_umma_last_wave_split(variant, tail, reset_tuning):
 _TAIL_CACHE = {}
 
 
+@pytest.mark.parametrize("dtype", [W.PEAK_BF16_BF16, W.PEAK_F16_F32])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_umma_512_wide_tiles(dtype, ta, tb, reset_tuning):
+    """256 x 512 pair tiles computed as two 256-column halves over both accumulator slots: exact on integer
+    inputs (several tiles per CTA pair so that the half-by-half hand-over between epilogue and main loop is
+    exercised), bounds on real inputs with alpha/beta and ragged edges."""
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 512)
+    for idx, (M, N, K) in enumerate([(256, 512, 64), (512, 1024, 320), (300, 700, 200), (8192, 6144, 128)]):
+        pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+        ci = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.125, beta=-1.0, case=idx, pad_a=pa, pad_b=pb, pad_c=8)
+        dc = R.DeviceCase(ci)
+        dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+        if M * N * K <= 2e9:
+            ref, _ = dc.oracle_full()
+            got = dc.result()
+        else:                       # 192 tiles over 74 CTA pairs: check a sub-grid that samples every tile
+            rows, cols = R.sample_grid(ci, 256, 256, budget_macs=4e8)
+            ref, _ = dc.oracle_sub(rows, cols)
+            got = dc.result()[np.ix_(rows, cols)]
+        want = oracle.round_to(R.OT[ci.out_type], ref)
+        got = got.view(np.uint32) if ci.out_type == "f32" else got
+        assert np.array_equal(got, want), f"{ci.name}: 512-wide tiles differ from the oracle"
+        if M * N * K <= 2e9:
+            cr = mk(dtype, ta, tb, M, N, K, alpha=0.5, beta=2.0, case=idx, pad_a=pa, pad_b=pb)
+            dr = R.DeviceCase(cr)
+            dr.run(P.PEAK_VARIANT_UMMA_2CTA)
+            R.check_full(dr, what=f"{cr.name} 512-wide")
+
+
 def test_auto_dispatch_skinny_shapes(reset_tuning):
     """Shapes with few output tiles (the dispatcher may split K): results against the oracle, run twice
     for bit-identical output (the split reduction is in a fixed order)."""
