@@ -461,7 +461,7 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": {"f16": "f16", "bf16": "bf16", "f32": "f32"}[case.in_type] + " x, f32 accumulate",
+            "dtype": case.in_type,
             "data": "synthetic", "config": workload_config(case, l2_note),
             "variant": P.peak_variant_string(P.peak_query_variant(
                 case.dtype, case.transA, case.transB, case.M, case.N, case.K, case.alpha, dc.A, case.lda, dc.B,

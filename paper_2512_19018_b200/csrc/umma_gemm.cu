@@ -36,6 +36,9 @@ peak_mc_gemm_fn mc_entry() {
     return fn;
 }
 
+constexpr double kL2BytesPerClk = 40.0;        // L2 -> shared-memory bytes per cycle one SM sustains (measured ~39)
+constexpr double kSplitFixedCycles = 20000.0;  // workspace allocation + second launch of a split (~12 us)
+
 struct Plan {
     int bn;           // tile width: 256 or 128
     int full_tiles;   // tiles computed whole
@@ -48,7 +51,7 @@ int64_t tiles_of(const GemmArgs &g, int cg, int bn) {
 
 // Tile width and k-splitting from a small cost model (cycles): an item costs its k-blocks times the slower
 // of the tensor pipe (2*BN cycles per k-block per SM) and the operand stream (bytes per k-block over an
-// assumed 64 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread over
+// about 40 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread over
 // the units in waves.  Splitting additionally pays for writing and re-reading fp32 partials and for the
 // second launch.  Candidates: no split; every tile split s ways (few tiles); only the last wave split.
 Plan choose_plan(const GemmArgs &g, int cg, int units) {

@@ -57,8 +57,6 @@ inline int sm_count() {
     return sms[dev];
 }
 
-constexpr double kL2BytesPerClk = 64.0;      // assumed L2 -> shared-memory bandwidth per SM
-constexpr double kSplitFixedCycles = 20000.0;  // workspace allocation + second launch of a split (~12 us)
 
 }  // namespace umma
 }  // namespace peak

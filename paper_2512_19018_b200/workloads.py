@@ -8,7 +8,7 @@ see byte-identical inputs.
 
 The paper's workload is square random matrices (n = 2048, 4096; fp32 or fp16;
 section 4.3); it uses no dataset.  The cases below add the shapes, layouts and
-value distributions of the benchmark configurations this library is judged on.
+value distributions of the benchmark configurations this library is measured on.
 
 Storage convention (row-major, as in the paper's section 2.2):
   A is stored (K x M if transA else M x K) with row pitch lda,
