@@ -209,7 +209,9 @@ typedef enum peak_tuning_key {
                                    waits run out: the call's result is then wrong by design and peak_check()
                                    reports PEAK_ERR_TIMEOUT; nothing hangs and the context stays usable */
     PEAK_TUNE_MULTICAST = 10,   /* cluster-multicast plug-in: 1 = never use it, 2 = use it whenever it can run */
-    PEAK_TUNE_COUNT_ = 11
+    PEAK_TUNE_BALANCED_GRID = 11, /* 1 = always launch one CTA (pair) per SM instead of the fewest that give the
+                                     same number of waves */
+    PEAK_TUNE_COUNT_ = 12
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

@@ -21,6 +21,7 @@ struct peak_mc_request {
     int wait_ms;            // PEAK_TUNE_WAIT_MS value
     int dependent_launch;   // PEAK_TUNE_DEPENDENT_LAUNCH value
     int inject_stall;       // PEAK_TUNE_INJECT_STALL value
+    int balanced_grid;      // PEAK_TUNE_BALANCED_GRID value
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

@@ -71,7 +71,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.num_kb = (int)((r->K + BK - 1) / BK);
     p.tiles_m = (int)((r->M + 4 * BM - 1) / (4 * BM));  // 512-row super-tiles
     p.tiles_n = (int)((r->N + BN - 1) / BN);
-    p.group = r->raster_group > 0 ? r->raster_group : 4;
+    p.group = r->raster_group > 0 ? r->raster_group : 2;  // super-tile rows per raster group (measured best)
     const int tiles = p.tiles_m * p.tiles_n;
     p.full_tiles = tiles; p.tail_splits = 1; p.kb_per_split = p.num_kb; p.total_items = tiles;
     p.a_mn = a_mn; p.b_mn = b_mn;
@@ -109,6 +109,10 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
         max_clusters = (oe == cudaSuccess && n > 0) ? n : 32;
     }
     int clusters = max_clusters < tiles ? max_clusters : tiles;
+    if (r->balanced_grid != 1) {  // the fewest clusters that finish in the same number of waves
+        const int waves = (tiles + clusters - 1) / clusters;
+        clusters = (tiles + waves - 1) / waves;
+    }
     cfg.gridDim = dim3((unsigned)(clusters * 4));
     cfg.numAttrs = r->dependent_launch == 1 ? 1 : 2;
     CUtensorMap tmW = tmA;

@@ -235,7 +235,7 @@ def test_launch_counter_moves():
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(11):
+    for key in range(12):
         P.peak_set_tuning(key, 0)
 
 
