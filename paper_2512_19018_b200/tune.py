@@ -1,0 +1,152 @@
+"""Enumerating tuner: run every valid combination of the library's performance knobs on one GEMM shape and
+report the fastest.  This is the paper's "performance evaluator" (section 3.3: enumerate all valid
+tuning-parameter combinations, prune the invalid ones, keep the best) applied to `peak_set_tuning`.
+
+    python -m paper_2512_19018_b200.tune --dtype bf16_bf16 --layout NN -M 4096 -N 4096 -K 4096 [--seconds 0.3]
+
+Knobs never change results, so the tuner only times; combinations a kernel family cannot run come back as
+PEAK_ERR_UNSUPPORTED and are pruned.  Timing: CUDA events around back-to-back calls on rotating buffers.
+"""
+from __future__ import annotations
+
+import argparse
+import itertools
+import json
+import sys
+
+DTYPES = {"f16_f32": 0, "bf16_bf16": 1, "f32_f32": 2, "f16_f16": 3, "bf16_f32": 4}
+
+# knob -> candidate values (0 = library default); keys are peak_tuning_key_t
+SPACE_16BIT = {
+    "variant": ["umma_1cta", "umma_2cta"],
+    1: [128, 256, 512],          # PEAK_TUNE_TILE_N
+    2: [1, 2, 4, 8],             # PEAK_TUNE_SPLIT_K
+    3: [1, 2],                   # PEAK_TUNE_EPILOGUE
+    10: [1, 2],                  # PEAK_TUNE_MULTICAST
+    0: [0, 2, 16],               # PEAK_TUNE_RASTER_GROUP
+}
+SPACE_F32 = {
+    "variant": ["sgemm"],
+    4: [1, 2],                   # PEAK_TUNE_SGEMM_FMA
+    7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
+    0: [0, 4, 16],
+}
+NUM_KEYS = 12
+
+
+def candidates(space: dict, quick: bool = False):
+    """All combinations of the space as (variant name, {key: value}) pairs; `quick` keeps the first two values
+    of every knob."""
+    keys = [k for k in space if k != "variant"]
+    lists = [space[k][:2] if quick else space[k] for k in keys]
+    for variant in space["variant"]:
+        for combo in itertools.product(*lists):
+            yield variant, dict(zip(keys, combo))
+
+
+def prune(variant: str, knobs: dict, M: int, N: int, K: int) -> bool:
+    """Static pruning of combinations that cannot differ from another one or cannot run."""
+    if variant == "umma_1cta" and (knobs.get(1) == 512 or knobs.get(10) == 2):
+        return False                                   # 512-wide tiles and the multicast plug-in need CTA pairs
+    if knobs.get(1, 0) != 256 and knobs.get(10) == 2:
+        return False                                   # the plug-in runs 256-wide tiles only
+    if knobs.get(2, 1) > 1 and (knobs.get(1) == 512 or knobs.get(10) == 2):
+        return False                                   # no k-split with wide tiles / plug-in
+    if knobs.get(2, 1) > max(1, (K + 63) // 64):
+        return False
+    return True
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--dtype", default="bf16_bf16", choices=sorted(DTYPES))
+    ap.add_argument("--layout", default="NN", choices=["NN", "NT", "TN", "TT"])
+    ap.add_argument("-M", type=int, default=4096)
+    ap.add_argument("-N", type=int, default=4096)
+    ap.add_argument("-K", type=int, default=4096)
+    ap.add_argument("--alpha", type=float, default=1.0)
+    ap.add_argument("--beta", type=float, default=0.0)
+    ap.add_argument("--seconds", type=float, default=0.2, help="timed work per candidate")
+    ap.add_argument("--quick", action="store_true")
+    args = ap.parse_args(argv)
+
+    import numpy as np
+    import torch
+
+    from . import binding as P
+    from . import workloads as W
+
+    dtype = DTYPES[args.dtype]
+    ta, tb = args.layout[0] == "T", args.layout[1] == "T"
+    case = W.GemmCase("tune", dtype, ta, tb, args.M, args.N, args.K, args.alpha, args.beta, "uniform")
+    A_h, B_h, C_h = W.make_inputs(case, need_c0=True)
+
+    def up(a, t):
+        if t == "f32":
+            return torch.from_numpy(a).cuda()
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.float16 if t == "f16" else torch.bfloat16)
+
+    per_set = A_h.nbytes + B_h.nbytes + C_h.nbytes
+    nsets = int(max(2, min(8, 4e8 // per_set + 1)))
+    sets = [(up(A_h, case.in_type), up(B_h, case.in_type), up(C_h, case.out_type)) for _ in range(nsets)]
+    variants = {"umma_1cta": P.PEAK_VARIANT_UMMA_1CTA, "umma_2cta": P.PEAK_VARIANT_UMMA_2CTA,
+                "sgemm": P.PEAK_VARIANT_SGEMM, "auto": P.PEAK_VARIANT_AUTO}
+    space = SPACE_F32 if case.in_type == "f32" else SPACE_16BIT
+
+    def call(variant, i):
+        A, B, C = sets[i % nsets]
+        return P.peak_gemm_variant(variants[variant], dtype, ta, tb, case.M, case.N, case.K, case.alpha, A, case.lda,
+                                   B, case.ldb, case.beta, C, case.ldc, check=False)
+
+    def timed(variant, knobs):
+        for k in range(NUM_KEYS):
+            P.peak_set_tuning(k, knobs.get(k, 0))
+        rc = call(variant, 0)
+        if rc != P.PEAK_OK:
+            return None
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(3):
+            call(variant, i)
+        e1.record()
+        torch.cuda.synchronize()
+        per = max(e0.elapsed_time(e1) / 3, 1e-3)
+        steps = int(max(5, min(20000, args.seconds * 1e3 / per)))
+        e0.record()
+        for i in range(steps):
+            call(variant, i)
+        e1.record()
+        torch.cuda.synchronize()
+        if P.peak_check()[0] != P.PEAK_OK:
+            return None
+        return e0.elapsed_time(e1) / steps
+
+    results = []
+    base = timed("auto", {})
+    results.append(("auto", {}, base))
+    for variant, knobs in candidates(space, args.quick):
+        if not prune(variant, knobs, case.M, case.N, case.K):
+            continue
+        if variant.startswith("umma") and knobs.get(10) == 2 and not P.peak_multicast_available():
+            continue
+        ms = timed(variant, knobs)
+        if ms is not None:
+            results.append((variant, knobs, ms))
+    for k in range(NUM_KEYS):
+        P.peak_set_tuning(k, 0)
+    results.sort(key=lambda r: r[2])
+    best = results[0]
+    out = {"shape": [case.M, case.N, case.K], "dtype": args.dtype, "layout": args.layout,
+           "candidates_timed": len(results),
+           "auto_ms": base, "auto_tflops": case.flops / (base * 1e-3) / 1e12 if base else None,
+           "best": {"variant": best[0], "knobs": {str(k): v for k, v in best[1].items()}, "ms": best[2],
+                    "tflops": case.flops / (best[2] * 1e-3) / 1e12},
+           "top5": [{"variant": v, "knobs": {str(k): x for k, x in kn.items()}, "ms": ms} for v, kn, ms in results[:5]]}
+    print(json.dumps(out))
+    return out
+
+
+if __name__ == "__main__":
+    main()
+    sys.exit(0)

@@ -398,3 +398,40 @@ def test_set_tuning_rejects_bad_arguments():
         P.peak_set_tuning(99, 1)
     with pytest.raises(P.PeakError):
         P.peak_set_tuning(P.PEAK_TUNE_TILE_N, -1)
+
+
+def test_tuner_runs_and_restores_defaults():
+    from paper_2512_19018_b200 import tune
+    out = tune.main(["--dtype", "bf16_bf16", "--layout", "NT", "-M", "512", "-N", "512", "-K", "512", "--seconds",
+                     "0.002", "--quick"])
+    assert out["candidates_timed"] >= 4 and out["best"]["ms"] <= out["auto_ms"] * 1.5
+    # the tuner leaves the library at its defaults
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 512, 512, 512)
+    dc = R.DeviceCase(c)
+    dc.run()
+    R.check_full(dc)
+
+
+def test_cuda_graph_capture_and_replay():
+    """Calls that need no workspace allocate nothing and can be captured into a CUDA graph; replays recompute
+    C from whatever A and B then hold."""
+    c = mk(W.PEAK_BF16_BF16, 0, 0, 768, 512, 384)
+    dc = R.DeviceCase(c)
+    stream = torch.cuda.Stream()
+    dc.run(stream=None)                                        # warm-up outside the capture (first-use set-up)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            P.peak_gemm(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta, dc.C,
+                        c.ldc, stream)
+    dc.reset_c_in_place = None
+    dc.C.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert P.peak_check()[0] == P.PEAK_OK
+    R.check_full(dc)
+    dc.A.mul_(2.0)                                             # new operand values, same buffers
+    dc.A_h = R.to_host(dc.A, c.in_type)
+    graph.replay()
+    torch.cuda.synchronize()
+    R.check_full(dc)

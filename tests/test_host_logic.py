@@ -132,3 +132,16 @@ def test_workload_generators_are_seeded_and_shaped():
     A, B, C0 = W.make_inputs(p)
     assert A.shape == (5, 9) and np.isnan(A[:, 7:]).all() and C0.shape == (5, 7)
     assert W.config1().min_bytes() == 3 * 4096 * 4096 * 2
+
+
+def test_tuner_enumerates_and_prunes():
+    from paper_2512_19018_b200 import tune
+    cands = [(v, k) for v, k in tune.candidates(tune.SPACE_16BIT) if tune.prune(v, k, 4096, 4096, 4096)]
+    assert len(cands) > 20 and len(set((v, tuple(sorted(k.items()))) for v, k in cands)) == len(cands)
+    for v, k in cands:
+        assert not (v == "umma_1cta" and k.get(1) == 512)             # wide tiles need CTA pairs
+        assert not (k.get(10) == 2 and k.get(1) != 256)                # the plug-in runs 256-wide tiles only
+        assert not (k.get(2, 1) > 1 and k.get(1) == 512)
+    # a k-split cannot have more slices than k-blocks
+    assert not tune.prune("umma_2cta", {1: 256, 2: 8, 3: 2, 10: 1, 0: 0}, 256, 256, 128)
+    assert len(list(tune.candidates(tune.SPACE_F32, quick=True))) == 8
