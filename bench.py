@@ -223,12 +223,14 @@ def aggregate_value(case, world: int, steps: int, max_ms: float) -> float:
     return world * case.flops * steps / (max_ms * 1e-3) / 1e12
 
 
-def workload_config(case, l2_note):
+def workload_config(case, l2_note, epilogue="none"):
     cfg = {"workload": case.name, "M": case.M, "N": case.N, "K": case.K, "layout": case.layout,
            "in": case.in_type, "out": case.out_type, "alpha": case.alpha, "beta": case.beta,
            "inputs": case.dist, "seed": case.seed}
     if l2_note:
         cfg["l2"] = l2_note
+    if epilogue != "none":
+        cfg["fused_epilogue"] = epilogue
     return cfg
 
 
@@ -242,6 +244,8 @@ def main():
     ap.add_argument("--workload", default="bf16_4096_nn")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads and the CPU baseline")
+    ap.add_argument("--epilogue", default="none", choices=["none", "bias", "bias_relu", "bias_gelu"],
+                    help="time peak_gemm_fused with this fused tail instead of peak_gemm")
     ap.add_argument("--tune", default="", help="comma-separated key=value pairs passed to peak_set_tuning")
     ap.add_argument("--list", action="store_true")
     args = ap.parse_args()
@@ -289,10 +293,20 @@ def main():
         """W warm-up steps, then exactly `steps` back-to-back calls timed with CUDA events on the launching
         stream, rotating through `sets` so that no step finds its inputs in L2."""
         stream = torch.cuda.current_stream()
+        act = {"none": P.PEAK_ACT_NONE, "bias": P.PEAK_ACT_NONE, "bias_relu": P.PEAK_ACT_RELU,
+               "bias_gelu": P.PEAK_ACT_GELU}[args.epilogue]
+        bias = None
+        if args.epilogue != "none":
+            rng = np.random.Generator(np.random.Philox(case.seed + 99))
+            bias = torch.from_numpy(rng.standard_normal(case.N, dtype=np.float32)).cuda()
         def step(i):
             A, B, C = sets[i % len(sets)]
-            P.peak_gemm_variant(variant, case.dtype, case.transA, case.transB, case.M, case.N, case.K, case.alpha,
-                                A, case.lda, B, case.ldb, case.beta, C, case.ldc, stream)
+            if args.epilogue == "none":
+                P.peak_gemm_variant(variant, case.dtype, case.transA, case.transB, case.M, case.N, case.K, case.alpha,
+                                    A, case.lda, B, case.ldb, case.beta, C, case.ldc, stream)
+            else:
+                P.peak_gemm_fused(case.dtype, case.transA, case.transB, case.M, case.N, case.K, case.alpha, A, case.lda,
+                                  B, case.ldb, case.beta, C, case.ldc, bias, act, stream, variant=variant)
         for i in range(warmup):
             step(i)
         rc, detail = P.peak_check(stream)
@@ -462,7 +476,7 @@ def main():
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": case.in_type,
-            "data": "synthetic", "config": workload_config(case, l2_note),
+            "data": "synthetic", "config": workload_config(case, l2_note, args.epilogue),
             "variant": P.peak_variant_string(P.peak_query_variant(
                 case.dtype, case.transA, case.transB, case.M, case.N, case.K, case.alpha, dc.A, case.lda, dc.B,
                 case.ldb, case.beta, dc.C, case.ldc)) if variant == P.PEAK_VARIANT_AUTO else args.variant,

@@ -71,6 +71,13 @@ typedef enum peak_status {
     PEAK_ERR_WORKSPACE_TOO_SMALL = 7 /* peak_gemm_static_ws: the partial tiles do not fit the fixed workspace */
 } peak_status_t;
 
+/* Activation of the fused epilogue. */
+typedef enum peak_activation {
+    PEAK_ACT_NONE = 0,
+    PEAK_ACT_RELU = 1, /* max(x, 0) */
+    PEAK_ACT_GELU = 2  /* 0.5 x (1 + erf(x / sqrt 2)) */
+} peak_activation_t;
+
 /* Kernel families.  PEAK_VARIANT_AUTO lets the dispatcher choose. */
 typedef enum peak_variant {
     PEAK_VARIANT_AUTO = 0,
@@ -108,6 +115,25 @@ int peak_gemm(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K
 int peak_gemm_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
                       const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc,
                       void *stream);
+
+/*
+ * peak_gemm_fused: GEMM with a fused epilogue tail,
+ *     C = act( alpha*op(A)*op(B) + beta*C + bias ),   bias broadcast down the rows (one value per column).
+ * The paper builds its kernels incrementally so that neighbouring operations can be fused into them
+ * (sections 1 and 3.2); this is that fusion for the two operations that follow a linear layer.
+ *   bias        device pointer to N fp32 values, or NULL for none
+ *   activation  a peak_activation_t
+ * Everything else is as for peak_gemm: same kernels, layouts, quick returns (with K == 0 or alpha == 0 the
+ * result is act(beta*C + bias)), asynchrony and errors.  The sum alpha*acc + beta*C + bias and the activation
+ * are evaluated in fp32 (erff for GELU) and rounded once to the output type.
+ * peak_gemm_fused_variant additionally names the kernel family, like peak_gemm_variant.
+ */
+int peak_gemm_fused(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+                    int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, const float *bias,
+                    int activation, void *stream);
+int peak_gemm_fused_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K,
+                            float alpha, const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C,
+                            int64_t ldc, const float *bias, int activation, void *stream);
 
 /*
  * peak_gemm_host: the same operation on HOST buffers (the paper's "driver", section 3.1: allocate,

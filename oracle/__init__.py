@@ -62,6 +62,8 @@ def _load():
         lib.oracle_gemm_points.argtypes = common + [i64, vp, vp, vp, vp]
         lib.oracle_gemm_submatrix.restype = ci
         lib.oracle_gemm_submatrix.argtypes = common + [i64, vp, i64, vp, vp, vp]
+        lib.oracle_bias_act.restype = ci
+        lib.oracle_bias_act.argtypes = [vp, i64, i64, vp, ci]
         _lib = lib
     return _lib
 
@@ -173,6 +175,24 @@ def gemm_submatrix(in_type, c_type, transA, transB, M, N, K, alpha, A, lda, B, l
     if rc:
         raise ValueError(f"oracle_gemm_submatrix failed: {rc}")
     return ref, S
+
+
+ACT_NONE, ACT_RELU, ACT_GELU = 0, 1, 2
+
+
+def bias_act(ref, bias=None, act=ACT_NONE) -> np.ndarray:
+    """Fused tail on top of a computed ref (2-D): ref + bias[col], then the activation; returns a new array."""
+    lib = _load()
+    x = np.array(ref, dtype=np.float64, order="C", copy=True)
+    if x.ndim != 2:
+        raise ValueError("ref must be 2-D")
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float64)
+    if b is not None and b.shape != (x.shape[1],):
+        raise ValueError("bias must have one value per column")
+    rc = lib.oracle_bias_act(_ptr(x), x.shape[0], x.shape[1], _ptr(b), int(act))
+    if rc:
+        raise ValueError(f"oracle_bias_act failed: {rc}")
+    return x
 
 
 def num_threads() -> int:

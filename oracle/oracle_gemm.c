@@ -20,6 +20,8 @@
  *     opB(k,j) = transB ? B[j*ldb + k] : B[k*ldb + j]
  *     C0(i,j)  = C0[i*ldc + j]
  *
+ * oracle_bias_act() applies the fused tail, ref + bias[j] followed by ReLU or GELU, on top of that.
+ *
  * Stored elements (binary16, bfloat16, binary32) are decoded to double by the
  * bit-level decoders below, exactly; nothing here includes a CUDA header.
  * bfloat16, alpha, beta, op() and leading dimensions are not in the paper;
@@ -319,6 +321,30 @@ int oracle_gemm(int in_type, int c_type, int transA, int transB, int64_t M, int6
 {
     return oracle_gemm_submatrix(in_type, c_type, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C0, ldc,
                                  M, NULL, N, NULL, ref, S);
+}
+
+/* ---- fused epilogue tail ---------------------------------------------------- */
+
+/* The library's fused entry point computes act(alpha*op(A)*op(B) + beta*C + bias) with the bias broadcast
+ * down the rows; the paper motivates such fusion (sections 1 and 3.2) without defining one.  Here the
+ * tail is applied, in fp64, to an already computed `x` (rows x cols, dense): x += bias[col], then
+ *   act 0: identity;   act 1: ReLU, max(x, 0);   act 2: GELU, 0.5 x (1 + erf(x / sqrt 2)) = x * Phi(x). */
+int oracle_bias_act(double *x, int64_t rows, int64_t cols, const double *bias, int act)
+{
+    if (rows < 0 || cols < 0 || act < 0 || act > 2 || (rows * cols > 0 && !x))
+        return ORACLE_BAD_ARG;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            double v = x[i * cols + j];
+            if (bias)
+                v += bias[j];
+            if (act == 1)
+                v = v > 0.0 ? v : (v == v ? 0.0 : v); /* NaN stays NaN */
+            else if (act == 2)
+                v = 0.5 * v * (1.0 + erf(v * 0.70710678118654752440));
+            x[i * cols + j] = v;
+        }
+    return ORACLE_OK;
 }
 
 size_t oracle_elem_size(int t)

@@ -22,7 +22,8 @@ _lib = None
 
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
-           "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available"]
+           "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available", "peak_gemm_fused",
+           "peak_gemm_fused_variant"]
 
 
 class PeakError(RuntimeError):
@@ -56,6 +57,10 @@ def load():
     lib.peak_gemm_static_ws.argtypes = gemm_args[:-1] + [i, vp]
     lib.peak_static_ws_bytes.restype = ctypes.c_size_t
     lib.peak_static_ws_bytes.argtypes = []
+    lib.peak_gemm_fused.restype = i
+    lib.peak_gemm_fused.argtypes = gemm_args[:-1] + [vp, i, vp]
+    lib.peak_gemm_fused_variant.restype = i
+    lib.peak_gemm_fused_variant.argtypes = [i] + gemm_args[:-1] + [vp, i, vp]
     lib.peak_multicast_available.restype = i
     lib.peak_multicast_available.argtypes = []
     lib.peak_release_staging.restype = i
@@ -139,6 +144,28 @@ def peak_gemm_static_ws(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, b
 
 def peak_static_ws_bytes() -> int:
     return load().peak_static_ws_bytes()
+
+
+PEAK_ACT_NONE, PEAK_ACT_RELU, PEAK_ACT_GELU = 0, 1, 2
+
+
+def peak_gemm_fused(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation, stream=None,
+                    check=True, variant=None):
+    """C = act(alpha*op(A)*op(B) + beta*C + bias); `variant` (optional) names the kernel family."""
+    lib = load()
+    if variant is None:
+        rc = lib.peak_gemm_fused(dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda, _ptr(B), ldb, beta,
+                                 _ptr(C), ldc, _ptr(bias), int(activation), _stream(stream))
+    else:
+        rc = lib.peak_gemm_fused_variant(int(variant), dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda,
+                                         _ptr(B), ldb, beta, _ptr(C), ldc, _ptr(bias), int(activation), _stream(stream))
+    return _raise(rc, "peak_gemm_fused") if check else rc
+
+
+def peak_gemm_fused_variant(variant, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias,
+                            activation, stream=None, check=True):
+    return peak_gemm_fused(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation,
+                           stream, check, variant)
 
 
 def peak_multicast_available() -> bool:

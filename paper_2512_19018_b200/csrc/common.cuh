@@ -38,6 +38,17 @@ __device__ __forceinline__ float epilogue_f32(float alpha, float acc, float beta
     return r;
 }
 
+// Fused epilogue tail: x + bias (one fp32 value per column), then the activation (a peak_activation_t).
+__device__ __forceinline__ float activate_f32(float x, int act) {
+    if (act == PEAK_ACT_RELU) return fmaxf(x, 0.0f);
+    if (act == PEAK_ACT_GELU) return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f));
+    return x;
+}
+__device__ __forceinline__ float finish_f32(float x, const float *bias, int64_t col, int act) {
+    if (bias) x += __ldg(bias + col);
+    return activate_f32(x, act);
+}
+
 // ---- host-side bookkeeping (api.cu owns the definitions) ---------------------------------------
 void count_launch(int n = 1);
 void set_cuda_error(cudaError_t e);
@@ -52,6 +63,8 @@ struct GemmArgs {
     void *C;
     int64_t lda, ldb, ldc;
     cudaStream_t stream;
+    const float *bias;  // fused epilogue: one fp32 value per column of C (device), or nullptr
+    int act;            // fused epilogue: a peak_activation_t
 };
 
 // kernel-family launchers; each returns a peak_status_t

@@ -22,6 +22,8 @@ struct peak_mc_request {
     int dependent_launch;   // PEAK_TUNE_DEPENDENT_LAUNCH value
     int inject_stall;       // PEAK_TUNE_INJECT_STALL value
     int balanced_grid;      // PEAK_TUNE_BALANCED_GRID value
+    const float *bias;      // fused epilogue: fp32 value per column (device) or NULL
+    int activation;         // fused epilogue: a peak_activation_t
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

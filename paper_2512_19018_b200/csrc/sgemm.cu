@@ -50,7 +50,8 @@ template <bool KCONTIG> struct Loader {
 template <bool TA, bool TB, bool PACKED>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
-             int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int group) {
+             int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int group,
+             const float *__restrict__ bias, int act) {
     __shared__ __align__(16) float As[2][SG_BK][SG_LD];
     __shared__ __align__(16) float Bs[2][SG_BK][SG_LD];
     const int tid = threadIdx.x;
@@ -126,10 +127,11 @@ sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int6
             float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
             if (beta != 0.0f) o = *dst;
             float4 r;
-            r.x = epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x);
-            r.y = epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y);
-            r.z = epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z);
-            r.w = epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w);
+            const int64_t n = n0 + tx * 4 + h * 64;
+            r.x = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x), bias, n + 0, act);
+            r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), bias, n + 1, act);
+            r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), bias, n + 2, act);
+            r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), bias, n + 3, act);
             *dst = r;
         }
     }
@@ -183,7 +185,7 @@ template <bool TA, bool TB, bool PACKED>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 sgemm_async_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m,
-                   int tiles_n, int group) {
+                   int tiles_n, int group, const float *__restrict__ bias, int act) {
     extern __shared__ __align__(16) float sg_smem[];
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
@@ -258,10 +260,11 @@ sgemm_async_kernel(int M, int N, int K, float alpha, const float *__restrict__ A
             float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
             if (beta != 0.0f) o = *dst;
             float4 r;
-            r.x = epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x);
-            r.y = epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y);
-            r.z = epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z);
-            r.w = epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w);
+            const int64_t n = n0 + tx * 4 + h * 64;
+            r.x = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x), bias, n + 0, act);
+            r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), bias, n + 1, act);
+            r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), bias, n + 2, act);
+            r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), bias, n + 3, act);
             *dst = r;
         }
     }
@@ -275,7 +278,7 @@ template <bool TA, bool TB, bool PACKED> int run_sgemm_async(const GemmArgs &g) 
     const int group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 8;
     kernel<<<(unsigned)(tiles_m * tiles_n), SG_THREADS, SA_SMEM_BYTES, g.stream>>>(
         (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-        (float *)g.C, g.ldc, tiles_m, tiles_n, group);
+        (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
@@ -293,11 +296,11 @@ template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
     if (tuning(PEAK_TUNE_SGEMM_FMA) == 1)
         sgemm_kernel<TA, TB, false><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
             (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-            (float *)g.C, g.ldc, tiles_m, tiles_n, group);
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
     else
         sgemm_kernel<TA, TB, true><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
             (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-            (float *)g.C, g.ldc, tiles_m, tiles_n, group);
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }

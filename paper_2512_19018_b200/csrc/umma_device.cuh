@@ -79,6 +79,8 @@ struct UmmaParams {
     int64_t ldc;
     int vec_ok;            // C base and pitch allow 16-byte vector access
     int tma_store;         // epilogue stores through TMA
+    const float *bias;     // fused epilogue: fp32 value per column of C, or nullptr
+    int act;               // fused epilogue: a peak_activation_t
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;
@@ -204,7 +206,7 @@ template <typename T, int BN>
 __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, bool tma, bool vec,
-                                              float alpha, float beta) {
+                                              float alpha, float beta, const float *bias = nullptr, int act = 0) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
@@ -238,6 +240,26 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[i]);
+            }
+            if (bias != nullptr) {  // fused tail: every thread of the warp adds the same 32 bias values
+                if (valid == 32 && (reinterpret_cast<uintptr_t>(bias + col) & 15u) == 0) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + col) + i);
+                        v[4 * i] += b4.x; v[4 * i + 1] += b4.y; v[4 * i + 2] += b4.z; v[4 * i + 3] += b4.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < valid) v[i] += __ldg(bias + col + i);
+                }
+            }
+            if (act == PEAK_ACT_RELU) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.0f);
+            } else if (act == PEAK_ACT_GELU) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = activate_f32(v[i], PEAK_ACT_GELU);
             }
             if (tma) stage_row32<T>(buf, lane, h, v);
             else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
@@ -509,7 +531,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // whole tile: alpha/beta epilogue straight to C
                     epilogue_tile<TOut, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C),
                                                     p.ldc, row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0,
-                                                    p.tma_store != 0, vec, p.alpha, p.beta);
+                                                    p.tma_store != 0, vec, p.alpha, p.beta, p.bias, p.act);
                 } else {
                     // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
@@ -552,7 +574,7 @@ template <typename TOut>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
                      int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
-                     int vec_ok) {
+                     int vec_ok, const float *__restrict__ bias, int act) {
     const int blocks_per_tile = gridDim.y;
     const int t = blockIdx.x;  // split tile number
     int64_t tm, tn;
@@ -590,7 +612,7 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
             }
             float rr[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) rr[k] = epilogue_f32(alpha, a4[k], beta, o[k]);
+            for (int k = 0; k < 4; ++k) rr[k] = finish_f32(epilogue_f32(alpha, a4[k], beta, o[k]), bias, j + k, act);
             if constexpr (sizeof(TOut) == 4) {
                 *reinterpret_cast<float4 *>(dst) = make_float4(rr[0], rr[1], rr[2], rr[3]);
             } else {
@@ -601,7 +623,7 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
             for (int k = 0; k < 4; ++k) {
                 if (j + k < N) {
                     const float c_old = (beta != 0.0f) ? to_f32(dst[k]) : 0.0f;
-                    dst[k] = from_f32<TOut>(epilogue_f32(alpha, a4[k], beta, c_old));
+                    dst[k] = from_f32<TOut>(finish_f32(epilogue_f32(alpha, a4[k], beta, c_old), bias, j + k, act));
                 }
             }
         }

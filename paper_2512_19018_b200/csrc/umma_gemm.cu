@@ -140,6 +140,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
               ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.ldc = g.ldc;
+    p.bias = g.bias; p.act = g.act;
     const int ob = elem_bytes(eout);
     p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0) ? 1 : 0;
     const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
@@ -193,7 +194,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     dim3 rgrid((unsigned)split_tiles, split_tiles >= 64 ? 2u : 8u);
     splitk_reduce_kernel<TOut><<<rgrid, 256, 0, g.stream>>>(ws, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
                                                             p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C,
-                                                            g.ldc, p.vec_ok);
+                                                            g.ldc, p.vec_ok, g.bias, g.act);
     count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
@@ -323,7 +324,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
             peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
-                              tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), 0};
+                              tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act, 0};
             if (!r.status) return PEAK_ERR_CUDA;
             const int rc = mc_entry()(&r);
             if (rc == PEAK_OK) { count_launch(); return rc; }

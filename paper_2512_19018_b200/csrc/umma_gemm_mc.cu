@@ -80,6 +80,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = r->alpha; p.beta = r->beta;
     p.C = r->C; p.ldc = r->ldc;
+    p.bias = r->bias; p.act = r->activation;
     const int ob = elem_bytes(eout);
     p.vec_ok = ((reinterpret_cast<uintptr_t>(r->C) % 16) == 0 && (r->ldc * ob) % 16 == 0) ? 1 : 0;
     p.tma_store = (p.vec_ok && (r->N * ob) % 16 == 0 && r->epilogue != 1) ? 1 : 0;

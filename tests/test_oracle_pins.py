@@ -309,3 +309,32 @@ def test_bad_arguments_rejected(oracle):
         oracle.gemm(0, 2, 0, 0, 4, 4, 4, 1.0, z, 4, z, 4, 1.0, None, 4)      # beta != 0 without C0
     with pytest.raises(ValueError):
         oracle.gemm_points(0, 2, 0, 0, 4, 4, 4, 1.0, z, 4, z, 4, 0.0, None, 4, [4], [0])   # row out of range
+
+
+# ---------------------------------------------------------------- fused tail (bias + activation)
+def test_bias_act_closed_forms(oracle):
+    from scipy import special, stats
+    rng = np.random.default_rng(50)
+    x = np.concatenate([rng.standard_normal((6, 40)) * 3, np.array([[0.0, -0.0, 1.0, -1.0, 8.0, -8.0, 1e-9, -1e-9] * 5])])
+    bias = rng.standard_normal(40)
+    # identity and ReLU against numpy
+    assert np.array_equal(oracle.bias_act(x, None, oracle.ACT_NONE), x)
+    assert np.array_equal(oracle.bias_act(x, bias, oracle.ACT_NONE), x + bias[None, :])
+    assert np.array_equal(oracle.bias_act(x, bias, oracle.ACT_RELU), np.maximum(x + bias[None, :], 0.0))
+    # GELU: x * Phi(x) with scipy's normal CDF, and the erf form with scipy's erf (independent implementations)
+    g = oracle.bias_act(x, None, oracle.ACT_GELU)
+    assert np.allclose(g, x * stats.norm.cdf(x), rtol=1e-13, atol=1e-15)
+    assert np.allclose(g, 0.5 * x * (1 + special.erf(x / np.sqrt(2))), rtol=1e-14, atol=0)
+    # textbook values: gelu(0) = 0, gelu(1) = Phi(1) = 0.8413447460685429..., and gelu(x) - gelu(-x) = x
+    one = oracle.bias_act(np.array([[0.0, 1.0]]), None, oracle.ACT_GELU)
+    assert one[0, 0] == 0.0 and abs(one[0, 1] - 0.8413447460685429) < 1e-15
+    assert np.allclose(g - oracle.bias_act(-x, None, oracle.ACT_GELU), x, rtol=1e-14, atol=1e-300)
+    # the bias is added per column, before the activation: a bias of -x's column maximum zeroes ReLU everywhere
+    big = -(np.abs(x).max(axis=0) + 1.0)
+    assert not oracle.bias_act(x, big, oracle.ACT_RELU).any()
+    # NaN is not swallowed by ReLU; arguments are checked
+    assert np.isnan(oracle.bias_act(np.array([[np.nan]]), None, oracle.ACT_RELU)[0, 0])
+    with pytest.raises(ValueError):
+        oracle.bias_act(x, bias[:3], oracle.ACT_NONE)
+    with pytest.raises(ValueError):
+        oracle.bias_act(x, None, 7)
