@@ -136,6 +136,23 @@ int peak_gemm_fused_variant(int variant, int dtype, int transA, int transB, int6
                             int64_t ldc, const float *bias, int activation, void *stream);
 
 /*
+ * peak_gemm_strided_batched: `batch` independent GEMMs of one shape,
+ *     C_b = alpha * op(A_b) * op(B_b) + beta * C_b,   X_b = X + b * strideX   (strides in elements),
+ * the second half of the paper's fusion / specialisation motive (sections 1, 3.1: kernels are specialised
+ * to the shapes of a workload, and attention-style workloads are batches of small GEMMs).
+ * Arguments are those of peak_gemm plus the three strides and the batch count.  strideA and strideB may be 0
+ * (the same matrix for every b); the C matrices must not overlap (strideC >= (M-1)*ldc + N, else
+ * PEAK_ERR_INVALID_VALUE).  batch == 0 does nothing.  On the tensor-core path the whole batch is ONE launch
+ * of the persistent kernel (tiles are numbered across the batch; the batch index is the third coordinate of
+ * the TMA descriptors), which needs strideA and strideB to be positive multiples of 8 elements; any other
+ * case runs one launch per matrix with the kernel peak_gemm would choose.
+ */
+int peak_gemm_strided_batched(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                              const void *A, int64_t lda, int64_t strideA, const void *B, int64_t ldb,
+                              int64_t strideB, float beta, void *C, int64_t ldc, int64_t strideC, int64_t batch,
+                              void *stream);
+
+/*
  * peak_gemm_host: the same operation on HOST buffers (the paper's "driver", section 3.1: allocate,
  * copy in, run, copy out).  A, B, C are host pointers (pinned memory makes the copies faster but is
  * not required).  Copies A and B (and C when beta != 0) to device staging buffers, runs peak_gemm,

@@ -23,7 +23,7 @@ _lib = None
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
            "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available", "peak_gemm_fused",
-           "peak_gemm_fused_variant"]
+           "peak_gemm_fused_variant", "peak_gemm_strided_batched"]
 
 
 class PeakError(RuntimeError):
@@ -61,6 +61,9 @@ def load():
     lib.peak_gemm_fused.argtypes = gemm_args[:-1] + [vp, i, vp]
     lib.peak_gemm_fused_variant.restype = i
     lib.peak_gemm_fused_variant.argtypes = [i] + gemm_args[:-1] + [vp, i, vp]
+    lib.peak_gemm_strided_batched.restype = i
+    lib.peak_gemm_strided_batched.argtypes = [i, i, i, i64, i64, i64, f, vp, i64, i64, vp, i64, i64, f, vp, i64, i64,
+                                              i64, vp]
     lib.peak_multicast_available.restype = i
     lib.peak_multicast_available.argtypes = []
     lib.peak_release_staging.restype = i
@@ -166,6 +169,13 @@ def peak_gemm_fused_variant(variant, dtype, transA, transB, M, N, K, alpha, A, l
                             activation, stream=None, check=True):
     return peak_gemm_fused(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation,
                            stream, check, variant)
+
+
+def peak_gemm_strided_batched(dtype, transA, transB, M, N, K, alpha, A, lda, strideA, B, ldb, strideB, beta, C, ldc,
+                              strideC, batch, stream=None, check=True):
+    rc = load().peak_gemm_strided_batched(dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda, strideA,
+                                          _ptr(B), ldb, strideB, beta, _ptr(C), ldc, strideC, batch, _stream(stream))
+    return _raise(rc, "peak_gemm_strided_batched") if check else rc
 
 
 def peak_multicast_available() -> bool:

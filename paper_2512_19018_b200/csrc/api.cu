@@ -179,6 +179,39 @@ int peak_gemm_fused_variant(int variant, int dtype, int transA, int transB, int6
                      activation);
 }
 
+int peak_gemm_strided_batched(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                              const void *A, int64_t lda, int64_t strideA, const void *B, int64_t ldb, int64_t strideB,
+                              float beta, void *C, int64_t ldc, int64_t strideC, int64_t batch, void *stream) {
+    t_last_cuda_error = 0;
+    int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
+    if (rc != PEAK_OK) return rc;
+    if (batch < 0 || strideA < 0 || strideB < 0 || strideC < 0) return PEAK_ERR_INVALID_VALUE;
+    if (batch > 1 && M > 0 && N > 0 && strideC < (M - 1) * ldc + N) return PEAK_ERR_INVALID_VALUE;  // C matrices overlap
+    if (batch == 0) return PEAK_OK;
+    GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, C, lda, ldb, ldc, (cudaStream_t)stream, nullptr,
+               PEAK_ACT_NONE, batch, strideA, strideB, strideC};
+    const int v = choose_variant(g);
+    if (v == PEAK_VARIANT_NONE) return PEAK_OK;
+    rc = check_arch();
+    if (rc != PEAK_OK) return rc;
+    if (v == PEAK_VARIANT_UMMA_1CTA || v == PEAK_VARIANT_UMMA_2CTA) {
+        rc = run_variant(v, g);  // one launch: the batch index is the third coordinate of the tensor maps
+        if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+    }
+    // every other kernel family: one launch per matrix
+    const int ib = elem_bytes(in_elem(dtype)), ob = elem_bytes(out_elem(dtype));
+    for (int64_t b = 0; b < batch; ++b) {
+        GemmArgs gb = g;
+        gb.batch = 0;
+        gb.A = A ? static_cast<const char *>(A) + b * strideA * ib : nullptr;
+        gb.B = B ? static_cast<const char *>(B) + b * strideB * ib : nullptr;
+        gb.C = static_cast<char *>(C) + b * strideC * ob;
+        rc = run_variant(choose_variant(gb), gb);
+        if (rc != PEAK_OK) return rc;
+    }
+    return PEAK_OK;
+}
+
 int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
                    int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream) {
     t_last_cuda_error = 0;

@@ -65,6 +65,9 @@ struct GemmArgs {
     cudaStream_t stream;
     const float *bias;  // fused epilogue: one fp32 value per column of C (device), or nullptr
     int act;            // fused epilogue: a peak_activation_t
+    int64_t batch;      // strided batch: number of independent problems (0 or 1: a single GEMM)
+    int64_t strideA, strideB, strideC;  // elements between consecutive matrices of the batch
+    int64_t nbatch() const { return batch > 1 ? batch : 1; }
 };
 
 // kernel-family launchers; each returns a peak_status_t

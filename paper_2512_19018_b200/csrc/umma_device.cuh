@@ -72,6 +72,9 @@ struct UmmaParams {
     int tail_splits;       // k-slices of every later tile (partials go to the workspace)
     int kb_per_split;
     int total_items;       // full_tiles + (tiles - full_tiles) * tail_splits
+    int batched;           // 1: the descriptors are three-dimensional, the third coordinate is the batch index
+    int tiles_per_batch;   // tiles_m * tiles_n: tile numbers run over all matrices of a strided batch
+    int64_t stride_c;      // elements between the C matrices of a batch
     int a_mn, b_mn;        // 1: operand is MN-major in memory (transA == 1 / transB == 0)
     uint32_t idesc;
     float alpha, beta;
@@ -201,12 +204,14 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
 
 // Epilogue of one accumulator tile for one warp: TMEM -> registers -> alpha/beta -> T -> staging + TMA
 // store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
-// column limit, `nrows` the row limit for `row`; (x0, y0) is where chunk 0 of this warp lands in `tm`.
+// column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
+// (z0 < 0: `tm` is two-dimensional).
 template <typename T, int BN>
 __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
-                                              int ncols, const CUtensorMap *tm, int x0, int y0, bool tma, bool vec,
-                                              float alpha, float beta, const float *bias = nullptr, int act = 0) {
+                                              int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
+                                              bool vec, float alpha, float beta, const float *bias = nullptr,
+                                              int act = 0) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
@@ -268,11 +273,26 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
             __syncwarp();
             if (lane == 0 && row0 < nrows) {
-                ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
+                if (z0 >= 0) ptx::tma_store_3d(tm, x0 + c * CHUNK_COLS, y0, z0, buf);
+                else ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
                 ptx::tma_store_commit();
             }
             ++chunk_no;
         }
+    }
+}
+
+// Tile copies with the descriptor rank chosen at run time: a single GEMM uses two-dimensional descriptors
+// (measured 1-3 % faster than three-dimensional ones with a batch of one), a strided batch three-dimensional.
+template <int CG>
+__device__ __forceinline__ void load_tile(bool batched, uint32_t dst, const CUtensorMap *tm, int x, int y, int z,
+                                          uint32_t bar) {
+    if (batched) {
+        if (CG == 1) ptx::tma_load_3d(dst, tm, x, y, z, bar);
+        else ptx::tma_load_3d_pair(dst, tm, x, y, z, bar);
+    } else {
+        if (CG == 1) ptx::tma_load_2d(dst, tm, x, y, bar);
+        else ptx::tma_load_2d_pair(dst, tm, x, y, bar);
     }
 }
 
@@ -282,7 +302,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
 // delivers it to the CTA of the same rank parity in the other pair as well.
 template <int MC> struct McOps;
 template <> struct McOps<0> {
-    __device__ static void load_b_quarter(uint32_t, const CUtensorMap *, int, int, uint32_t, uint16_t) {}
+    __device__ static void load_b_quarter(uint32_t, const CUtensorMap *, int, int, int, uint32_t, uint16_t) {}
 };
 
 template <int CG, int BN, typename TOut, int MC = 0>
@@ -362,8 +382,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             for (int item = unit; item < total_items && ok; item += num_units) {
                 const Item w = decode_item(p, item);
+                const bool batched = p.batched != 0;
+                const int bz = batched ? w.tile / p.tiles_per_batch : 0;  // matrix of the batch
                 int64_t tm, tn;
-                tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
+                tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
                 const int n_cta = (int)tn * BN + (int)rank * C_::HROWS;  // first B row of this CTA (half 0)
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
@@ -382,13 +404,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
                     const int k0 = kb * BK;
                     if (!p.a_mn) {
-                        if (CG == 1) ptx::tma_load_2d(a_dst, &tmA, k0, m_cta, bar);
-                        else ptx::tma_load_2d_pair(a_dst, &tmA, k0, m_cta, bar);
+                        load_tile<CG>(batched, a_dst, &tmA, k0, m_cta, bz, bar);
                     } else {
 #pragma unroll
                         for (int h = 0; h < BM / 64; ++h) {
-                            if (CG == 1) ptx::tma_load_2d(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bar);
-                            else ptx::tma_load_2d_pair(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bar);
+                            load_tile<CG>(batched, a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bz, bar);
                         }
                     }
                     if (MC) {
@@ -397,7 +417,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint16_t mask = (uint16_t)((1u << crank) | (1u << (crank ^ 2u)));
                         const int n_q = n_cta + 64 * (int)pair;
                         McOps<MC>::load_b_quarter(b_dst + pair * ATOM_BYTES, &tmB, p.b_mn ? n_q : k0, p.b_mn ? k0 : n_q,
-                                                  bar, mask);
+                                                  bz, bar, mask);
                     } else if (!p.b_mn) {
 #pragma unroll
                         for (int hf = 0; hf < C_::HALVES; ++hf) {
@@ -405,8 +425,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             for (int h = 0; h < C_::HROWS / C_::B_BOX_ROWS; ++h) {
                                 const uint32_t d = b_dst + (hf * C_::HROWS + h * C_::B_BOX_ROWS) * 128;
                                 const int n = n_cta + hf * C_::SLOT_N + C_::B_BOX_ROWS * h;
-                                if (CG == 1) ptx::tma_load_2d(d, &tmB, k0, n, bar);
-                                else ptx::tma_load_2d_pair(d, &tmB, k0, n, bar);
+                                load_tile<CG>(batched, d, &tmB, k0, n, bz, bar);
                             }
                         }
                     } else {
@@ -416,8 +435,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             for (int h = 0; h < C_::HROWS / 64; ++h) {
                                 const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * ATOM_BYTES;
                                 const int n = n_cta + hf * C_::SLOT_N + 64 * h;
-                                if (CG == 1) ptx::tma_load_2d(d, &tmB, n, k0, bar);
-                                else ptx::tma_load_2d_pair(d, &tmB, n, k0, bar);
+                                load_tile<CG>(batched, d, &tmB, n, k0, bz, bar);
                             }
                         }
                     }
@@ -509,8 +527,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
             const Item w = decode_item(p, item);
+            const int bz = p.batched ? w.tile / p.tiles_per_batch : 0;
             int64_t tm, tn;
-            tile_coord(w.tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
+            tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
             const int n0 = (int)tn * BN;
 #pragma unroll 1
@@ -529,14 +548,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nh = n0 + hf * C_::SLOT_N;  // first column of this half
                 if (w.ws_block < 0) {
                     // whole tile: alpha/beta epilogue straight to C
-                    epilogue_tile<TOut, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, reinterpret_cast<TOut *>(p.C),
-                                                    p.ldc, row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0,
+                    epilogue_tile<TOut, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane,
+                                                    reinterpret_cast<TOut *>(p.C) + (int64_t)bz * p.stride_c, p.ldc,
+                                                    row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0,
+                                                    p.batched ? bz : -1,
                                                     p.tma_store != 0, vec, p.alpha, p.beta, p.bias, p.act);
                 } else {
                     // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
                     epilogue_tile<float, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane,
-                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, true, true, 1.0f, 0.0f);
+                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, -1, true, true, 1.0f,
+                                                     0.0f);
                 }
                 // hand the accumulator slot back to the MMA issuer
                 ptx::tc_fence_before_sync();
@@ -574,11 +596,15 @@ template <typename TOut>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
                      int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
-                     int vec_ok, const float *__restrict__ bias, int act) {
+                     int64_t stride_c, int vec_ok, const float *__restrict__ bias, int act) {
     const int blocks_per_tile = gridDim.y;
     const int t = blockIdx.x;  // split tile number
+    const int tiles_per_batch = tiles_m * tiles_n;
+    const int gt = full_tiles + t;           // tile number over the whole batch
+    const int bz = gt / tiles_per_batch;
+    C += (int64_t)bz * stride_c;
     int64_t tm, tn;
-    tile_coord(full_tiles + t, tiles_m, tiles_n, group, tm, tn);
+    tile_coord(gt - bz * tiles_per_batch, tiles_m, tiles_n, group, tm, tn);
     const int vec_per_row = bn / 4;
     const int total_vec = rows_t * vec_per_row;
     const int64_t block_elems = (int64_t)rows_t * bn;

@@ -45,8 +45,9 @@ struct Plan {
     int tail_splits;  // k-slices of each remaining tile (1 when nothing is split)
 };
 
+// Tiles of the whole call (all matrices of a strided batch).
 int64_t tiles_of(const GemmArgs &g, int cg, int bn) {
-    return ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn);
+    return ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn) * g.nbatch();
 }
 
 // Tile width and k-splitting from a small cost model (cycles): an item costs its k-blocks times the slower
@@ -117,10 +118,12 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const int a_mn = g.transA ? 1 : 0;  // A stored K x M: M is the contiguous index
     const int b_mn = g.transB ? 0 : 1;  // B stored K x N: N is the contiguous index
     CUtensorMap tmA, tmB, tmC, tmW;
-    bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK) : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BK, 128);
-    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK)
-                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, C_::B_BOX_ROWS));
-    if (!ok) return PEAK_ERR_CUDA;
+    const int64_t nb = g.nbatch();
+    bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK, nb, g.strideA)
+                   : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BK, 128, nb, g.strideA);
+    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK, nb, g.strideB)
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, C_::B_BOX_ROWS, nb, g.strideB));
+    if (!ok) return nb > 1 ? PEAK_ERR_UNSUPPORTED : PEAK_ERR_CUDA;  // e.g. a batch stride TMA cannot express
 
     UmmaParams p;
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
@@ -129,7 +132,10 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.tiles_n = (int)((g.N + BN - 1) / BN);
     // tile-rows per raster group (measured: 16 rows of 256 x 512 tiles are 1 % faster than 8 at 8192^3)
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : ((CG == 1 || BN == 512) ? 16 : 8);
-    const int tiles = p.tiles_m * p.tiles_n;
+    p.batched = nb > 1 ? 1 : 0;
+    p.tiles_per_batch = p.tiles_m * p.tiles_n;
+    p.stride_c = g.strideC;
+    const int tiles = p.tiles_per_batch * (int)nb;
     p.full_tiles = plan.full_tiles;
     p.tail_splits = plan.tail_splits;
     p.kb_per_split = (p.num_kb + plan.tail_splits - 1) / plan.tail_splits;
@@ -142,14 +148,16 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.C = g.C; p.ldc = g.ldc;
     p.bias = g.bias; p.act = g.act;
     const int ob = elem_bytes(eout);
-    p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0) ? 1 : 0;
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0 &&
+                (nb == 1 || (g.strideC * ob) % 16 == 0)) ? 1 : 0;
     const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
     // TMA stores clip rows exactly but clip the contiguous index only at 16-byte granularity, so they are
     // used when a row of C is a whole number of 16-byte pieces; other widths take the direct-store path
     p.tma_store = (p.vec_ok && (g.N * ob) % 16 == 0 && epi != 1) ? 1 : 0;
     tmC = tmA;  // placeholders when unused
     tmW = tmA;
-    if (p.tma_store && plan.full_tiles > 0 && !make_map(&tmC, eout, g.C, g.N, g.M, g.ldc, 128 / ob, 32))
+    if (nb > 1 && (g.strideC * ob) % 16 != 0) p.tma_store = 0;  // the batch stride must suit the store map too
+    if (p.tma_store && plan.full_tiles > 0 && !make_map(&tmC, eout, g.C, g.N, g.M, g.ldc, 128 / ob, 32, nb, g.strideC))
         return PEAK_ERR_CUDA;
     if (plan.full_tiles < tiles) {
         // the workspace as one tall matrix of dense (BM*CG) x BN blocks, one per (split tile, slice)
@@ -194,7 +202,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     dim3 rgrid((unsigned)split_tiles, split_tiles >= 64 ? 2u : 8u);
     splitk_reduce_kernel<TOut><<<rgrid, 256, 0, g.stream>>>(ws, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
                                                             p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C,
-                                                            g.ldc, p.vec_ok, g.bias, g.act);
+                                                            g.ldc, g.strideC, p.vec_ok, g.bias, g.act);
     count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
@@ -297,8 +305,12 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
     if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16) return false;
     if (g.lda % 8 || g.ldb % 8) return false;  // TMA: row pitch must be a multiple of 16 bytes
     if (g.lda >= (1ll << 38) || g.ldb >= (1ll << 38) || g.ldc >= (1ll << 38)) return false;
-    const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 127) / 128);
+    const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 127) / 128) * g.nbatch();
     if (tiles * 16 >= (1ll << 31)) return false;
+    if (g.nbatch() > 1) {  // the batch is the third dimension of the tensor maps: strides in 16-byte units
+        if (g.strideA % 8 || g.strideB % 8 || g.strideA < 1 || g.strideB < 1) return false;
+        if (g.strideA >= (1ll << 38) || g.strideB >= (1ll << 38) || g.strideC >= (1ll << 38)) return false;
+    }
     return true;
 }
 
@@ -317,7 +329,8 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
     // Measured: +3 % at 4096^3, +12 % at 5000x3000x2500, but -2..-4 % on problems of 5e11 flop and more.
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
-    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && mc_entry()) {
+    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 &&
+        mc_entry()) {
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
         if (mc_mode == 2 || (super_tiles >= 32 && flops <= 3e11)) {

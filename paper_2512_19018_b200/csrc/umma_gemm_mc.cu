@@ -31,8 +31,8 @@ namespace umma {
 // 64 x 64-element box -> the same shared-memory offset in every CTA of `mask`; completion bytes are
 // signalled on the full barrier of each destination's pair leader.
 template <> struct McOps<1> {
-    __device__ static void load_b_quarter(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t leader_bar,
-                                          uint16_t mask) {
+    __device__ static void load_b_quarter(uint32_t dst, const CUtensorMap *tm, int x, int y, int /*batch: unused, the plug-in runs single GEMMs*/,
+                                          uint32_t leader_bar, uint16_t mask) {
         asm volatile(
             "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
             ".multicast::cluster [%0], [%1, {%2, %3}], [%4], %5;"
@@ -73,6 +73,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.tiles_n = (int)((r->N + BN - 1) / BN);
     p.group = r->raster_group > 0 ? r->raster_group : 2;  // super-tile rows per raster group (measured best)
     const int tiles = p.tiles_m * p.tiles_n;
+    p.batched = 0; p.tiles_per_batch = tiles; p.stride_c = 0;
     p.full_tiles = tiles; p.tail_splits = 1; p.kb_per_split = p.num_kb; p.total_items = tiles;
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;

@@ -26,20 +26,23 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Tensor map over a row-major 2-D array: `inner` contiguous elements per row, `outer` rows, `pitch`
-// elements between rows; box = box_inner x box_outer, 128-byte swizzle, zero fill.
+// Tensor map over a stack of `batch` row-major 2-D arrays `batch_stride` elements apart: `inner` contiguous
+// elements per row, `outer` rows, `pitch` elements between rows; box = box_inner x box_outer x 1, 128-byte
+// swizzle, zero fill.  batch <= 1 gives a two-dimensional map of the one matrix.
 inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
-              int box_outer) {
+              int box_outer, int64_t batch = 1, int64_t batch_stride = 0) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
                                    : e == Elem::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                                                      : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)pitch * (cuuint64_t)elem_bytes(e)};
-    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const cuuint64_t eb = (cuuint64_t)elem_bytes(e);
+    const cuuint32_t rank = batch > 1 ? 3 : 2;  // a single matrix gets a two-dimensional descriptor
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)(batch < 1 ? 1 : batch)};
+    cuuint64_t strides[2] = {(cuuint64_t)pitch * eb, (cuuint64_t)batch_stride * eb};
+    cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(tm, dt, rank, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
