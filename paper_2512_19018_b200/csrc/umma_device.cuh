@@ -72,7 +72,6 @@ struct UmmaParams {
     int tail_splits;       // k-slices of every later tile (partials go to the workspace)
     int kb_per_split;
     int total_items;       // full_tiles + (tiles - full_tiles) * tail_splits
-    int batched;           // 1: the descriptors are three-dimensional, the third coordinate is the batch index
     int tiles_per_batch;   // tiles_m * tiles_n: tile numbers run over all matrices of a strided batch
     int64_t stride_c;      // elements between the C matrices of a batch
     int a_mn, b_mn;        // 1: operand is MN-major in memory (transA == 1 / transB == 0)
@@ -205,8 +204,8 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
 // Epilogue of one accumulator tile for one warp: TMEM -> registers -> alpha/beta -> T -> staging + TMA
 // store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
 // column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
-// (z0 < 0: `tm` is two-dimensional).
-template <typename T, int BN>
+// (z0 is used when MAP3D says that `tm` is three-dimensional).
+template <typename T, int BN, bool MAP3D = false>
 __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
@@ -273,7 +272,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
             __syncwarp();
             if (lane == 0 && row0 < nrows) {
-                if (z0 >= 0) ptx::tma_store_3d(tm, x0 + c * CHUNK_COLS, y0, z0, buf);
+                if (MAP3D) ptx::tma_store_3d(tm, x0 + c * CHUNK_COLS, y0, z0, buf);
                 else ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
                 ptx::tma_store_commit();
             }
@@ -282,12 +281,12 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
     }
 }
 
-// Tile copies with the descriptor rank chosen at run time: a single GEMM uses two-dimensional descriptors
-// (measured 1-3 % faster than three-dimensional ones with a batch of one), a strided batch three-dimensional.
-template <int CG>
-__device__ __forceinline__ void load_tile(bool batched, uint32_t dst, const CUtensorMap *tm, int x, int y, int z,
-                                          uint32_t bar) {
-    if (batched) {
+// Tile copies: a single GEMM uses two-dimensional descriptors, a strided batch three-dimensional ones.  The
+// choice is a template parameter of the kernel: the single-GEMM instantiation carries no trace of the batch
+// (three-dimensional descriptors with a batch of one, or a run-time choice, measured 1-10 % slower).
+template <int CG, bool BATCHED>
+__device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar) {
+    if (BATCHED) {
         if (CG == 1) ptx::tma_load_3d(dst, tm, x, y, z, bar);
         else ptx::tma_load_3d_pair(dst, tm, x, y, z, bar);
     } else {
@@ -305,7 +304,7 @@ template <> struct McOps<0> {
     __device__ static void load_b_quarter(uint32_t, const CUtensorMap *, int, int, int, uint32_t, uint16_t) {}
 };
 
-template <int CG, int BN, typename TOut, int MC = 0>
+template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
@@ -382,8 +381,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             for (int item = unit; item < total_items && ok; item += num_units) {
                 const Item w = decode_item(p, item);
-                const bool batched = p.batched != 0;
-                const int bz = batched ? w.tile / p.tiles_per_batch : 0;  // matrix of the batch
+                const int bz = BATCHED ? w.tile / p.tiles_per_batch : 0;  // matrix of the batch
                 int64_t tm, tn;
                 tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
@@ -404,11 +402,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
                     const int k0 = kb * BK;
                     if (!p.a_mn) {
-                        load_tile<CG>(batched, a_dst, &tmA, k0, m_cta, bz, bar);
+                        load_tile<CG, BATCHED>(a_dst, &tmA, k0, m_cta, bz, bar);
                     } else {
 #pragma unroll
                         for (int h = 0; h < BM / 64; ++h) {
-                            load_tile<CG>(batched, a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bz, bar);
+                            load_tile<CG, BATCHED>(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bz, bar);
                         }
                     }
                     if (MC) {
@@ -425,7 +423,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             for (int h = 0; h < C_::HROWS / C_::B_BOX_ROWS; ++h) {
                                 const uint32_t d = b_dst + (hf * C_::HROWS + h * C_::B_BOX_ROWS) * 128;
                                 const int n = n_cta + hf * C_::SLOT_N + C_::B_BOX_ROWS * h;
-                                load_tile<CG>(batched, d, &tmB, k0, n, bz, bar);
+                                load_tile<CG, BATCHED>(d, &tmB, k0, n, bz, bar);
                             }
                         }
                     } else {
@@ -435,7 +433,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             for (int h = 0; h < C_::HROWS / 64; ++h) {
                                 const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * ATOM_BYTES;
                                 const int n = n_cta + hf * C_::SLOT_N + 64 * h;
-                                load_tile<CG>(batched, d, &tmB, n, k0, bz, bar);
+                                load_tile<CG, BATCHED>(d, &tmB, n, k0, bz, bar);
                             }
                         }
                     }
@@ -527,7 +525,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
             const Item w = decode_item(p, item);
-            const int bz = p.batched ? w.tile / p.tiles_per_batch : 0;
+            const int bz = BATCHED ? w.tile / p.tiles_per_batch : 0;
             int64_t tm, tn;
             tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
@@ -548,16 +546,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nh = n0 + hf * C_::SLOT_N;  // first column of this half
                 if (w.ws_block < 0) {
                     // whole tile: alpha/beta epilogue straight to C
-                    epilogue_tile<TOut, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane,
-                                                    reinterpret_cast<TOut *>(p.C) + (int64_t)bz * p.stride_c, p.ldc,
-                                                    row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0,
-                                                    p.batched ? bz : -1,
+                    TOut *c_base = reinterpret_cast<TOut *>(p.C);
+                    if (BATCHED) c_base += (int64_t)bz * p.stride_c;
+                    epilogue_tile<TOut, C_::SLOT_N, BATCHED>(t_addr, my_stage, chunk_no, lane, c_base, p.ldc,
+                                                    row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0, bz,
                                                     p.tma_store != 0, vec, p.alpha, p.beta, p.bias, p.act);
                 } else {
                     // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
                     epilogue_tile<float, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane,
-                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, -1, true, true, 1.0f,
+                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, 0, true, true, 1.0f,
                                                      0.0f);
                 }
                 // hand the accumulator slot back to the MMA issuer

@@ -103,10 +103,10 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     return best;
 }
 
-template <int CG, int BN, typename TOut>
+template <int CG, int BN, typename TOut, bool BATCHED>
 int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws) {
     using C_ = Cfg<CG, BN>;
-    auto kernel = umma_gemm_kernel<CG, BN, TOut>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -132,7 +132,6 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.tiles_n = (int)((g.N + BN - 1) / BN);
     // tile-rows per raster group (measured: 16 rows of 256 x 512 tiles are 1 % faster than 8 at 8192^3)
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : ((CG == 1 || BN == 512) ? 16 : 8);
-    p.batched = nb > 1 ? 1 : 0;
     p.tiles_per_batch = p.tiles_m * p.tiles_n;
     p.stride_c = g.strideC;
     const int tiles = p.tiles_per_batch * (int)nb;
@@ -211,9 +210,15 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 
 template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, int units, float *ws) {
     switch (out_elem(g.dtype)) {
-        case Elem::F32: return launch_kernel<CG, BN, float>(g, plan, units, ws);
-        case Elem::F16: return launch_kernel<CG, BN, __half>(g, plan, units, ws);
-        case Elem::BF16: return launch_kernel<CG, BN, __nv_bfloat16>(g, plan, units, ws);
+        case Elem::F32:
+            return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true>(g, plan, units, ws)
+                                  : launch_kernel<CG, BN, float, false>(g, plan, units, ws);
+        case Elem::F16:
+            return g.nbatch() > 1 ? launch_kernel<CG, BN, __half, true>(g, plan, units, ws)
+                                  : launch_kernel<CG, BN, __half, false>(g, plan, units, ws);
+        case Elem::BF16:
+            return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws)
+                                  : launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);
     }
     return PEAK_ERR_INVALID_VALUE;
 }

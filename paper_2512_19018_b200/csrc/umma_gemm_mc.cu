@@ -73,7 +73,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.tiles_n = (int)((r->N + BN - 1) / BN);
     p.group = r->raster_group > 0 ? r->raster_group : 2;  // super-tile rows per raster group (measured best)
     const int tiles = p.tiles_m * p.tiles_n;
-    p.batched = 0; p.tiles_per_batch = tiles; p.stride_c = 0;
+    p.tiles_per_batch = tiles; p.stride_c = 0;
     p.full_tiles = tiles; p.tail_splits = 1; p.kb_per_split = p.num_kb; p.total_items = tiles;
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
