@@ -19,7 +19,7 @@ import threading
 
 import numpy as np
 
-F16, BF16, F32 = 0, 1, 2
+F16, BF16, F32, E4M3, E5M2 = 0, 1, 2, 3, 4
 _NP_STORE = {F16: np.uint16, BF16: np.uint16, F32: np.uint32}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -53,6 +53,10 @@ def _load():
         lib.oracle_decode_bf16.argtypes = [ctypes.c_uint16]
         lib.oracle_decode_f32.restype = dbl
         lib.oracle_decode_f32.argtypes = [ctypes.c_uint32]
+        lib.oracle_decode_e4m3.restype = dbl
+        lib.oracle_decode_e4m3.argtypes = [ctypes.c_uint8]
+        lib.oracle_decode_e5m2.restype = dbl
+        lib.oracle_decode_e5m2.argtypes = [ctypes.c_uint8]
         lib.oracle_round.restype = ci
         lib.oracle_round.argtypes = [ci, vp, i64, vp]
         common = [ci, ci, ci, ci, i64, i64, i64, dbl, vp, i64, vp, i64, dbl, vp, i64]
@@ -77,6 +81,10 @@ def _store(a, t):
     if a is None:
         return None
     a = np.ascontiguousarray(a)
+    if t in (E4M3, E5M2):
+        if a.dtype != np.uint8:
+            raise TypeError("8-bit float operands must be uint8 bit patterns")
+        return a
     if t == F32:
         if a.dtype == np.float32:
             return a.view(np.uint32)
@@ -109,7 +117,8 @@ def _check_sizes(transA, transB, M, N, K, A, lda, B, ldb, C0, ldc, beta):
 def decode(t: int, bits) -> np.ndarray:
     """Decode stored bit patterns to float64 with the oracle's own decoders."""
     lib = _load()
-    fn = {F16: lib.oracle_decode_f16, BF16: lib.oracle_decode_bf16, F32: lib.oracle_decode_f32}[t]
+    fn = {F16: lib.oracle_decode_f16, BF16: lib.oracle_decode_bf16, F32: lib.oracle_decode_f32,
+          E4M3: lib.oracle_decode_e4m3, E5M2: lib.oracle_decode_e5m2}[t]
     flat = np.asarray(bits).ravel()
     return np.array([fn(int(b)) for b in flat], dtype=np.float64).reshape(np.shape(bits))
 

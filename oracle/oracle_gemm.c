@@ -37,7 +37,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORACLE_F16 = 0, ORACLE_BF16 = 1, ORACLE_F32 = 2 };
+enum { ORACLE_F16 = 0, ORACLE_BF16 = 1, ORACLE_F32 = 2, ORACLE_E4M3 = 3, ORACLE_E5M2 = 4 };
 
 enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1, ORACLE_NO_MEM = 2 };
 
@@ -91,9 +91,42 @@ double oracle_decode_f32(uint32_t w)
     return sign ? -v : v;
 }
 
+/* 8-bit float E4M3 ("fn" flavour used by GPUs; the paper only mentions fp8 as an existing type, section 2.1):
+ * 1 sign, 4 exponent (bias 7), 3 fraction bits; no infinities; only S.1111.111 is NaN; largest value 448. */
+double oracle_decode_e4m3(uint8_t b)
+{
+    int sign = (b >> 7) & 1;
+    int e = (b >> 3) & 0xf;
+    int f = b & 7;
+    double v;
+    if (e == 15 && f == 7)
+        v = NAN;
+    else if (e == 0)
+        v = ldexp((double)f, -9); /* subnormal: f * 2^-3 * 2^-6 */
+    else
+        v = ldexp((double)(8 + f), e - 10); /* (1 + f/8) * 2^(e-7) */
+    return sign ? -v : v;
+}
+
+/* 8-bit float E5M2: 1 sign, 5 exponent (bias 15), 2 fraction bits; IEEE-style infinities and NaNs. */
+double oracle_decode_e5m2(uint8_t b)
+{
+    int sign = (b >> 7) & 1;
+    int e = (b >> 2) & 0x1f;
+    int f = b & 3;
+    double v;
+    if (e == 0)
+        v = ldexp((double)f, -16); /* f * 2^-2 * 2^-14 */
+    else if (e == 31)
+        v = f ? NAN : INFINITY;
+    else
+        v = ldexp((double)(4 + f), e - 17); /* (1 + f/4) * 2^(e-15) */
+    return sign ? -v : v;
+}
+
 static size_t elem_size(int t)
 {
-    return t == ORACLE_F32 ? 4 : 2;
+    return t == ORACLE_F32 ? 4 : (t == ORACLE_E4M3 || t == ORACLE_E5M2) ? 1 : 2;
 }
 
 static double load_elem(int t, const void *base, int64_t idx)
@@ -102,6 +135,10 @@ static double load_elem(int t, const void *base, int64_t idx)
         return oracle_decode_f16(((const uint16_t *)base)[idx]);
     if (t == ORACLE_BF16)
         return oracle_decode_bf16(((const uint16_t *)base)[idx]);
+    if (t == ORACLE_E4M3)
+        return oracle_decode_e4m3(((const uint8_t *)base)[idx]);
+    if (t == ORACLE_E5M2)
+        return oracle_decode_e5m2(((const uint8_t *)base)[idx]);
     return oracle_decode_f32(((const uint32_t *)base)[idx]);
 }
 
@@ -181,7 +218,7 @@ int oracle_round(int type, const double *x, int64_t n, void *out)
 static int check_args(int in_type, int c_type, int transA, int transB, int64_t M, int64_t N, int64_t K,
                       int64_t lda, int64_t ldb, int64_t ldc)
 {
-    if (in_type < 0 || in_type > 2 || c_type < 0 || c_type > 2)
+    if (in_type < 0 || in_type > 4 || c_type < 0 || c_type > 2)
         return ORACLE_BAD_ARG;
     if ((transA != 0 && transA != 1) || (transB != 0 && transB != 1))
         return ORACLE_BAD_ARG;

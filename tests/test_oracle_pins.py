@@ -338,3 +338,36 @@ def test_bias_act_closed_forms(oracle):
         oracle.bias_act(x, bias[:3], oracle.ACT_NONE)
     with pytest.raises(ValueError):
         oracle.bias_act(x, None, 7)
+
+
+# ---------------------------------------------------------------- 8-bit floats
+def test_decode_fp8_exhaustive(oracle):
+    """All 256 patterns of each 8-bit format against torch's float8 types (an independent library decoder),
+    plus the format's landmark values."""
+    import torch
+    bits = np.arange(256, dtype=np.uint8)
+    for t, tt in ((oracle.E4M3, torch.float8_e4m3fn), (oracle.E5M2, torch.float8_e5m2)):
+        want = torch.from_numpy(bits.copy()).view(tt).to(torch.float32).numpy().astype(np.float64)
+        got = oracle.decode(t, bits)
+        nan = np.isnan(want)
+        assert np.array_equal(np.isnan(got), nan)
+        assert np.array_equal(got[~nan], want[~nan])
+        assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+    d4 = lambda b: oracle.decode(oracle.E4M3, [b])[0]
+    d5 = lambda b: oracle.decode(oracle.E5M2, [b])[0]
+    assert d4(0x7E) == 448.0 and np.isnan(d4(0x7F)) and d4(0x38) == 1.0 and d4(0x01) == 2.0 ** -9 and d4(0xC0) == -2.0
+    assert d5(0x7B) == 57344.0 and np.isinf(d5(0x7C)) and np.isnan(d5(0x7D)) and d5(0x3C) == 1.0 and d5(0x01) == 2.0 ** -16
+
+
+def test_fp8_gemm_exact_integers(oracle):
+    """E4M3 / E5M2 inputs holding small integers: the oracle's result equals int64 matmul exactly."""
+    import torch
+    rng = np.random.default_rng(60)
+    for t, tt in ((oracle.E4M3, torch.float8_e4m3fn), (oracle.E5M2, torch.float8_e5m2)):
+        M, N, K = 9, 14, 37
+        a = rng.integers(-4, 5, (M, K)); b = rng.integers(-4, 5, (N, K))       # NT: B stored N x K
+        A = torch.from_numpy(a.astype(np.float32)).to(tt).view(torch.uint8).numpy()
+        B = torch.from_numpy(b.astype(np.float32)).to(tt).view(torch.uint8).numpy()
+        ref, S = oracle.gemm(t, oracle.F32, 0, 1, M, N, K, 1.0, A, K, B, K, 0.0, None, N)
+        assert np.array_equal(ref, (a @ b.T).astype(np.float64))
+        assert np.array_equal(S, (np.abs(a) @ np.abs(b).T).astype(np.float64))
