@@ -58,6 +58,10 @@ def workloads_table():
         for lay in ("NN", "TN"):
             c = W.config2(n, lay)
             t[c.name] = c
+    for n in (4096, 8192):
+        for it in ("e4m3", "e5m2"):
+            c = W.fp8_workload(n, it)
+            t[c.name] = c
     for i in range(3):
         t[W.config3(i).name] = W.config3(i)
         t[W.config4_ragged(i).name] = W.config4_ragged(i)
@@ -148,7 +152,7 @@ def oracle_sampler(case, A, B, C0, target_seconds: float):
     """The CPU oracle (as it stands) on a rows x cols sub-grid of the workload sized, from a short probe,
     for roughly `target_seconds` of work.  Returns (run, description, threads); run() -> (tflops, seconds)."""
     import oracle
-    T = {"f16": oracle.F16, "bf16": oracle.BF16, "f32": oracle.F32}
+    T = {"f16": oracle.F16, "bf16": oracle.BF16, "f32": oracle.F32, "e4m3": oracle.E4M3, "e5m2": oracle.E5M2}
 
     def run_pq(p, q):
         rows = np.linspace(0, case.M - 1, p).astype(np.int64)
@@ -352,7 +356,7 @@ def main():
 
         @staticmethod
         def up(arr, t):
-            if t == "f32":
+            if t in ("f32", "e4m3", "e5m2"):          # float32 values / raw bytes
                 return torch.from_numpy(arr).cuda()
             return torch.from_numpy(arr.view(np.int16)).cuda().view(torch.float16 if t == "f16" else torch.bfloat16)
 
@@ -365,7 +369,7 @@ def main():
 
     # default K: about one second of timed work, long enough for the NVML clock samples to mean something
     # (the driver updates them every ~100 ms) and for the power cap to settle -- a sustained figure
-    expected_tflops = 55.0 if case.in_type == "f32" else 1200.0
+    expected_tflops = {"f32": 55.0, "e4m3": 2500.0, "e5m2": 2500.0}.get(case.in_type, 1200.0)
     steps = args.steps if args.steps is not None else max(20, min(20000, int(1.0 * expected_tflops * 1e12 / case.flops)))
     warmup = args.warmup if args.warmup is not None else 10
     warmup = max(warmup, 3)
@@ -384,10 +388,14 @@ def main():
         # denominator there, the burst figure for short runs
         long_run = ms >= 500.0
         burst, sustained = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+        ratio_note = ""
+        if case.in_type in ("e4m3", "e5m2"):
+            # no 8-bit peak was measured: the bf16 figure times the nominal dense ratio (4.5 / 2.25 PFLOP/s)
+            burst, sustained, ratio_note = 2.0 * burst, 2.0 * sustained, " x 2 (nominal fp8 : bf16 ratio)"
         roof = {"bound": "tensor", "achieved": case.flops / (kernel_ms * 1e-3) / 1e12,
                 "peak": sustained if long_run else burst, "unit": "TFLOP/s",
-                "peak_kind": f"{peak_kind} cuBLAS bf16 8192^3, " + ("sustained (timed region >= 0.5 s)" if long_run
-                                                                     else "burst (timed region < 0.5 s)"),
+                "peak_kind": f"{peak_kind} cuBLAS bf16 8192^3{ratio_note}, " +
+                             ("sustained (timed region >= 0.5 s)" if long_run else "burst (timed region < 0.5 s)"),
                 "frac_of_burst_peak": case.flops / (kernel_ms * 1e-3) / 1e12 / burst,
                 "frac_of_sustained_peak": case.flops / (kernel_ms * 1e-3) / 1e12 / sustained}
     roof["frac"] = roof["achieved"] / roof["peak"]
@@ -400,8 +408,9 @@ def main():
     e2e = None
     if rank == 0 or distributed:
         c = dc.case
-        hA = torch.from_numpy(dc.A_h.view(np.int16) if c.in_type != "f32" else dc.A_h).pin_memory()
-        hB = torch.from_numpy(dc.B_h.view(np.int16) if c.in_type != "f32" else dc.B_h).pin_memory()
+        two_byte = c.in_type in ("f16", "bf16")
+        hA = torch.from_numpy(dc.A_h.view(np.int16) if two_byte else dc.A_h).pin_memory()
+        hB = torch.from_numpy(dc.B_h.view(np.int16) if two_byte else dc.B_h).pin_memory()
         hC = torch.from_numpy(dc.C0_h.view(np.int16) if c.out_type != "f32" else dc.C0_h).clone().pin_memory()
         h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + \
             (hC.numel() * hC.element_size() if c.beta != 0 else 0)
@@ -451,8 +460,19 @@ def main():
             csets, _ = make_sets(case, dcc)
             opA = [(a.t() if case.transA else a)[:case.M, :case.K] for a, _, _ in csets]
             opB = [(b.t() if case.transB else b)[:case.K, :case.N] for _, b, _ in csets]
-            def mm(i):
-                torch.matmul(opA[i % len(csets)], opB[i % len(csets)])
+            if case.in_type in ("e4m3", "e5m2"):
+                # the library's 8-bit GEMM (cuBLASLt through torch._scaled_mm) with unit scales
+                f8 = torch.float8_e4m3fn if case.in_type == "e4m3" else torch.float8_e5m2
+                opA = [a.view(f8) for a in opA]
+                opB = [b.view(f8) for b in opB]
+                one = torch.ones((), dtype=torch.float32, device="cuda")
+                out_t = torch.bfloat16 if case.out_type == "bf16" else torch.float32
+                def mm(i):
+                    torch._scaled_mm(opA[i % len(csets)], opB[i % len(csets)], scale_a=one, scale_b=one,
+                                     out_dtype=out_t)
+            else:
+                def mm(i):
+                    torch.matmul(opA[i % len(csets)], opB[i % len(csets)])
             for i in range(10):
                 mm(i)
             torch.cuda.synchronize()
@@ -463,7 +483,7 @@ def main():
             c1.record()
             torch.cuda.synchronize()
             extra["cublas_context"] = {"workload": case.name, "tflops": case.flops * steps / (c0.elapsed_time(c1) * 1e-3) / 1e12,
-                                       "steps": steps, "note": "torch.matmul, same rotation and step count; not this library"}
+                                       "steps": steps, "note": "torch.matmul (torch._scaled_mm for 8-bit inputs), same rotation and step count; not this library"}
             del dcc, csets, opA, opB
         except Exception as exc:  # context only: never fail the bench for it
             extra["cublas_context"] = {"error": str(exc)[:200]}

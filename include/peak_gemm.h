@@ -57,7 +57,13 @@ typedef enum peak_dtype {
     PEAK_BF16_BF16 = 1, /* A, B bfloat16; C bfloat16 */
     PEAK_F32_F32 = 2,   /* A, B, C binary32 (CUDA-core SGEMM, no TF32) */
     PEAK_F16_F16 = 3,   /* A, B, C binary16 */
-    PEAK_BF16_F32 = 4   /* A, B bfloat16; C binary32 */
+    PEAK_BF16_F32 = 4,  /* A, B bfloat16; C binary32 */
+    /* 8-bit float inputs (the paper names fp8 only as an existing GPU type, section 2.1): E4M3 is the "fn"
+       flavour (no infinities, one NaN pattern, largest value 448), E5M2 the IEEE-style one. */
+    PEAK_E4M3_BF16 = 5, /* A, B E4M3; C bfloat16 */
+    PEAK_E4M3_F32 = 6,  /* A, B E4M3; C binary32 */
+    PEAK_E5M2_BF16 = 7, /* A, B E5M2; C bfloat16 */
+    PEAK_E5M2_F32 = 8   /* A, B E5M2; C binary32 */
 } peak_dtype_t;
 
 typedef enum peak_status {
@@ -101,7 +107,8 @@ typedef enum peak_variant {
  *   lda, ldb, ldc  row pitches in elements
  *   stream         cudaStream_t
  * The fastest variant whose preconditions hold is chosen: the tensor-core path needs 16-byte aligned
- * base pointers and row pitches that are multiples of 16 bytes; anything else runs on the fallback
+ * base pointers and row pitches that are multiples of 16 bytes, and for the 8-bit input types also
+ * transA = 0, transB = 1 (both operands stored with K innermost); anything else runs on the fallback
  * kernel with the same result contract.  Returns after enqueueing; never synchronises.
  */
 int peak_gemm(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,

@@ -11,6 +11,7 @@ import ctypes
 import os
 
 PEAK_F16_F32, PEAK_BF16_BF16, PEAK_F32_F32, PEAK_F16_F16, PEAK_BF16_F32 = 0, 1, 2, 3, 4
+PEAK_E4M3_BF16, PEAK_E4M3_F32, PEAK_E5M2_BF16, PEAK_E5M2_F32 = 5, 6, 7, 8
 PEAK_OK, PEAK_ERR_INVALID_VALUE, PEAK_ERR_ARCH, PEAK_ERR_CUDA, PEAK_ERR_UNSUPPORTED, PEAK_ERR_TIMEOUT, \
     PEAK_ERR_NO_MEMORY, PEAK_ERR_WORKSPACE_TOO_SMALL = range(8)
 PEAK_VARIANT_AUTO, PEAK_VARIANT_FALLBACK, PEAK_VARIANT_UMMA_1CTA, PEAK_VARIANT_UMMA_2CTA, PEAK_VARIANT_SGEMM, \

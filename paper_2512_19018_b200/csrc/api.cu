@@ -43,7 +43,7 @@ uint32_t *device_status_word() {
 
 namespace {
 
-bool valid_dtype(int d) { return d >= PEAK_F16_F32 && d <= PEAK_BF16_F32; }
+bool valid_dtype(int d) { return d >= PEAK_F16_F32 && d <= PEAK_E5M2_F32; }
 
 // Returns PEAK_OK or PEAK_ERR_INVALID_VALUE; checks only the arguments, touches no device.
 int validate(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, const void *A, int64_t lda,

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -10,21 +11,30 @@
 namespace peak {
 
 // ---- storage types ---------------------------------------------------------------------------
-enum class Elem : int { F16 = 0, BF16 = 1, F32 = 2 };
+enum class Elem : int { F16 = 0, BF16 = 1, F32 = 2, E4M3 = 3, E5M2 = 4 };
 
 __host__ __device__ inline Elem in_elem(int dtype) {
-    return (dtype == PEAK_F16_F32 || dtype == PEAK_F16_F16) ? Elem::F16
-           : (dtype == PEAK_F32_F32)                       ? Elem::F32
-                                                           : Elem::BF16;
+    return (dtype == PEAK_F16_F32 || dtype == PEAK_F16_F16)     ? Elem::F16
+           : (dtype == PEAK_F32_F32)                           ? Elem::F32
+           : (dtype == PEAK_E4M3_BF16 || dtype == PEAK_E4M3_F32) ? Elem::E4M3
+           : (dtype == PEAK_E5M2_BF16 || dtype == PEAK_E5M2_F32) ? Elem::E5M2
+                                                               : Elem::BF16;
 }
 __host__ __device__ inline Elem out_elem(int dtype) {
-    return (dtype == PEAK_BF16_BF16) ? Elem::BF16 : (dtype == PEAK_F16_F16) ? Elem::F16 : Elem::F32;
+    return (dtype == PEAK_BF16_BF16 || dtype == PEAK_E4M3_BF16 || dtype == PEAK_E5M2_BF16) ? Elem::BF16
+           : (dtype == PEAK_F16_F16)                                                       ? Elem::F16
+                                                                                           : Elem::F32;
 }
-__host__ __device__ inline int elem_bytes(Elem e) { return e == Elem::F32 ? 4 : 2; }
+__host__ __device__ inline int elem_bytes(Elem e) {
+    return e == Elem::F32 ? 4 : (e == Elem::E4M3 || e == Elem::E5M2) ? 1 : 2;
+}
+__host__ __device__ inline bool is_fp8(Elem e) { return e == Elem::E4M3 || e == Elem::E5M2; }
 
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__nv_fp8_e4m3 v) { return float(v); }
+__device__ __forceinline__ float to_f32(__nv_fp8_e5m2 v) { return float(v); }
 
 template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }

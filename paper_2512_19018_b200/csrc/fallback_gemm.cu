@@ -153,6 +153,10 @@ int launch_fallback(const GemmArgs &g) {
         case PEAK_F32_F32: return run_fallback<float, float>(g);
         case PEAK_F16_F16: return run_fallback<__half, __half>(g);
         case PEAK_BF16_F32: return run_fallback<__nv_bfloat16, float>(g);
+        case PEAK_E4M3_BF16: return run_fallback<__nv_fp8_e4m3, __nv_bfloat16>(g);
+        case PEAK_E4M3_F32: return run_fallback<__nv_fp8_e4m3, float>(g);
+        case PEAK_E5M2_BF16: return run_fallback<__nv_fp8_e5m2, __nv_bfloat16>(g);
+        case PEAK_E5M2_F32: return run_fallback<__nv_fp8_e5m2, float>(g);
     }
     return PEAK_ERR_INVALID_VALUE;
 }
@@ -164,6 +168,10 @@ int launch_xcheck_f64(const GemmArgs &g, const void *C0, double *Cref, int64_t l
         case PEAK_F32_F32: return run_xcheck<float, float>(g, C0, Cref, ldcref);
         case PEAK_F16_F16: return run_xcheck<__half, __half>(g, C0, Cref, ldcref);
         case PEAK_BF16_F32: return run_xcheck<__nv_bfloat16, float>(g, C0, Cref, ldcref);
+        case PEAK_E4M3_BF16: return run_xcheck<__nv_fp8_e4m3, __nv_bfloat16>(g, C0, Cref, ldcref);
+        case PEAK_E4M3_F32: return run_xcheck<__nv_fp8_e4m3, float>(g, C0, Cref, ldcref);
+        case PEAK_E5M2_BF16: return run_xcheck<__nv_fp8_e5m2, __nv_bfloat16>(g, C0, Cref, ldcref);
+        case PEAK_E5M2_F32: return run_xcheck<__nv_fp8_e5m2, float>(g, C0, Cref, ldcref);
     }
     return PEAK_ERR_INVALID_VALUE;
 }

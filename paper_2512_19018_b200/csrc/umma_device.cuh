@@ -65,7 +65,7 @@ template <int CG, int BN> struct Cfg {
 
 struct UmmaParams {
     int M, N, K;
-    int num_kb;            // ceil(K / BK)
+    int num_kb;            // k-blocks: ceil(K / 64) for 16-bit inputs, ceil(K / 128) for 8-bit ones
     int tiles_m, tiles_n;  // in units of (128*CG) x BN
     int group;             // tile-rows per raster group
     int full_tiles;        // tiles [0, full_tiles) are computed whole and stored to C
@@ -304,7 +304,10 @@ template <> struct McOps<0> {
     __device__ static void load_b_quarter(uint32_t, const CUtensorMap *, int, int, int, uint32_t, uint16_t) {}
 };
 
-template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false>
+// IN8: the inputs are 8-bit floats.  A k-block is still one 128-byte swizzle row per matrix row, so it holds
+// 128 elements instead of 64, every byte count and descriptor stays as it is, and the MMA is the f8f6f4 kind
+// with K = 32 per instruction.  Both operands must be K-major (A not transposed, B transposed).
+template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
@@ -400,7 +403,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (CG == 2) bar = ptx::map_to_cta(bar, leader_crank);
                     const uint32_t a_dst = stage_base + s * C_::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                    const int k0 = kb * BK;
+                    const int k0 = kb * (IN8 ? 2 * BK : BK);  // element coordinate of the k-block
                     if (!p.a_mn) {
                         load_tile<CG, BATCHED>(a_dst, &tmA, k0, m_cta, bz, bar);
                     } else {
@@ -498,7 +501,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         for (int k = 0; k < BK / UMMA_K; ++k) {
                             const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
                             const uint64_t bd = smem_desc(bh_base + k * b_kstep, b_lbo, 1024u);
-                            ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
+                            if (IN8) ptx::umma_f8<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
+                            else ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
                         }
                     }
                     if (!ok) break;

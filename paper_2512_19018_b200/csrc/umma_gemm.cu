@@ -56,7 +56,8 @@ int64_t tiles_of(const GemmArgs &g, int cg, int bn) {
 // the units in waves.  Splitting additionally pays for writing and re-reading fp32 partials and for the
 // second launch.  Candidates: no split; every tile split s ways (few tiles); only the last wave split.
 Plan choose_plan(const GemmArgs &g, int cg, int units) {
-    const int64_t num_kb = (g.K + BK - 1) / BK;
+    const int bke = is_fp8(in_elem(g.dtype)) ? 2 * BK : BK;  // elements per k-block (one 128-byte row)
+    const int64_t num_kb = (g.K + bke - 1) / bke;
     Plan best{256, 0, 1};
     double best_cost = 1e300;
     const int force_bn = tuning(PEAK_TUNE_TILE_N), force_split = tuning(PEAK_TUNE_SPLIT_K);
@@ -103,10 +104,11 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     return best;
 }
 
-template <int CG, int BN, typename TOut, bool BATCHED>
+template <int CG, int BN, typename TOut, bool BATCHED, bool IN8 = false>
 int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws) {
     using C_ = Cfg<CG, BN>;
-    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED>;
+    constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -119,15 +121,16 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const int b_mn = g.transB ? 0 : 1;  // B stored K x N: N is the contiguous index
     CUtensorMap tmA, tmB, tmC, tmW;
     const int64_t nb = g.nbatch();
+    if (IN8 && (a_mn || b_mn)) return PEAK_ERR_UNSUPPORTED;  // 8-bit operands: K-major only
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK, nb, g.strideA)
-                   : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BK, 128, nb, g.strideA);
+                   : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, 128, nb, g.strideA);
     ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK, nb, g.strideB)
-                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BK, C_::B_BOX_ROWS, nb, g.strideB));
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS, nb, g.strideB));
     if (!ok) return nb > 1 ? PEAK_ERR_UNSUPPORTED : PEAK_ERR_CUDA;  // e.g. a batch stride TMA cannot express
 
     UmmaParams p;
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
-    p.num_kb = (int)((g.K + BK - 1) / BK);
+    p.num_kb = (int)((g.K + BKE - 1) / BKE);
     p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((g.N + BN - 1) / BN);
     // tile-rows per raster group (measured: 16 rows of 256 x 512 tiles are 1 % faster than 8 at 8192^3)
@@ -140,7 +143,8 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.kb_per_split = (p.num_kb + plan.tail_splits - 1) / plan.tail_splits;
     p.total_items = plan.full_tiles + (tiles - plan.full_tiles) * plan.tail_splits;
     p.a_mn = a_mn; p.b_mn = b_mn;
-    const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
+    // operand format field: f16 kind: 0 = fp16, 1 = bf16; f8f6f4 kind: 0 = E4M3, 1 = E5M2
+    const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
@@ -211,12 +215,18 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, int units, float *ws) {
     switch (out_elem(g.dtype)) {
         case Elem::F32:
+            if (is_fp8(in_elem(g.dtype)))
+                return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true, true>(g, plan, units, ws)
+                                      : launch_kernel<CG, BN, float, false, true>(g, plan, units, ws);
             return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true>(g, plan, units, ws)
                                   : launch_kernel<CG, BN, float, false>(g, plan, units, ws);
         case Elem::F16:
             return g.nbatch() > 1 ? launch_kernel<CG, BN, __half, true>(g, plan, units, ws)
                                   : launch_kernel<CG, BN, __half, false>(g, plan, units, ws);
         case Elem::BF16:
+            if (is_fp8(in_elem(g.dtype)))
+                return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true, true>(g, plan, units, ws)
+                                      : launch_kernel<CG, BN, __nv_bfloat16, false, true>(g, plan, units, ws);
             return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws)
                                   : launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);
     }
@@ -308,12 +318,15 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
     if (g.M < 1 || g.N < 1 || g.K < 1) return false;
     if (g.M >= (1ll << 31) - 512 || g.N >= (1ll << 31) - 512 || g.K >= (1ll << 31) - 512) return false;
     if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16) return false;
-    if (g.lda % 8 || g.ldb % 8) return false;  // TMA: row pitch must be a multiple of 16 bytes
+    const bool in8 = is_fp8(in_elem(g.dtype));
+    if (in8 && (g.transA || !g.transB)) return false;  // 8-bit operands: K-major only (A as is, B transposed)
+    const int pitch_unit = in8 ? 16 : 8;               // TMA: row pitch must be a multiple of 16 bytes
+    if (g.lda % pitch_unit || g.ldb % pitch_unit) return false;
     if (g.lda >= (1ll << 38) || g.ldb >= (1ll << 38) || g.ldc >= (1ll << 38)) return false;
     const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 127) / 128) * g.nbatch();
     if (tiles * 16 >= (1ll << 31)) return false;
     if (g.nbatch() > 1) {  // the batch is the third dimension of the tensor maps: strides in 16-byte units
-        if (g.strideA % 8 || g.strideB % 8 || g.strideA < 1 || g.strideB < 1) return false;
+        if (g.strideA % pitch_unit || g.strideB % pitch_unit || g.strideA < 1 || g.strideB < 1) return false;
         if (g.strideA >= (1ll << 38) || g.strideB >= (1ll << 38) || g.strideC >= (1ll << 38)) return false;
     }
     return true;
@@ -335,7 +348,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // Measured: +3 % at 4096^3, +12 % at 5000x3000x2500, but -2..-4 % on problems of 5e11 flop and more.
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
     if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 &&
-        mc_entry()) {
+        !is_fp8(in_elem(g.dtype)) && mc_entry()) {
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
         if (mc_mode == 2 || (super_tiles >= 32 && flops <= 3e11)) {

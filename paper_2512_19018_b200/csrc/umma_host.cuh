@@ -35,6 +35,7 @@ inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, i
     if (!fn) return false;
     const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
                                    : e == Elem::BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                   : is_fp8(e)       ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                                      : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     const cuuint64_t eb = (cuuint64_t)elem_bytes(e);
     const cuuint32_t rank = batch > 1 ? 3 : 2;  // a single matrix gets a two-dimensional descriptor

@@ -29,13 +29,17 @@ BASE_SEED = 0x5045414B  # "PEAK"
 
 # dtype pair codes of the C ABI (include/peak_gemm.h)
 PEAK_F16_F32, PEAK_BF16_BF16, PEAK_F32_F32, PEAK_F16_F16, PEAK_BF16_F32 = 0, 1, 2, 3, 4
+PEAK_E4M3_BF16, PEAK_E4M3_F32, PEAK_E5M2_BF16, PEAK_E5M2_F32 = 5, 6, 7, 8
 IN_TYPE = {PEAK_F16_F32: "f16", PEAK_BF16_BF16: "bf16", PEAK_F32_F32: "f32", PEAK_F16_F16: "f16",
-           PEAK_BF16_F32: "bf16"}
+           PEAK_BF16_F32: "bf16", PEAK_E4M3_BF16: "e4m3", PEAK_E4M3_F32: "e4m3", PEAK_E5M2_BF16: "e5m2",
+           PEAK_E5M2_F32: "e5m2"}
 OUT_TYPE = {PEAK_F16_F32: "f32", PEAK_BF16_BF16: "bf16", PEAK_F32_F32: "f32", PEAK_F16_F16: "f16",
-            PEAK_BF16_F32: "f32"}
-NP_STORE = {"f16": np.uint16, "bf16": np.uint16, "f32": np.float32}
-ELEM_BYTES = {"f16": 2, "bf16": 2, "f32": 4}
-NAN_BITS = {"f16": 0x7E00, "bf16": 0x7FC0}
+            PEAK_BF16_F32: "f32", PEAK_E4M3_BF16: "bf16", PEAK_E4M3_F32: "f32", PEAK_E5M2_BF16: "bf16",
+            PEAK_E5M2_F32: "f32"}
+NP_STORE = {"f16": np.uint16, "bf16": np.uint16, "f32": np.float32, "e4m3": np.uint8, "e5m2": np.uint8}
+ELEM_BYTES = {"f16": 2, "bf16": 2, "f32": 4, "e4m3": 1, "e5m2": 1}
+NAN_BITS = {"f16": 0x7E00, "bf16": 0x7FC0, "e4m3": 0x7F, "e5m2": 0x7E}
+_TORCH_FP8 = {"e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}
 
 
 @dataclass(frozen=True)
@@ -116,6 +120,9 @@ def encode(values_f32: np.ndarray, t: str) -> np.ndarray:
     if t == "bf16":
         tt = torch.from_numpy(np.ascontiguousarray(values_f32, dtype=np.float32)).to(torch.bfloat16)
         return tt.view(torch.int16).numpy().view(np.uint16)
+    if t in _TORCH_FP8:
+        tt = torch.from_numpy(np.ascontiguousarray(values_f32, dtype=np.float32)).to(_TORCH_FP8[t])
+        return tt.view(torch.uint8).numpy()
     raise ValueError(t)
 
 
@@ -127,6 +134,9 @@ def to_float64(stored: np.ndarray, t: str) -> np.ndarray:
         return stored.view(np.float16).astype(np.float64)
     if t == "bf16":
         return (stored.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    if t in _TORCH_FP8:
+        tt = torch.from_numpy(np.ascontiguousarray(stored)).view(_TORCH_FP8[t]).to(torch.float32)
+        return tt.numpy().astype(np.float64)
     raise ValueError(t)
 
 
@@ -243,6 +253,13 @@ def config4_ragged(which: int) -> GemmCase:
 def bench_workload() -> GemmCase:
     """The configuration the headline throughput is quoted on."""
     return config1()
+
+
+def fp8_workload(n: int, in_type: str = "e4m3") -> GemmCase:
+    """8-bit float inputs, bf16 output, n^3, K-major operands (A row-major, B stored N x K): uniform[-1, 1]
+    values so that the operands use the formats' range (normal / sqrt(K) would fall into the subnormals)."""
+    dt = PEAK_E4M3_BF16 if in_type == "e4m3" else PEAK_E5M2_BF16
+    return GemmCase(f"{in_type}_{n}_nt", dt, False, True, n, n, n, 1.0, 0.0, "uniform", config=5, case=n)
 
 
 def target_workload() -> GemmCase:

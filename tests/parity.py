@@ -8,6 +8,7 @@ The tolerances are written out here:
     exact in fp32, so only the <= K fp32 accumulation roundings and the single output rounding contribute:
         |C - ref| <= 2 * u_out * |ref| + 4 * K * 2^-24 * S' + tiny,
     u_out = 2^-8 (bf16), 2^-11 (fp16), 2^-24 (fp32);
+  * 8-bit inputs: products of two 8-bit floats are exact in fp32 as well, so the same two bounds apply;
   * exact cases (small integers): the output bits equal the oracle's correctly rounded result.
 """
 from __future__ import annotations
@@ -19,7 +20,7 @@ import oracle
 from paper_2512_19018_b200 import binding as P
 from paper_2512_19018_b200 import workloads as W
 
-OT = {"f16": oracle.F16, "bf16": oracle.BF16, "f32": oracle.F32}
+OT = {"f16": oracle.F16, "bf16": oracle.BF16, "f32": oracle.F32, "e4m3": oracle.E4M3, "e5m2": oracle.E5M2}
 U_OUT = {"bf16": 2.0 ** -8, "f16": 2.0 ** -11, "f32": 2.0 ** -24}
 TORCH_STORE = {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}
 GUARD_ROWS = 3
@@ -27,7 +28,7 @@ GUARD_ROWS = 3
 
 def to_device(arr: np.ndarray, t: str) -> torch.Tensor:
     """Upload stored bits unchanged."""
-    if t == "f32":
+    if t in ("f32", "e4m3", "e5m2"):     # float32 values / raw bytes
         return torch.from_numpy(arr).cuda()
     return torch.from_numpy(arr.view(np.int16)).cuda().view(TORCH_STORE[t])
 

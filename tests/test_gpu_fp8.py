@@ -1,0 +1,139 @@
+"""GPU parity for 8-bit floating-point inputs (E4M3 / E5M2 operands, bf16 or fp32 output) against the CPU
+oracle, whose decoders are written from the bit layout and pinned separately.  The tensor-core path takes
+K-major operands only (A as stored, B transposed); the other layouts run on the portable kernel."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2512_19018_b200 import binding as P
+from paper_2512_19018_b200 import workloads as W
+from tests import parity as R
+
+pytestmark = pytest.mark.gpu
+
+PAIRS_8 = [W.PEAK_E4M3_BF16, W.PEAK_E4M3_F32, W.PEAK_E5M2_BF16, W.PEAK_E5M2_F32]
+LAYOUTS = [(0, 0), (0, 1), (1, 0), (1, 1)]
+UMMA = [P.PEAK_VARIANT_UMMA_1CTA, P.PEAK_VARIANT_UMMA_2CTA]
+
+
+def mk(dtype, ta, tb, M, N, K, **kw):
+    return W.GemmCase(f"q{dtype}_{ta}{tb}_{M}x{N}x{K}", dtype, bool(ta), bool(tb), M, N, K, **kw)
+
+
+def pad16(n):
+    return (-n) % 16
+
+
+def k_major(dtype, M, N, K, **kw):
+    """A row-major M x K, B stored N x K (transB), pitches padded to 16 bytes as the TMA path needs."""
+    return mk(dtype, 0, 1, M, N, K, pad_a=pad16(K), pad_b=pad16(K), **kw)
+
+
+@pytest.fixture
+def reset_tuning():
+    yield
+    for key in range(12):
+        P.peak_set_tuning(key, 0)
+
+
+def assert_bits_equal(c, dc, what):
+    ref, _ = dc.oracle_full()
+    want = oracle.round_to(R.OT[c.out_type], ref)
+    got = dc.result()
+    if c.out_type == "f32":
+        got = got.view(np.uint32)
+    if not np.array_equal(got, want):
+        bad = np.argwhere(got != want)
+        raise AssertionError(f"{what}: {len(bad)} of {got.size} wrong, first at {bad[0]}")
+
+
+@pytest.mark.parametrize("dtype", PAIRS_8)
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_fallback_fp8_any_layout_any_pitch(dtype, ta, tb):
+    for (M, N, K, a, b) in [(1, 1, 1, 1.0, 0.0), (67, 130, 45, 0.5, 2.0), (128, 64, 200, -1.0, 1.0)]:
+        c = mk(dtype, ta, tb, M, N, K, alpha=a, beta=b, pad_a=1, pad_b=3, pad_c=5, case=M)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_FALLBACK)
+        R.check_full(dc)
+
+
+def test_every_fp8_bit_pattern_decodes_as_the_oracle_does():
+    """A = all 256 bit patterns minus the NaNs / infinities (one per row, K = 1), B = [1]: C = decode(A)."""
+    for dtype, t in [(W.PEAK_E4M3_F32, "e4m3"), (W.PEAK_E5M2_F32, "e5m2")]:
+        bits = np.arange(256, dtype=np.uint8)
+        vals = oracle.decode(R.OT[t], bits)
+        keep = np.isfinite(vals)
+        a = np.zeros((256, 16), dtype=np.uint8)
+        a[:, 0] = np.where(keep, bits, 0)
+        one = W.encode(np.ones((1, 1), np.float32), t)
+        b = np.zeros((16, 16), dtype=np.uint8)
+        b[0, 0] = one[0, 0]
+        import torch
+        A, B = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+        for variant in [P.PEAK_VARIANT_FALLBACK] + UMMA:
+            C = torch.full((256, 16), float("nan"), dtype=torch.float32, device="cuda")
+            # K = 16 with zero padding so that the TMA pitch rule holds; B is N x K (transB)
+            P.peak_gemm_variant(variant, dtype, 0, 1, 256, 16, 16, 1.0, A, 16, B, 16, 0.0, C, 16, None)
+            rc, _ = P.peak_check(None)
+            assert rc == P.PEAK_OK
+            got = C.cpu().numpy()[:, 0].astype(np.float64)
+            want = np.where(keep, vals, 0.0)
+            assert np.array_equal(got, want), f"{t} {P.peak_variant_string(variant)}"
+            assert (C.cpu().numpy()[:, 1:] == 0).all()
+
+
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("dtype", PAIRS_8)
+def test_umma_fp8_exact_small_integers(variant, dtype):
+    """Entries in [-4, 4] are exact in both 8-bit formats; every partial sum is an integer below 2^24, so the
+    result must equal the oracle's correctly rounded value bit for bit.  K spans one, several and a ragged
+    number of 128-element k-blocks."""
+    for (M, N, K) in [(128, 256, 128), (256, 512, 384), (384, 256, 512), (200, 328, 208), (130, 72, 48)]:
+        c = k_major(dtype, M, N, K, dist="smallint", case=K)
+        if c.out_type != "f32":
+            c = c.with_(alpha=0.125)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        assert_bits_equal(c, dc, f"{c.name} {P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("variant", UMMA + [P.PEAK_VARIANT_AUTO])
+@pytest.mark.parametrize("dtype", PAIRS_8)
+def test_umma_fp8_ragged_alpha_beta(variant, dtype):
+    for (M, N, K, a, b, dist) in [(300, 520, 1000, 1.0, 0.0, "uniform"), (129, 257, 4100, 0.5, 2.0, "uniform"),
+                                  (512, 768, 2048, -1.0, 1.0, "transformer"), (64, 1000, 336, 2.0, 0.0, "normal_rsqrtk")]:
+        c = k_major(dtype, M, N, K, alpha=a, beta=b, dist=dist, pad_c=pad16(N) + 8, case=K)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        R.check_full(dc, what=f"{c.name} {P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32])
+def test_fp8_tensor_core_variant_refuses_other_layouts(dtype):
+    c = mk(dtype, 1, 0, 256, 256, 256)
+    dc = R.DeviceCase(c)
+    with pytest.raises(P.PeakError):
+        dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+    dc.run(P.PEAK_VARIANT_AUTO)      # the dispatcher routes it to the portable kernel instead
+    R.check_full(dc)
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32])
+@pytest.mark.parametrize("tile_n,split", [(128, 0), (256, 3), (512, 0), (256, 0)])
+def test_umma_fp8_tiles_and_split_k(dtype, tile_n, split, reset_tuning):
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, tile_n)
+    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+    c = k_major(dtype, 512, 1024, 3000 + 8, dist="uniform", alpha=0.75, beta=0.5, case=tile_n + split)
+    for variant in UMMA:
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        R.check_full(dc, what=f"{c.name} bn{tile_n} split{split} {P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E4M3_F32])
+def test_fp8_full_size_sampled(dtype):
+    """8192^3 K-major in the launch configuration the benchmark times, on a sampled sub-grid."""
+    c = k_major(dtype, 8192, 8192, 8192, dist="uniform")
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    R.check_sampled(dc, tile_m=256, tile_n=256, budget_macs=6e8)

@@ -87,7 +87,14 @@ def test_dispatch_choices(lib):
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 0, 1.0, None, 1, None, 64, 0.5, al, 64) == P.PEAK_VARIANT_SCALE
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 1.0, al, 64) == P.PEAK_VARIANT_NONE
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 0.0, al, 64) == P.PEAK_VARIANT_SCALE
-    assert q(7, 0, 0, 64, 64, 64, 1.0, al, 64, al, 64, 0.0, al, 64) == -P.PEAK_ERR_INVALID_VALUE
+    assert q(9, 0, 0, 64, 64, 64, 1.0, al, 64, al, 64, 0.0, al, 64) == -P.PEAK_ERR_INVALID_VALUE
+    # 8-bit float inputs: tensor cores only for K-major operands (A as stored, B transposed), 16-byte pitches
+    for dt in (P.PEAK_E4M3_BF16, P.PEAK_E4M3_F32, P.PEAK_E5M2_BF16, P.PEAK_E5M2_F32):
+        assert q(dt, 0, 1, 1024, 1024, 1024, 1.0, al, 1024, al, 1024, 0.0, al, 1024) == P.PEAK_VARIANT_UMMA_2CTA
+        for ta, tb in [(0, 0), (1, 0), (1, 1)]:
+            assert q(dt, ta, tb, 1024, 1024, 1024, 1.0, al, 1024, al, 1024, 0.0, al, 1024) == P.PEAK_VARIANT_FALLBACK
+        assert q(dt, 0, 1, 1024, 1024, 1000, 1.0, al, 1000, al, 1000, 0.0, al, 1024) == P.PEAK_VARIANT_FALLBACK
+        assert q(dt, 0, 1, 1024, 1024, 1000, 1.0, al, 1008, al, 1008, 0.0, al, 1024) == P.PEAK_VARIANT_UMMA_2CTA
 
 
 @pytest.mark.parametrize("tiles_m,tiles_n,group", [(1, 1, 8), (64, 32, 16), (32, 32, 8), (20, 12, 16), (7, 5, 3),
