@@ -26,6 +26,7 @@
 // tile (full_tiles = 0); shapes whose tile count is not a multiple of the SM (pair) count split only the
 // tiles of the last, partly filled wave, so that the wave finishes in a fraction of a tile time.
 #pragma once
+#include <type_traits>
 #include <cuda.h>
 
 #include "common.cuh"
@@ -101,9 +102,17 @@ __device__ __forceinline__ void report_timeout(const UmmaParams &p, volatile uin
     *abort_flag = 1;
 }
 
+// Two fp32 values -> one 32-bit word of two 16-bit outputs (lo in the low half), round to nearest even.
+// The packed conversion is one instruction; converting the halves one by one and merging them made the
+// staging of a 32 x 32 chunk three times as long (about 540 instead of 190 cycles per warp).
 template <typename TOut> __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-    TOut a = from_f32<TOut>(lo), b = from_f32<TOut>(hi);
-    return (uint32_t)(*reinterpret_cast<uint16_t *>(&a)) | ((uint32_t)(*reinterpret_cast<uint16_t *>(&b)) << 16);
+    static_assert(sizeof(TOut) == 2, "pack2 packs 16-bit outputs");
+    uint32_t d;
+    if constexpr (std::is_same<TOut, __nv_bfloat16>::value)
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    else
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
 }
 
 // 32 consecutive outputs of one row -> global memory (vector path when aligned and whole)
