@@ -40,15 +40,22 @@ constexpr int BK = 64;    // k-block: 64 16-bit elements = one 128-byte swizzle 
 constexpr int UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KiB
 constexpr int ATOM_BYTES = 64 * BK * 2;     // one 64-wide MN-major box: 64 k-rows of 128 bytes = 8 KiB
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_BUF_BYTES = 32 * 128;               // one staging buffer: 32 rows x 128 bytes
-constexpr int EPI_BYTES = 4 * 2 * EPI_BUF_BYTES;      // 4 epilogue warps x 2 buffers = 32 KiB
+// Warp 0 loads, warp 1 issues the MMAs, the others run the epilogue.  A warp may only read the 32 TMEM lanes
+// of quadrant (warp % 4), so epilogue warps come in groups of four that cover all 128 rows.  A one-slot tile
+// has one group (its epilogue hides behind the next tile's main loop); a two-half tile, whose epilogue is
+// exposed because the tile fills the whole tensor memory, has two groups that drain one half each at the
+// same time.
+constexpr int MAX_EPI_WARPS = 8;
+constexpr int EPI_BUF_BYTES = 32 * 128;                    // one staging buffer: 32 rows x 128 bytes
+constexpr int EPI_BYTES = MAX_EPI_WARPS * EPI_BUF_BYTES;   // 32 KiB: one buffer per epilogue warp
 constexpr int SMEM_LIMIT = 232448;                    // 227 KiB of dynamic shared memory per CTA
 
 template <int CG, int BN> struct Cfg {
     // A tile wider than one MMA (BN = 512) is computed as two 256-column halves, one per accumulator slot.
     static constexpr int SLOT_N = BN > 256 ? 256 : BN;     // MMA N = width of one accumulator slot
     static constexpr int HALVES = BN / SLOT_N;
+    static constexpr int EPI_GROUPS = HALVES;              // groups of four epilogue warps
+    static constexpr int THREADS = 64 + 128 * EPI_GROUPS;
     static constexpr int HROWS = SLOT_N / CG;              // rows of op(B)^T this CTA stages per half
     static constexpr int B_ROWS = HALVES * HROWS;
     static constexpr int B_BOX_ROWS = HROWS < 128 ? HROWS : 128;
@@ -215,7 +222,7 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
 // column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
 // (z0 is used when MAP3D says that `tm` is three-dimensional).
 template <typename T, int BN, bool MAP3D = false>
-__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage, uint32_t &chunk_no, int lane,
+__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t buf, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
                                               bool vec, float alpha, float beta, const float *bias = nullptr,
@@ -225,19 +232,14 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
         const int col0 = cbase + c * CHUNK_COLS;
         if (col0 >= ncols) break;  // warp-uniform
-        uint32_t buf = 0;
-        if (tma) {
-            // the store that last read this buffer (two chunks ago) must have drained it
-            buf = my_stage + (chunk_no & 1u) * EPI_BUF_BYTES;
-            if (lane == 0) ptx::tma_store_wait_read<1>();
-            __syncwarp();
-        }
+        // the whole chunk is requested from tensor memory before the first wait
+        uint32_t r[CHUNK_COLS / 32][32];
+#pragma unroll
+        for (int h = 0; h < CHUNK_COLS / 32; ++h) ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r[h]);
+        ptx::tmem_ld_wait();
 #pragma unroll
         for (int h = 0; h < CHUNK_COLS / 32; ++h) {
             const int col = col0 + h * 32;
-            uint32_t r[32];
-            ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r);
-            ptx::tmem_ld_wait();
             const int valid = (ncols - col >= 32) ? 32 : (ncols - col > 0 ? ncols - col : 0);
             T *dst = base + (int64_t)row * ld + col;
             float v[32];
@@ -249,10 +251,10 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
                     for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
                 }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = fmaf(beta, cold[i], alpha * __uint_as_float(r[i]));
+                for (int i = 0; i < 32; ++i) v[i] = fmaf(beta, cold[i], alpha * __uint_as_float(r[h][i]));
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[i]);
+                for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[h][i]);
             }
             if (bias != nullptr) {  // fused tail: every thread of the warp adds the same 32 bias values
                 if (valid == 32 && (reinterpret_cast<uintptr_t>(bias + col) & 15u) == 0) {
@@ -274,8 +276,15 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = activate_f32(v[i], PEAK_ACT_GELU);
             }
-            if (tma) stage_row32<T>(buf, lane, h, v);
-            else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
+            if (tma) {
+                if (h == 0) {
+                    // the store of the previous chunk must have read the staging buffer; it had the time of
+                    // this chunk's tensor-memory load and arithmetic to do so
+                    if (lane == 0) ptx::tma_store_wait_read<0>();
+                    __syncwarp();
+                }
+                stage_row32<T>(buf, lane, h, v);
+            } else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
         }
         if (tma) {
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA engine
@@ -285,7 +294,6 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t my_stage
                 else ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
                 ptx::tma_store_commit();
             }
-            ++chunk_no;
         }
     }
 }
@@ -317,7 +325,7 @@ template <> struct McOps<0> {
 // 128 elements instead of 64, every byte count and descriptor stays as it is, and the MMA is the f8f6f4 kind
 // with K = 32 per instruction.  Both operands must be K-major (A not transposed, B transposed).
 template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__((Cfg<CG, BN>::THREADS), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
                  float *__restrict__ ws, const UmmaParams p) {
@@ -358,7 +366,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(accfull0 + 8 * b, 1);
-            ptx::mbar_init(accempty0 + 8 * b, 4 * CG);  // one arrival per epilogue warp of every CTA
+            ptx::mbar_init(accempty0 + 8 * b, 4 * CG);  // one arrival per epilogue warp (of one group) per CTA
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -530,11 +538,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue (4 warps)
-        const int q = warp & 3;  // TMEM lane quadrant this warp may read
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
+        // ------------------------------------------------------------------ epilogue (4 or 8 warps)
+        const int q = warp & 3;          // TMEM lane quadrant this warp may read
+        const int grp = (warp - 2) >> 2; // group of four warps: drains half `grp` of a two-half tile
+        constexpr int W = C_::SLOT_N;    // columns a warp drains per tile
+        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;
         const bool vec = p.vec_ok != 0;
-        uint32_t tl = 0, chunk_no = 0;
+        uint32_t tl = 0;
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
             const Item w = decode_item(p, item);
@@ -543,8 +553,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
             const int n0 = (int)tn * BN;
-#pragma unroll 1
-            for (int hf = 0; hf < C_::HALVES && ok; ++hf) {
+            {
+                const int hf = (C_::HALVES == 2) ? grp : 0;
                 const uint32_t b = (C_::HALVES == 1) ? (tl & 1u) : (uint32_t)hf;
                 const uint32_t aph = (C_::HALVES == 1) ? ((tl >> 1) & 1u) : (tl & 1u);
                 // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
@@ -555,21 +565,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     break;
                 }
                 ptx::tc_fence_after_sync();
+                const int co = hf * C_::SLOT_N;  // first tile column of this warp
                 const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * C_::SLOT_N;
-                const int nh = n0 + hf * C_::SLOT_N;  // first column of this half
+                const int nh = n0 + co;
                 if (w.ws_block < 0) {
                     // whole tile: alpha/beta epilogue straight to C
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;
-                    epilogue_tile<TOut, C_::SLOT_N, BATCHED>(t_addr, my_stage, chunk_no, lane, c_base, p.ldc,
+                    epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc,
                                                     row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0, bz,
                                                     p.tma_store != 0, vec, p.alpha, p.beta, p.bias, p.act);
                 } else {
                     // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
-                    epilogue_tile<float, C_::SLOT_N>(t_addr, my_stage, chunk_no, lane, ws, (int64_t)BN, wrow0 + lane,
-                                                     wrow0, 0x7fffffff, 0, BN, &tmW, 0, wrow0, 0, true, true, 1.0f,
-                                                     0.0f);
+                    epilogue_tile<float, W>(t_addr, my_stage, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
+                                            0x7fffffff, co, BN, &tmW, co, wrow0, 0, true, true, 1.0f, 0.0f);
                 }
                 // hand the accumulator slot back to the MMA issuer
                 ptx::tc_fence_before_sync();

@@ -185,7 +185,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(units * CG));
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(C_::THREADS);
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = g.stream;
     cudaLaunchAttribute attr[2];
@@ -338,20 +338,16 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
     const int units = sm_count() / cta_group;
     Plan plan = choose_plan(g, cta_group, units);
-    // Measured on B200 under the power cap (sustained, random inputs): 256 x 512 pair tiles are 4-12 % faster
-    // than 256 x 256 ones when the main loop is long (K >= 8192) and there are at least two waves of them, and
-    // up to 13 % slower at K = 4096 where their half-overlapped epilogue shows.
-    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && !tuning(PEAK_TUNE_TILE_N) &&
-        g.K >= 8192 && tiles_of(g, 2, 512) >= 2 * units)
-        plan = Plan{512, (int)tiles_of(g, 2, 512), 1};
+    const bool in8 = is_fp8(in_elem(g.dtype));
+    const bool whole256 = cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1;
     // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
-    // Measured: +3 % at 4096^3, +12 % at 5000x3000x2500, but -2..-4 % on problems of 5e11 flop and more.
+    // Measured (sustained, random inputs): +2..3 % at 4096^3, +12 % at 5000x3000x2500, but -3..-6 % from
+    // 2.7e11 flop on (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
-    if (cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1 && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 &&
-        !is_fp8(in_elem(g.dtype)) && mc_entry()) {
+    if (whole256 && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
-        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 3e11)) {
+        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {
             peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
@@ -362,6 +358,23 @@ int launch_umma(const GemmArgs &g, int cta_group) {
             if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
             if (rc != PEAK_ERR_UNSUPPORTED) return rc;
         }
+    }
+    // 256 x 512 pair tiles move a third less operand data per flop, but the tile fills the tensor memory, so
+    // its epilogue (two groups of warps, one per half) is exposed once per tile.  Measured under the power
+    // cap (sustained, random inputs): with 16-bit inputs and beta = 0 they win from 64 k-blocks on (+2 % at
+    // 8192x8192x4096, +5 % at 8192^3, +9 % at fp16 8192^3 TN), with beta != 0 (the epilogue also reads C)
+    // only from 128 k-blocks on (-7 % at 16384x14336x4096, +3 % at 16384x4096x14336); 8-bit inputs, whose
+    // k-blocks take the same time but whose 256-wide tiles are less starved, from 128 k-blocks (K = 16384)
+    // on (+3 %).  They must fill the grid as well as the 256-wide tiles do (4096x8192x4096: 3.46 waves
+    // against 6.9, -3 %).
+    if (whole256 && !tuning(PEAK_TUNE_TILE_N)) {
+        const int bke = in8 ? 2 * BK : BK;
+        const int64_t num_kb = (g.K + bke - 1) / bke;
+        const bool light_tail = g.beta == 0.0f && g.act != PEAK_ACT_GELU;
+        const int64_t min_kb = (!in8 && light_tail) ? 64 : 128;
+        auto fill = [&](int64_t tiles) { return (double)tiles / (double)(((tiles + units - 1) / units) * units); };
+        const int64_t t512 = tiles_of(g, 2, 512), t256 = tiles_of(g, 2, 256);
+        if (num_kb >= min_kb && t512 >= units && fill(t512) >= fill(t256) - 0.02) plan = Plan{512, (int)t512, 1};
     }
     if (cta_group == 2) {
         if (plan.bn == 512) return run_umma<2, 512>(g, plan, units);

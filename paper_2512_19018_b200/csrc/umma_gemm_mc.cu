@@ -92,7 +92,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.inject_stall = r->inject_stall == 1 ? 1 : 0;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(C_::THREADS);
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = r->stream;
     cudaLaunchAttribute attr[2];
