@@ -88,6 +88,7 @@ int launch_sgemm(const GemmArgs &g);
 bool sgemm_supports(const GemmArgs &g);
 int launch_umma(const GemmArgs &g, int cta_group);
 bool umma_supports(const GemmArgs &g, int cta_group);
+int umma_units(int cta_group);  // CTAs (cta_group 1) or CTA pairs (2) a persistent launch can keep resident
 bool umma_multicast_available();
 
 // status word layout: bit 31 = a bounded wait gave up; bits 0..7 = role, 8..15 = barrier index

@@ -334,6 +334,8 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
 
 bool umma_multicast_available() { return mc_entry() != nullptr; }
 
+int umma_units(int cta_group) { return sm_count() / (cta_group == 2 ? 2 : 1); }
+
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
     const int units = sm_count() / cta_group;

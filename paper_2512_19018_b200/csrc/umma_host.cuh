@@ -29,8 +29,8 @@ inline EncodeTiledFn encode_fn() {
 // Tensor map over a stack of `batch` row-major 2-D arrays `batch_stride` elements apart: `inner` contiguous
 // elements per row, `outer` rows, `pitch` elements between rows; box = box_inner x box_outer x 1, 128-byte
 // swizzle, zero fill.  batch <= 1 gives a two-dimensional map of the one matrix.
-inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
-              int box_outer, int64_t batch = 1, int64_t batch_stride = 0) {
+inline bool encode_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch,
+                       int box_inner, int box_outer, int64_t batch, int64_t batch_stride) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
@@ -46,6 +46,53 @@ inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, i
     CUresult r = fn(tm, dt, rank, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+// Descriptor cache.  A tensor map is a pure function of the arguments above (it holds an address and a
+// shape, no reference to the memory), so a call that repeats a (pointer, shape, pitch, box) combination --
+// the same weights every step, a buffer reused across layers -- takes the 128-byte descriptor from a small
+// direct-mapped table instead of encoding it again.  The table is per host thread: no lock, no sharing.
+struct MapKey {
+    const void *base;
+    int64_t inner, outer, pitch, batch, batch_stride;
+    int elem, box_inner, box_outer;
+    bool operator==(const MapKey &o) const {
+        return base == o.base && inner == o.inner && outer == o.outer && pitch == o.pitch && batch == o.batch &&
+               batch_stride == o.batch_stride && elem == o.elem && box_inner == o.box_inner && box_outer == o.box_outer;
+    }
+};
+constexpr int kMapCacheSlots = 64;
+struct MapCache {
+    MapKey key[kMapCacheSlots];
+    CUtensorMap map[kMapCacheSlots];
+    bool used[kMapCacheSlots];
+    uint64_t hits, misses;
+};
+inline MapCache &map_cache() {
+    thread_local MapCache c{};
+    return c;
+}
+inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
+                     int box_outer, int64_t batch = 1, int64_t batch_stride = 0) {
+    const MapKey k{base, inner, outer, pitch, batch, batch_stride, (int)e, box_inner, box_outer};
+    uint64_t h = (uint64_t)reinterpret_cast<uintptr_t>(base) >> 4;
+    h ^= (uint64_t)inner * 0x9E3779B97F4A7C15ull;
+    h ^= ((uint64_t)outer + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
+    h ^= (uint64_t)(box_outer * 131 + box_inner) * 0x165667B19E3779F9ull;
+    h ^= h >> 29;
+    MapCache &c = map_cache();
+    const int slot = (int)(h % kMapCacheSlots);
+    if (c.used[slot] && c.key[slot] == k) {
+        *tm = c.map[slot];
+        ++c.hits;
+        return true;
+    }
+    if (!encode_map(tm, e, base, inner, outer, pitch, box_inner, box_outer, batch, batch_stride)) return false;
+    c.key[slot] = k;
+    c.map[slot] = *tm;
+    c.used[slot] = true;
+    ++c.misses;
+    return true;
 }
 
 inline int sm_count() {

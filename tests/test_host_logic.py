@@ -90,11 +90,16 @@ def test_dispatch_choices(lib):
     assert q(9, 0, 0, 64, 64, 64, 1.0, al, 64, al, 64, 0.0, al, 64) == -P.PEAK_ERR_INVALID_VALUE
     # 8-bit float inputs: tensor cores only for K-major operands (A as stored, B transposed), 16-byte pitches
     for dt in (P.PEAK_E4M3_BF16, P.PEAK_E4M3_F32, P.PEAK_E5M2_BF16, P.PEAK_E5M2_F32):
-        assert q(dt, 0, 1, 1024, 1024, 1024, 1.0, al, 1024, al, 1024, 0.0, al, 1024) == P.PEAK_VARIANT_UMMA_2CTA
+        assert q(dt, 0, 1, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_2CTA
         for ta, tb in [(0, 0), (1, 0), (1, 1)]:
-            assert q(dt, ta, tb, 1024, 1024, 1024, 1.0, al, 1024, al, 1024, 0.0, al, 1024) == P.PEAK_VARIANT_FALLBACK
-        assert q(dt, 0, 1, 1024, 1024, 1000, 1.0, al, 1000, al, 1000, 0.0, al, 1024) == P.PEAK_VARIANT_FALLBACK
-        assert q(dt, 0, 1, 1024, 1024, 1000, 1.0, al, 1008, al, 1008, 0.0, al, 1024) == P.PEAK_VARIANT_UMMA_2CTA
+            assert q(dt, ta, tb, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
+        assert q(dt, 0, 1, 4096, 4096, 1000, 1.0, al, 1000, al, 1000, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
+        assert q(dt, 0, 1, 4096, 4096, 1000, 1.0, al, 1008, al, 1008, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_2CTA
+    # few tiles: single-CTA tiles spread the problem over more SMs than 256-row pair tiles would
+    assert q(P.PEAK_BF16_BF16, 0, 0, 1024, 1024, 1024, 1.0, al, 1024, al, 1024, 0.0, al, 1024) == P.PEAK_VARIANT_UMMA_1CTA
+    assert q(P.PEAK_BF16_BF16, 0, 0, 1536, 1536, 1536, 1.0, al, 1536, al, 1536, 0.0, al, 1536) == P.PEAK_VARIANT_UMMA_1CTA
+    assert q(P.PEAK_BF16_BF16, 0, 0, 2048, 2048, 2048, 1.0, al, 2048, al, 2048, 0.0, al, 2048) == P.PEAK_VARIANT_UMMA_2CTA
+    assert q(P.PEAK_BF16_BF16, 0, 0, 128, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_1CTA
 
 
 @pytest.mark.parametrize("tiles_m,tiles_n,group", [(1, 1, 8), (64, 32, 16), (32, 32, 8), (20, 12, 16), (7, 5, 3),
