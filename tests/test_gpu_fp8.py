@@ -137,3 +137,29 @@ def test_fp8_full_size_sampled(dtype):
     dc = R.DeviceCase(c)
     dc.run(P.PEAK_VARIANT_AUTO)
     R.check_sampled(dc, tile_m=256, tile_n=256, budget_macs=6e8)
+
+
+def test_fp8_strided_batched_one_launch():
+    """8-bit inputs through the batched entry point: one persistent launch (3-D tensor maps, byte elements)."""
+    from tests.test_gpu_batched import Batch
+    for dtype in (W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32):
+        n0 = P.peak_kernel_launches()
+        c = k_major(dtype, 264, 328, 400, alpha=0.25, beta=-1.0, dist="smallint", pad_c=0)
+        b = Batch(c, batch=4, gap=16)
+        b.run()
+        assert P.peak_kernel_launches() - n0 == 1
+        b.check(exact=True, what=f"fp8 batch {dtype}")
+        b = Batch(k_major(dtype, 136, 200, 272, alpha=0.5, beta=2.0, dist="uniform"), batch=3, gap=32)
+        b.run()
+        b.check(what=f"fp8 batch real {dtype}")
+
+
+@pytest.mark.parametrize("act", [P.PEAK_ACT_NONE, P.PEAK_ACT_RELU, P.PEAK_ACT_GELU])
+def test_fp8_fused_bias_activation(act):
+    from tests.test_gpu_fused import run_fused, check_fused
+    rng = np.random.default_rng(11)
+    for variant in [P.PEAK_VARIANT_FALLBACK] + UMMA:
+        c = k_major(W.PEAK_E4M3_BF16, 300, 520, 400, alpha=0.5, beta=1.0, dist="uniform", case=act)
+        bias = (rng.standard_normal(c.N) * 2).astype(np.float32)
+        dc = run_fused(c, variant, bias, act)
+        check_fused(dc, bias, act, f"fp8 fused act={act} {P.peak_variant_string(variant)}")
