@@ -249,7 +249,8 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_RASTER_GROUP = 0, /* tile-rows per raster group of the persistent scheduler */
     PEAK_TUNE_TILE_N = 1,       /* tensor-core tile width: 128, 256, or (CTA pairs only) 512 */
     PEAK_TUNE_SPLIT_K = 2,      /* k-slices per tile (1 = never split; capped by the number of k-blocks) */
-    PEAK_TUNE_EPILOGUE = 3,     /* 1 = direct global stores, 2 = shared-memory staging + TMA stores */
+    PEAK_TUNE_EPILOGUE = 3,     /* 1 = direct global stores, 2 = shared-memory staging + TMA stores (with beta != 0
+                                   old C arrives by TMA too), 3 = TMA stores but per-thread loads of old C */
     PEAK_TUNE_SGEMM_FMA = 4,    /* SGEMM inner product: 1 = scalar fp32 FMA, 2 = two-wide fp32 FMA (default) */
     PEAK_TUNE_TAIL_SPLIT = 5,   /* 2 = split the tiles of the last, partly filled wave whenever possible (off by default) */
     PEAK_TUNE_DEPENDENT_LAUNCH = 6, /* 1 = launch the tensor-core kernel without programmatic dependent launch */

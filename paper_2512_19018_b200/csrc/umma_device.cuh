@@ -47,7 +47,7 @@ constexpr int ATOM_BYTES = 64 * BK * 2;     // one 64-wide MN-major box: 64 k-ro
 // same time.
 constexpr int MAX_EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 32 * 128;                    // one staging buffer: 32 rows x 128 bytes
-constexpr int EPI_BYTES = MAX_EPI_WARPS * EPI_BUF_BYTES;   // 32 KiB: one buffer per epilogue warp
+constexpr int EPI_BYTES = MAX_EPI_WARPS * EPI_BUF_BYTES;   // 32 KiB: two buffers per warp (one group) or one
 constexpr int SMEM_LIMIT = 232448;                    // 227 KiB of dynamic shared memory per CTA
 
 template <int CG, int BN> struct Cfg {
@@ -68,7 +68,9 @@ template <int CG, int BN> struct Cfg {
     static constexpr int TMEM_COLS = 2 * SLOT_N;           // two fp32 accumulator slots
     static_assert(HALVES == 1 || CG == 2, "512-wide tiles are for CTA pairs");
     static_assert(STAGES >= 3, "pipeline too shallow");
-    static_assert(8 * (2 * STAGES + 4) + 8 <= AUX_BYTES, "barrier area too small");
+    // full[S], empty[S], acc_full[2], acc_empty[2], two old-C barriers for each of four epilogue warps, TMEM
+    // slot, abort flag
+    static_assert(8 * (2 * STAGES + 4 + 8) + 8 <= AUX_BYTES, "barrier area too small");
 };
 
 struct UmmaParams {
@@ -89,6 +91,7 @@ struct UmmaParams {
     int64_t ldc;
     int vec_ok;            // C base and pitch allow 16-byte vector access
     int tma_store;         // epilogue stores through TMA
+    int c_prefetch;        // beta != 0: old C chunks arrive by TMA in the staging buffers (one-slot tiles only)
     const float *bias;     // fused epilogue: fp32 value per column of C, or nullptr
     int act;               // fused epilogue: a peak_activation_t
     long long wait_cycles; // budget of every mbarrier wait
@@ -197,6 +200,52 @@ __device__ __forceinline__ void stage_row32(uint32_t buf, int lane, int h, const
     }
 }
 
+// The reverse of stage_row32: 32 consecutive stored values of row `lane` out of a 128-byte-swizzled box that a
+// TMA load has filled.
+template <typename TOut>
+__device__ __forceinline__ void unstage_row32(uint32_t buf, int lane, int h, float (&c)[32]) {
+    constexpr int PIECES = 32 * (int)sizeof(TOut) / 16;
+    const uint32_t row = buf + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int j = 0; j < PIECES; ++j) {
+        const uint32_t piece = (uint32_t)((h * PIECES + j) ^ (lane & 7));
+        uint32_t w[4];
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
+                     : "r"(row + piece * 16u)
+                     : "memory");
+        if constexpr (sizeof(TOut) == 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) c[4 * j + i] = __uint_as_float(w[i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint16_t lo = (uint16_t)(w[i] & 0xffffu), hi = (uint16_t)(w[i] >> 16);
+                c[8 * j + 2 * i] = to_f32(*reinterpret_cast<TOut *>(&lo));
+                c[8 * j + 2 * i + 1] = to_f32(*reinterpret_cast<TOut *>(&hi));
+            }
+        }
+    }
+}
+
+// Old-C prefetch of one epilogue warp (beta != 0 with TMA stores): chunk c of a tile is loaded by TMA into
+// staging buffer c & 1, where the result later overwrites it in place and leaves by a TMA store.
+struct CFetch {
+    uint32_t bar0;    // two mbarriers of this warp, 8 bytes apart
+    uint32_t phases;  // bit b: parity the next wait on barrier b uses
+    bool on;
+};
+template <typename T, bool MAP3D>
+__device__ __forceinline__ void cfetch_issue(const CFetch &cf, uint32_t my_stage, int c, const CUtensorMap *tm, int x0,
+                                             int y0, int z0) {
+    constexpr int CHUNK_COLS = 128 / (int)sizeof(T);
+    const uint32_t bar = cf.bar0 + 8u * (uint32_t)(c & 1);
+    ptx::mbar_arrive_expect_tx(bar, (uint32_t)EPI_BUF_BYTES);
+    const uint32_t dst = my_stage + (uint32_t)(c & 1) * EPI_BUF_BYTES;
+    if (MAP3D) ptx::tma_load_3d(dst, tm, x0 + c * CHUNK_COLS, y0, z0, bar);
+    else ptx::tma_load_2d(dst, tm, x0 + c * CHUNK_COLS, y0, bar);
+}
+
 // Work item -> tile, k-block range and destination (ws_block < 0: the tile is whole and goes to C;
 // otherwise the index of the (tile, slice) block of the partial-tile workspace).
 struct Item {
@@ -222,21 +271,37 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
 // column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
 // (z0 is used when MAP3D says that `tm` is three-dimensional).
 template <typename T, int BN, bool MAP3D = false>
-__device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t buf, int lane,
+__device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
-                                              bool vec, float alpha, float beta, const float *bias = nullptr,
-                                              int act = 0) {
+                                              bool vec, float alpha, float beta, const float *bias, int act,
+                                              CFetch &cf, volatile uint32_t *abort_flag, long long wait_cycles) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
         const int col0 = cbase + c * CHUNK_COLS;
         if (col0 >= ncols) break;  // warp-uniform
+        const uint32_t buf = my_stage + (cf.on ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
         // the whole chunk is requested from tensor memory before the first wait
         uint32_t r[CHUNK_COLS / 32][32];
 #pragma unroll
         for (int h = 0; h < CHUNK_COLS / 32; ++h) ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r[h]);
         ptx::tmem_ld_wait();
+        if (cf.on) {
+            // chunks 0 and 1 were requested before the accumulator was waited for; chunk c + 1 (c >= 1) goes
+            // into the buffer chunk c - 1 left by a store, which has had this chunk's tensor-memory load to
+            // finish reading it
+            if (c >= 1 && c + 1 < BN / CHUNK_COLS && cbase + (c + 1) * CHUNK_COLS < ncols) {
+                if (lane == 0) {
+                    ptx::tma_store_wait_read<0>();
+                    cfetch_issue<T, MAP3D>(cf, my_stage, c + 1, tm, x0, y0, z0);
+                }
+            }
+            const uint32_t b = (uint32_t)(c & 1);
+            const bool got = ptx::mbar_wait<false>(cf.bar0 + 8u * b, (cf.phases >> b) & 1u, abort_flag, wait_cycles);
+            cf.phases ^= 1u << b;
+            if (!__all_sync(0xffffffffu, got)) return false;
+        }
 #pragma unroll
         for (int h = 0; h < CHUNK_COLS / 32; ++h) {
             const int col = col0 + h * 32;
@@ -245,7 +310,8 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t buf, int
             float v[32];
             if (beta != 0.0f) {
                 float cold[32];
-                if (row < nrows && valid > 0) load_row32<T>(dst, cold, valid, vec);
+                if (cf.on) unstage_row32<T>(buf, lane, h, cold);  // out-of-range elements were zero-filled
+                else if (row < nrows && valid > 0) load_row32<T>(dst, cold, valid, vec);
                 else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) cold[i] = 0.0f;
@@ -277,13 +343,13 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t buf, int
                 for (int i = 0; i < 32; ++i) v[i] = activate_f32(v[i], PEAK_ACT_GELU);
             }
             if (tma) {
-                if (h == 0) {
+                if (h == 0 && !cf.on) {
                     // the store of the previous chunk must have read the staging buffer; it had the time of
                     // this chunk's tensor-memory load and arithmetic to do so
                     if (lane == 0) ptx::tma_store_wait_read<0>();
                     __syncwarp();
                 }
-                stage_row32<T>(buf, lane, h, v);
+                stage_row32<T>(buf, lane, h, v);  // with prefetched C: in place, over this thread's own row
             } else if (row < nrows && valid > 0) store_row32<T>(dst, v, valid, vec);
         }
         if (tma) {
@@ -296,6 +362,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t t_addr, uint32_t buf, int
             }
         }
     }
+    return true;
 }
 
 // Tile copies: a single GEMM uses two-dimensional descriptors, a strided batch three-dimensional ones.  The
@@ -338,13 +405,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t epi_base = stage_base + STAGES * C_::STAGE_BYTES;
     uint8_t *aux = smem_raw + (epi_base - raw) + EPI_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * (2 * STAGES + 4));
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aux + 8 * (2 * STAGES + 4 + 8));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const uint32_t full0 = ptx::smem_u32(bars);
     const uint32_t empty0 = full0 + 8 * STAGES;
     const uint32_t accfull0 = empty0 + 8 * STAGES;
     const uint32_t accempty0 = accfull0 + 16;
+    const uint32_t cbar0 = accempty0 + 16;  // old-C barriers: two per epilogue warp of a one-group kernel
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -368,6 +436,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::mbar_init(accfull0 + 8 * b, 1);
             ptx::mbar_init(accempty0 + 8 * b, 4 * CG);  // one arrival per epilogue warp (of one group) per CTA
         }
+        for (int b = 0; b < 8; ++b) ptx::mbar_init(cbar0 + 8 * b, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
@@ -542,8 +611,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;          // TMEM lane quadrant this warp may read
         const int grp = (warp - 2) >> 2; // group of four warps: drains half `grp` of a two-half tile
         constexpr int W = C_::SLOT_N;    // columns a warp drains per tile
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * EPI_BUF_BYTES;
+        // staging: two buffers per warp in a one-group kernel (old C of chunk c + 1 arrives while chunk c is
+        // worked on), one per warp with two groups
+        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (C_::HALVES == 1 ? 2u : 1u) * EPI_BUF_BYTES;
         const bool vec = p.vec_ok != 0;
+        CFetch cf{cbar0 + 16u * (uint32_t)(warp - 2), 0u, C_::HALVES == 1 && p.c_prefetch != 0};
+        CFetch no_cf{0u, 0u, false};
         uint32_t tl = 0;
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
@@ -557,6 +630,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int hf = (C_::HALVES == 2) ? grp : 0;
                 const uint32_t b = (C_::HALVES == 1) ? (tl & 1u) : (uint32_t)hf;
                 const uint32_t aph = (C_::HALVES == 1) ? ((tl >> 1) & 1u) : (tl & 1u);
+                if (cf.on && w.ws_block < 0) {
+                    // old C of the first two chunks is requested while the main loop still runs
+                    constexpr int CC = 128 / (int)sizeof(TOut);
+                    if (lane == 0) {
+                        ptx::tma_store_wait_read<0>();  // the previous tile's stores have read both buffers
+                        cfetch_issue<TOut, BATCHED>(cf, my_stage, 0, &tmC, n0, row0, bz);
+                        if (n0 + CC < p.N && CC < C_::SLOT_N) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, n0, row0, bz);
+                    }
+                    __syncwarp();
+                }
                 // the outcome is made warp-uniform: tcgen05.ld below needs the whole warp
                 const bool got = ptx::mbar_wait<CG == 2>(accfull0 + 8 * b, aph, abort_flag, p.wait_cycles);
                 if (!__all_sync(0xffffffffu, got)) {
@@ -572,14 +655,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // whole tile: alpha/beta epilogue straight to C
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;
-                    epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc,
-                                                    row0 + lane, row0, p.M, nh, p.N, &tmC, nh, row0, bz,
-                                                    p.tma_store != 0, vec, p.alpha, p.beta, p.bias, p.act);
+                    if (!epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc, row0 + lane, row0, p.M,
+                                                         nh, p.N, &tmC, nh, row0, bz, p.tma_store != 0, vec, p.alpha,
+                                                         p.beta, p.bias, p.act, cf, abort_flag, p.wait_cycles)) {
+                        if (lane == 0) report_timeout(p, abort_flag, 6, b);
+                        ok = false;
+                        break;
+                    }
                 } else {
                     // k-slice: raw fp32 partial tile to its dense (BM*CG) x BN block of the workspace
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
                     epilogue_tile<float, W>(t_addr, my_stage, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
-                                            0x7fffffff, co, BN, &tmW, co, wrow0, 0, true, true, 1.0f, 0.0f);
+                                            0x7fffffff, co, BN, &tmW, co, wrow0, 0, true, true, 1.0f, 0.0f, nullptr, 0,
+                                            no_cf, abort_flag, p.wait_cycles);
                 }
                 // hand the accumulator slot back to the MMA issuer
                 ptx::tc_fence_before_sync();

@@ -160,6 +160,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     tmC = tmA;  // placeholders when unused
     tmW = tmA;
     if (nb > 1 && (g.strideC * ob) % 16 != 0) p.tma_store = 0;  // the batch stride must suit the store map too
+    // beta != 0 with TMA stores on one-slot tiles: old C comes in by TMA as well (PEAK_TUNE_EPILOGUE 3 keeps the
+    // per-thread loads)
+    p.c_prefetch = (p.tma_store && g.beta != 0.0f && epi != 3) ? 1 : 0;
     if (p.tma_store && plan.full_tiles > 0 && !make_map(&tmC, eout, g.C, g.N, g.M, g.ldc, 128 / ob, 32, nb, g.strideC))
         return PEAK_ERR_CUDA;
     if (plan.full_tiles < tiles) {

@@ -86,6 +86,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.vec_ok = ((reinterpret_cast<uintptr_t>(r->C) % 16) == 0 && (r->ldc * ob) % 16 == 0) ? 1 : 0;
     p.tma_store = (p.vec_ok && (r->N * ob) % 16 == 0 && r->epilogue != 1) ? 1 : 0;
     tmC = tmA;
+    p.c_prefetch = (p.tma_store && r->beta != 0.0f && r->epilogue != 3) ? 1 : 0;
     if (p.tma_store && !make_map(&tmC, eout, r->C, r->N, r->M, r->ldc, 128 / ob, 32)) return PEAK_ERR_CUDA;
     p.status = r->status;
     p.wait_cycles = r->wait_ms > 0 ? (long long)r->wait_ms * 2000000LL : ptx::kWaitBudgetCycles;

@@ -241,7 +241,7 @@ def reset_tuning():
 
 @pytest.mark.parametrize("variant", UMMA)
 @pytest.mark.parametrize("tile_n", [128, 256])
-@pytest.mark.parametrize("epilogue", [1, 2])
+@pytest.mark.parametrize("epilogue", [1, 2, 3])
 def test_umma_tile_width_epilogue_and_split_k(variant, tile_n, epilogue, reset_tuning):
     """Tile width, epilogue store path and k-split are performance knobs: with integer inputs every
     combination must give the oracle's correctly rounded result bit for bit (which also shows that a split
