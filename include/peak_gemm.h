@@ -163,7 +163,9 @@ int peak_gemm_strided_batched(int dtype, int transA, int transB, int64_t M, int6
  * peak_gemm_host: the same operation on HOST buffers (the paper's "driver", section 3.1: allocate,
  * copy in, run, copy out).  A, B, C are host pointers (pinned memory makes the copies faster but is
  * not required).  Copies A and B (and C when beta != 0) to device staging buffers, runs peak_gemm,
- * copies C back, and synchronises `stream` before returning.  The staging buffers are owned by the
+ * copies C back, and synchronises `stream` before returning.  From 1024 rows on the work is cut into up to
+ * eight row panels of op(A) and C: panel i + 1 is copied in and panel i - 1 copied out (two internal
+ * streams, ordered against `stream` by events) while panel i is multiplied on `stream`.  The staging buffers are owned by the
  * library, grow on demand and are reused by later calls; peak_release_staging() frees them.
  * Not thread-safe with respect to other peak_gemm_host calls.
  */

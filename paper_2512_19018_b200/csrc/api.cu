@@ -1,6 +1,7 @@
 // The C ABI: argument validation, quick returns, variant selection, the host-buffer entry point and the
 // small amount of process state (launch counter, last CUDA error, per-device status word, staging buffers).
 #include <atomic>
+#include <algorithm>
 #include <mutex>
 
 #include "common.cuh"
@@ -137,6 +138,16 @@ struct Staging {
     size_t bytes = 0;
 };
 Staging g_stage[3];
+
+// Streams and events of the host-buffer entry point's copy / compute pipeline (created on first use, for the
+// device that is current then; guarded by g_stage_mutex like the staging buffers).
+constexpr int kHostPanels = 8;
+struct HostPipeline {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, out_done = nullptr, in_done[kHostPanels] = {}, mm_done[kHostPanels] = {};
+    int device = -1;
+};
+HostPipeline g_pipe;
 std::mutex g_stage_mutex;
 
 int ensure(Staging &s, size_t need) {
@@ -145,6 +156,37 @@ int ensure(Staging &s, size_t need) {
     cudaError_t e = cudaMalloc(&s.ptr, need);
     if (e != cudaSuccess) { set_cuda_error(e); s.ptr = nullptr; return PEAK_ERR_NO_MEMORY; }
     s.bytes = need;
+    return PEAK_OK;
+}
+
+void release_pipeline() {
+    if (g_pipe.in) cudaStreamDestroy(g_pipe.in);
+    if (g_pipe.out) cudaStreamDestroy(g_pipe.out);
+    if (g_pipe.start) cudaEventDestroy(g_pipe.start);
+    if (g_pipe.out_done) cudaEventDestroy(g_pipe.out_done);
+    for (int i = 0; i < kHostPanels; ++i) {
+        if (g_pipe.in_done[i]) cudaEventDestroy(g_pipe.in_done[i]);
+        if (g_pipe.mm_done[i]) cudaEventDestroy(g_pipe.mm_done[i]);
+    }
+    g_pipe = HostPipeline{};
+}
+
+int ensure_pipeline() {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (g_pipe.in && g_pipe.device == dev) return PEAK_OK;
+    release_pipeline();
+    e = cudaStreamCreateWithFlags(&g_pipe.in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&g_pipe.out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_pipe.start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_pipe.out_done, cudaEventDisableTiming);
+    for (int i = 0; i < kHostPanels && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&g_pipe.in_done[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_pipe.mm_done[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) { set_cuda_error(e); release_pipeline(); return PEAK_ERR_CUDA; }
+    g_pipe.device = dev;
     return PEAK_OK;
 }
 
@@ -235,20 +277,76 @@ int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int6
     std::lock_guard<std::mutex> lock(g_stage_mutex);
     if ((rc = ensure(g_stage[0], a_bytes)) || (rc = ensure(g_stage[1], b_bytes)) || (rc = ensure(g_stage[2], c_bytes)))
         return rc;
-    cudaError_t e = cudaSuccess;
-    if (a_bytes) e = cudaMemcpyAsync(g_stage[0].ptr, A, a_bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess && b_bytes) e = cudaMemcpyAsync(g_stage[1].ptr, B, b_bytes, cudaMemcpyHostToDevice, st);
     // C travels to the device when its old values are needed, or when the pitch leaves gaps that the
     // copy back would otherwise overwrite with stale staging contents
-    if (e == cudaSuccess && (beta != 0.0f || ldc != N))
-        e = cudaMemcpyAsync(g_stage[2].ptr, C, c_bytes, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
-    rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, g_stage[0].ptr, lda, g_stage[1].ptr, ldb,
-                   beta, g_stage[2].ptr, ldc, stream);
+    const bool c_in = beta != 0.0f || ldc != N;
+    char *dA = static_cast<char *>(g_stage[0].ptr), *dB = static_cast<char *>(g_stage[1].ptr),
+         *dC = static_cast<char *>(g_stage[2].ptr);
+    const char *hA = static_cast<const char *>(A);
+    char *hC = static_cast<char *>(C);
+    cudaError_t e = cudaSuccess;
+    auto fail = [&](cudaError_t err) { set_cuda_error(err); return (int)PEAK_ERR_CUDA; };
+
+    // Row panels of op(A) and C: the copy engines bring panel i + 1 in and take panel i - 1 out while the SMs
+    // multiply panel i.  Copies in run on one internal stream (B first, then the panels in order), the
+    // products on the caller's stream, copies out on a second internal stream; events order them.
+    const int64_t panels = need_ab ? std::max<int64_t>(1, std::min<int64_t>(kHostPanels, M / 512)) : 1;
+    if (panels > 1 && (rc = ensure_pipeline()) != PEAK_OK) return rc;
+    if (panels == 1) {
+        if (a_bytes) e = cudaMemcpyAsync(dA, A, a_bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && b_bytes) e = cudaMemcpyAsync(dB, B, b_bytes, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && c_in) e = cudaMemcpyAsync(dC, C, c_bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail(e);
+        rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, dA, lda, dB, ldb, beta, dC, ldc, stream);
+        if (rc != PEAK_OK) return rc;
+        e = cudaMemcpyAsync(C, dC, c_bytes, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return fail(e);
+        return PEAK_OK;
+    }
+    cudaStream_t s_in = g_pipe.in, s_out = g_pipe.out;
+    // the internal streams start after whatever the caller's stream already holds
+    if ((e = cudaEventRecord(g_pipe.start, st)) != cudaSuccess) return fail(e);
+    if ((e = cudaStreamWaitEvent(s_in, g_pipe.start, 0)) != cudaSuccess) return fail(e);
+    if ((e = cudaStreamWaitEvent(s_out, g_pipe.start, 0)) != cudaSuccess) return fail(e);
+    if ((e = cudaMemcpyAsync(dB, B, b_bytes, cudaMemcpyHostToDevice, s_in)) != cudaSuccess) return fail(e);
+    const int64_t rows_per = ((M + panels - 1) / panels + 127) / 128 * 128;  // whole 128-row tiles per panel
+    for (int64_t i = 0; i < panels; ++i) {
+        const int64_t m0 = i * rows_per, mp = std::min(rows_per, M - m0);
+        if (mp <= 0) break;
+        const size_t c_off = (size_t)m0 * (size_t)ldc * (size_t)ob;
+        const size_t c_len = span_bytes(mp, N, ldc, ob);
+        if (!transA) {  // rows m0 .. m0 + mp of a row-major M x K matrix: one contiguous span
+            const size_t off = (size_t)m0 * (size_t)lda * (size_t)ib;
+            e = cudaMemcpyAsync(dA + off, hA + off, span_bytes(mp, K, lda, ib), cudaMemcpyHostToDevice, s_in);
+        } else {        // columns m0 .. m0 + mp of the stored K x M matrix: a strided copy
+            const size_t off = (size_t)m0 * (size_t)ib;
+            e = cudaMemcpy2DAsync(dA + off, (size_t)lda * ib, hA + off, (size_t)lda * ib, (size_t)mp * ib, (size_t)K,
+                                  cudaMemcpyHostToDevice, s_in);
+        }
+        if (e == cudaSuccess && c_in) e = cudaMemcpyAsync(dC + c_off, hC + c_off, c_len, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(g_pipe.in_done[i], s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, g_pipe.in_done[i], 0);
+        if (e != cudaSuccess) return fail(e);
+        const char *a_panel = transA ? dA + (size_t)m0 * ib : dA + (size_t)m0 * (size_t)lda * ib;
+        rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, mp, N, K, alpha, a_panel, lda, dB, ldb, beta, dC + c_off,
+                       ldc, stream);
+        if (rc != PEAK_OK) break;
+        if ((e = cudaEventRecord(g_pipe.mm_done[i], st)) != cudaSuccess) return fail(e);
+        if ((e = cudaStreamWaitEvent(s_out, g_pipe.mm_done[i], 0)) != cudaSuccess) return fail(e);
+        if ((e = cudaMemcpyAsync(hC + c_off, dC + c_off, c_len, cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
+            return fail(e);
+    }
+    // everything rejoins the caller's stream, which is then drained (also when a panel's product was refused, so
+    // that no copy is still in flight when the caller gets its buffers back)
+    cudaError_t e1 = cudaEventRecord(g_pipe.out_done, s_out);
+    if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(st, g_pipe.out_done, 0);
+    cudaError_t e2 = cudaStreamSynchronize(s_in);
+    cudaError_t e3 = cudaStreamSynchronize(st);
     if (rc != PEAK_OK) return rc;
-    e = cudaMemcpyAsync(C, g_stage[2].ptr, c_bytes, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (e1 != cudaSuccess) return fail(e1);
+    if (e2 != cudaSuccess) return fail(e2);
+    if (e3 != cudaSuccess) return fail(e3);
     return PEAK_OK;
 }
 
@@ -259,6 +357,7 @@ int peak_release_staging(void) {
         s.ptr = nullptr;
         s.bytes = 0;
     }
+    release_pipeline();
     return PEAK_OK;
 }
 

@@ -224,6 +224,27 @@ def test_host_buffer_entry_point():
     P.peak_release_staging()
 
 
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_host_buffer_entry_point_pipelined_panels(ta, tb):
+    """From 1024 rows on the host entry point works in row panels (copy in / multiply / copy out overlap):
+    ragged panel sizes, both storage orders of A, old C needed or not, pitch padding kept."""
+    for (M, N, K, beta, pad_c) in [(1500, 328, 264, 2.0, 8), (4100, 136, 200, 0.0, 0), (1030, 520, 72, 0.0, 8)]:
+        c = mk(W.PEAK_BF16_BF16, ta, tb, M, N, K, alpha=0.5, beta=beta, pad_a=(-(M if ta else K)) % 8,
+               pad_b=(-(K if tb else N)) % 8, pad_c=pad_c, case=M)
+        A, B, C0 = W.make_inputs(c, need_c0=True)
+        C = C0.copy()
+        n0 = P.peak_kernel_launches()
+        P.peak_gemm_host(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, A, c.lda, B, c.ldb, c.beta, C, c.ldc)
+        assert P.peak_kernel_launches() - n0 >= 2                 # more than one panel
+        ref, S = oracle.gemm(oracle.BF16, oracle.BF16, ta, tb, c.M, c.N, c.K, c.alpha, A, c.lda, B, c.ldb, c.beta,
+                             C0 if beta != 0 else None, c.ldc)
+        c0 = W.to_float64(C0[:, :c.N], "bf16") if beta != 0 else 0.0
+        R.check_values(c, C[:, :c.N], ref, S, c0, what=f"host panels {M}x{N}x{K} {ta}{tb}")
+        if pad_c:
+            assert np.array_equal(C[:, c.N:], C0[:, c.N:])
+    P.peak_release_staging()
+
+
 def test_launch_counter_moves():
     n0 = P.peak_kernel_launches()
     dc = R.DeviceCase(W.config0())
