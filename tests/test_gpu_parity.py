@@ -456,3 +456,68 @@ def test_cuda_graph_capture_and_replay():
     graph.replay()
     torch.cuda.synchronize()
     R.check_full(dc)
+
+
+@pytest.mark.parametrize("variant", [P.PEAK_VARIANT_FALLBACK] + UMMA)
+@pytest.mark.parametrize("dtype,tiny,big", [(W.PEAK_F16_F32, 2.0 ** -24, 2.0 ** 12), (W.PEAK_BF16_F32, 2.0 ** -133, 2.0 ** 120)])
+def test_subnormal_inputs_are_honoured(variant, dtype, tiny, big):
+    """A holds subnormal values of the input format (small integer multiples of its smallest subnormal), B
+    large powers of two: every product and every partial sum is exactly representable in fp32, so the
+    result must equal the oracle bit for bit.  A path that flushed subnormal inputs to zero would return 0."""
+    M, N, K = 128, 128, 64
+    rng = np.random.default_rng(5)
+    a = rng.integers(-7, 8, size=(M, K)).astype(np.float64) * tiny
+    b = rng.integers(-2, 3, size=(K, N)).astype(np.float64) * big
+    t = W.IN_TYPE[dtype]
+    A_h = oracle.round_to(R.OT[t], a)
+    B_h = oracle.round_to(R.OT[t], b)
+    assert np.array_equal(oracle.decode(R.OT[t], A_h), a) and np.array_equal(oracle.decode(R.OT[t], B_h), b)
+    A, B = R.to_device(A_h, t), R.to_device(B_h, t)
+    C = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    P.peak_gemm_variant(variant, dtype, 0, 0, M, N, K, 1.0, A, K, B, N, 0.0, C, N)
+    rc, _ = P.peak_check()
+    assert rc == P.PEAK_OK
+    ref, _ = oracle.gemm(R.OT[t], oracle.F32, 0, 0, M, N, K, 1.0, A_h, K, B_h, N, 0.0, None, N)
+    want = oracle.round_to(oracle.F32, ref)
+    assert np.abs(ref).max() > 0
+    got = C.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {got.size} differ"
+
+
+@pytest.mark.parametrize("variant", [P.PEAK_VARIANT_FALLBACK] + UMMA)
+@pytest.mark.parametrize("dtype", [W.PEAK_F16_F16, W.PEAK_BF16_BF16, W.PEAK_F16_F32])
+def test_inf_nan_propagate_and_outputs_overflow_to_inf(variant, dtype):
+    """IEEE propagation through the sum (an infinity in A makes its row of C infinite, NaN where it meets a
+    zero of B; a NaN poisons its row) and no saturation when the rounded output overflows."""
+    M, N, K = 128, 256, 64
+    c = mk(dtype, 0, 0, M, N, K, dist="smallint", case=77)
+    A_h, B_h, _ = W.make_inputs(c)
+    t = c.in_type
+    inf_bits = {"f16": 0x7C00, "bf16": 0x7F80}[t]
+    A_h[3, 5] = inf_bits                       # +inf in row 3
+    A_h[9, 0] = W.NAN_BITS[t]                  # NaN in row 9
+    A, B = R.to_device(A_h, t), R.to_device(B_h, t)
+    Cd = R.to_device(W.poison_c(c), c.out_type)
+    P.peak_gemm_variant(variant, dtype, 0, 0, M, N, K, 1.0, A, c.lda, B, c.ldb, 0.0, Cd, c.ldc)
+    assert P.peak_check()[0] == P.PEAK_OK
+    got = W.to_float64(R.to_host(Cd, c.out_type), c.out_type)[:, :N]
+    ref, _ = oracle.gemm(R.OT[t], R.OT[c.out_type], 0, 0, M, N, K, 1.0, A_h, c.lda, B_h, c.ldb, 0.0, None, c.ldc)
+    assert np.isnan(ref[9]).all() and np.isinf(ref[3]).any() and np.isnan(ref[3]).any()
+    assert np.array_equal(np.isnan(got), np.isnan(ref))
+    assert np.array_equal(np.isposinf(got), np.isposinf(ref)) and np.array_equal(np.isneginf(got), np.isneginf(ref))
+    fin = np.isfinite(ref)
+    assert np.array_equal(got[fin], ref[fin])                      # small integers elsewhere: exact
+    if c.out_type != "f32":
+        # alpha pushes finite sums beyond the largest finite 16-bit value: +-inf, not the largest finite number
+        big = 3.0e38 if c.out_type == "bf16" else 6.0e4
+        Cd = R.to_device(W.poison_c(c), c.out_type)
+        A2_h, B2_h, _ = W.make_inputs(c)
+        P.peak_gemm_variant(variant, dtype, 0, 0, M, N, K, big, R.to_device(A2_h, t), c.lda, R.to_device(B2_h, t), c.ldb,
+                            0.0, Cd, c.ldc)
+        assert P.peak_check()[0] == P.PEAK_OK
+        got = W.to_float64(R.to_host(Cd, c.out_type), c.out_type)[:, :N]
+        ref, _ = oracle.gemm(R.OT[t], R.OT[c.out_type], 0, 0, M, N, K, float(np.float32(big)), A2_h, c.lda, B2_h, c.ldb,
+                             0.0, None, c.ldc)
+        want = W.to_float64(oracle.round_to(R.OT[c.out_type], ref), c.out_type)
+        assert np.isinf(want).any() and np.array_equal(np.isinf(got), np.isinf(want))
+        assert np.array_equal(np.sign(got[np.isinf(got)]), np.sign(want[np.isinf(want)]))
