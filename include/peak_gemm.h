@@ -264,7 +264,10 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_MULTICAST = 10,   /* cluster-multicast plug-in: 1 = never use it, 2 = use it whenever it can run */
     PEAK_TUNE_BALANCED_GRID = 11, /* 1 = always launch one CTA (pair) per SM instead of the fewest that give the
                                      same number of waves */
-    PEAK_TUNE_COUNT_ = 12
+    PEAK_TUNE_EPILOGUE_WARPS = 12, /* one-slot (128- / 256-wide) tiles: 1 = one group of four epilogue warps, 2 = two
+                                      groups that drain half of the columns each (default: two for problems of at
+                                      most two waves) */
+    PEAK_TUNE_COUNT_ = 13
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

@@ -24,6 +24,7 @@ struct peak_mc_request {
     int balanced_grid;      // PEAK_TUNE_BALANCED_GRID value
     const float *bias;      // fused epilogue: fp32 value per column (device) or NULL
     int activation;         // fused epilogue: a peak_activation_t
+    int epilogue_warps;     // PEAK_TUNE_EPILOGUE_WARPS value
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

@@ -54,8 +54,8 @@ template <int CG, int BN> struct Cfg {
     // A tile wider than one MMA (BN = 512) is computed as two 256-column halves, one per accumulator slot.
     static constexpr int SLOT_N = BN > 256 ? 256 : BN;     // MMA N = width of one accumulator slot
     static constexpr int HALVES = BN / SLOT_N;
-    static constexpr int EPI_GROUPS = HALVES;              // groups of four epilogue warps
-    static constexpr int THREADS = 64 + 128 * EPI_GROUPS;
+    // groups of four epilogue warps: a two-half tile always has two; a one-slot tile may get two as well (G2)
+    static constexpr int threads(bool g2) { return 64 + 128 * ((HALVES == 2 || g2) ? 2 : 1); }
     static constexpr int HROWS = SLOT_N / CG;              // rows of op(B)^T this CTA stages per half
     static constexpr int B_ROWS = HALVES * HROWS;
     static constexpr int B_BOX_ROWS = HROWS < 128 ? HROWS : 128;
@@ -391,8 +391,11 @@ template <> struct McOps<0> {
 // IN8: the inputs are 8-bit floats.  A k-block is still one 128-byte swizzle row per matrix row, so it holds
 // 128 elements instead of 64, every byte count and descriptor stays as it is, and the MMA is the f8f6f4 kind
 // with K = 32 per instruction.  Both operands must be K-major (A not transposed, B transposed).
-template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false>
-__global__ void __launch_bounds__((Cfg<CG, BN>::THREADS), 1)
+// G2: a one-slot tile is drained by two groups of four epilogue warps, each taking half of the columns.  The
+// epilogue of such a tile hides behind the next tile's main loop, so the second group only pays when there is
+// no next tile: problems of at most two waves, where it shortens the exposed tail of the launch.
+template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false, bool G2 = false>
+__global__ void __launch_bounds__((Cfg<CG, BN>::threads(G2)), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
                  float *__restrict__ ws, const UmmaParams p) {
@@ -434,7 +437,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(accfull0 + 8 * b, 1);
-            ptx::mbar_init(accempty0 + 8 * b, 4 * CG);  // one arrival per epilogue warp (of one group) per CTA
+            // one arrival per epilogue warp that drains the slot, in every CTA
+            ptx::mbar_init(accempty0 + 8 * b, ((C_::HALVES == 1 && G2) ? 8 : 4) * CG);
         }
         for (int b = 0; b < 8; ++b) ptx::mbar_init(cbar0 + 8 * b, 1);
         *abort_flag = 0;
@@ -610,12 +614,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------------------------ epilogue (4 or 8 warps)
         const int q = warp & 3;          // TMEM lane quadrant this warp may read
         const int grp = (warp - 2) >> 2; // group of four warps: drains half `grp` of a two-half tile
-        constexpr int W = C_::SLOT_N;    // columns a warp drains per tile
+        constexpr bool SPLIT_COLS = C_::HALVES == 1 && G2;             // two groups share one slot
+        constexpr int W = SPLIT_COLS ? C_::SLOT_N / 2 : C_::SLOT_N;    // columns a warp drains per tile
         // staging: two buffers per warp in a one-group kernel (old C of chunk c + 1 arrives while chunk c is
         // worked on), one per warp with two groups
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (C_::HALVES == 1 ? 2u : 1u) * EPI_BUF_BYTES;
+        constexpr bool ONE_GROUP = C_::HALVES == 1 && !G2;
+        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (ONE_GROUP ? 2u : 1u) * EPI_BUF_BYTES;
         const bool vec = p.vec_ok != 0;
-        CFetch cf{cbar0 + 16u * (uint32_t)(warp - 2), 0u, C_::HALVES == 1 && p.c_prefetch != 0};
+        CFetch cf{cbar0 + 16u * (uint32_t)((warp - 2) & 3), 0u, ONE_GROUP && p.c_prefetch != 0};
         CFetch no_cf{0u, 0u, false};
         uint32_t tl = 0;
         bool ok = true;
@@ -626,11 +632,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
             const int n0 = (int)tn * BN;
+            const bool live = row0 < p.M;  // none of this warp's 32 rows exists otherwise: nothing to drain
             {
                 const int hf = (C_::HALVES == 2) ? grp : 0;
                 const uint32_t b = (C_::HALVES == 1) ? (tl & 1u) : (uint32_t)hf;
                 const uint32_t aph = (C_::HALVES == 1) ? ((tl >> 1) & 1u) : (tl & 1u);
-                if (cf.on && w.ws_block < 0) {
+                if (cf.on && live && w.ws_block < 0) {
                     // old C of the first two chunks is requested while the main loop still runs
                     constexpr int CC = 128 / (int)sizeof(TOut);
                     if (lane == 0) {
@@ -648,10 +655,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const int co = hf * C_::SLOT_N;  // first tile column of this warp
-                const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * C_::SLOT_N;
+                const int co = SPLIT_COLS ? grp * W : hf * C_::SLOT_N;  // first tile column of this warp
+                const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * C_::SLOT_N +
+                                        (SPLIT_COLS ? (uint32_t)(grp * W) : 0u);
                 const int nh = n0 + co;
-                if (w.ws_block < 0) {
+                if (!live) {
+                    // rows beyond M: the partial-tile reduction and C never look at them
+                } else if (w.ws_block < 0) {
                     // whole tile: alpha/beta epilogue straight to C
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;

@@ -104,11 +104,11 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     return best;
 }
 
-template <int CG, int BN, typename TOut, bool BATCHED, bool IN8 = false>
+template <int CG, int BN, typename TOut, bool BATCHED, bool IN8 = false, bool G2 = false>
 int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws) {
     using C_ = Cfg<CG, BN>;
     constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block
-    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8, G2>;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -188,7 +188,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(units * CG));
-    cfg.blockDim = dim3(C_::THREADS);
+    cfg.blockDim = dim3(C_::threads(G2));
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = g.stream;
     cudaLaunchAttribute attr[2];
@@ -215,23 +215,40 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     return PEAK_OK;
 }
 
+// Two groups of epilogue warps on a one-slot tile (G2): measured on problems of one or two waves, where the
+// last tile's epilogue is an exposed tail of the launch (fp16 2048^3 -> fp32: see the A/B notes); on longer
+// runs the extra warps cost about 1 %.  16-bit inputs, single matrices.
+template <int BN> bool want_two_groups(const GemmArgs &g, const Plan &plan, int units) {
+    if (BN == 512 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype))) return false;
+    const int mode = tuning(PEAK_TUNE_EPILOGUE_WARPS);  // 1 = four warps, 2 = eight warps
+    if (mode) return mode == 2;
+    return plan.tail_splits == 1 && (int64_t)plan.full_tiles <= 2 * (int64_t)units;
+}
+
 template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, int units, float *ws) {
+    const bool g2 = want_two_groups<BN>(g, plan, units);
     switch (out_elem(g.dtype)) {
         case Elem::F32:
             if (is_fp8(in_elem(g.dtype)))
                 return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true, true>(g, plan, units, ws)
                                       : launch_kernel<CG, BN, float, false, true>(g, plan, units, ws);
-            return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true>(g, plan, units, ws)
-                                  : launch_kernel<CG, BN, float, false>(g, plan, units, ws);
+            if (g.nbatch() > 1) return launch_kernel<CG, BN, float, true>(g, plan, units, ws);
+            if constexpr (BN != 512)
+                if (g2) return launch_kernel<CG, BN, float, false, false, true>(g, plan, units, ws);
+            return launch_kernel<CG, BN, float, false>(g, plan, units, ws);
         case Elem::F16:
-            return g.nbatch() > 1 ? launch_kernel<CG, BN, __half, true>(g, plan, units, ws)
-                                  : launch_kernel<CG, BN, __half, false>(g, plan, units, ws);
+            if (g.nbatch() > 1) return launch_kernel<CG, BN, __half, true>(g, plan, units, ws);
+            if constexpr (BN != 512)
+                if (g2) return launch_kernel<CG, BN, __half, false, false, true>(g, plan, units, ws);
+            return launch_kernel<CG, BN, __half, false>(g, plan, units, ws);
         case Elem::BF16:
             if (is_fp8(in_elem(g.dtype)))
                 return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true, true>(g, plan, units, ws)
                                       : launch_kernel<CG, BN, __nv_bfloat16, false, true>(g, plan, units, ws);
-            return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws)
-                                  : launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);
+            if (g.nbatch() > 1) return launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws);
+            if constexpr (BN != 512)
+                if (g2) return launch_kernel<CG, BN, __nv_bfloat16, false, false, true>(g, plan, units, ws);
+            return launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);
     }
     return PEAK_ERR_INVALID_VALUE;
 }
@@ -345,25 +362,6 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     Plan plan = choose_plan(g, cta_group, units);
     const bool in8 = is_fp8(in_elem(g.dtype));
     const bool whole256 = cta_group == 2 && plan.bn == 256 && plan.tail_splits == 1;
-    // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
-    // Measured (sustained, random inputs): +2..3 % at 4096^3, +12 % at 5000x3000x2500, but -3..-6 % from
-    // 2.7e11 flop on (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
-    const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
-    if (whole256 && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
-        const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
-        const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
-        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {
-            peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
-                              g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
-                              tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
-                              tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act, 0};
-            if (!r.status) return PEAK_ERR_CUDA;
-            const int rc = mc_entry()(&r);
-            if (rc == PEAK_OK) { count_launch(); return rc; }
-            if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
-            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
-        }
-    }
     // 256 x 512 pair tiles move a third less operand data per flop, but the tile fills the tensor memory, so
     // its epilogue (two groups of warps, one per half) is exposed once per tile.  Measured under the power
     // cap (sustained, random inputs): with 16-bit inputs and beta = 0 they win from 64 k-blocks on (+2 % at
@@ -372,6 +370,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // k-blocks take the same time but whose 256-wide tiles are less starved, from 128 k-blocks (K = 16384)
     // on (+3 %).  They must fill the grid as well as the 256-wide tiles do (4096x8192x4096: 3.46 waves
     // against 6.9, -3 %).
+    bool wide = false;
     if (whole256 && !tuning(PEAK_TUNE_TILE_N)) {
         const int bke = in8 ? 2 * BK : BK;
         const int64_t num_kb = (g.K + bke - 1) / bke;
@@ -379,8 +378,32 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         const int64_t min_kb = (!in8 && light_tail) ? 64 : 128;
         auto fill = [&](int64_t tiles) { return (double)tiles / (double)(((tiles + units - 1) / units) * units); };
         const int64_t t512 = tiles_of(g, 2, 512), t256 = tiles_of(g, 2, 256);
-        if (num_kb >= min_kb && t512 >= units && fill(t512) >= fill(t256) - 0.02) plan = Plan{512, (int)t512, 1};
+        wide = num_kb >= min_kb && t512 >= units && fill(t512) >= fill(t256) - 0.02;
     }
+    // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
+    // Measured (sustained, random inputs, interleaved): fp16 4096^3 -> fp32 1162 against 1132 (512-wide) and
+    // 1108 (256-wide); +12 % at 5000x3000x2500; but with 16-bit output, where the exposed epilogue of the wide
+    // tile is half as long, the wide tile wins (bf16 4096^3: 1231 against 1244-1249), and from 2.7e11 flop on
+    // the plug-in loses 3-6 % (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
+    const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
+    const bool wide_first = wide && elem_bytes(out_elem(g.dtype)) == 2;
+    if (whole256 && mc_mode != 1 && (mc_mode == 2 || !wide_first) && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
+        const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
+        const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
+        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {
+            peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
+                              g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
+                              tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
+                              tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act,
+                              tuning(PEAK_TUNE_EPILOGUE_WARPS), 0};
+            if (!r.status) return PEAK_ERR_CUDA;
+            const int rc = mc_entry()(&r);
+            if (rc == PEAK_OK) { count_launch(); return rc; }
+            if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
+            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+        }
+    }
+    if (wide) plan = Plan{512, (int)tiles_of(g, 2, 512), 1};
     if (cta_group == 2) {
         if (plan.bn == 512) return run_umma<2, 512>(g, plan, units);
         return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);

@@ -52,10 +52,10 @@ int tuning(int) { return 0; }
 namespace {
 using namespace umma;
 
-template <typename TOut> int launch_mc(peak_mc_request *r) {
+template <typename TOut, bool G2> int launch_mc(peak_mc_request *r) {
     constexpr int CG = 2, BN = 256;
     using C_ = Cfg<CG, BN>;
-    auto kernel = umma_gemm_kernel<CG, BN, TOut, 1>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 1, false, false, G2>;
     static cudaError_t attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
     if (attr_err != cudaSuccess) { r->cuda_error = (int)attr_err; return PEAK_ERR_CUDA; }
 
@@ -93,7 +93,7 @@ template <typename TOut> int launch_mc(peak_mc_request *r) {
     p.inject_stall = r->inject_stall == 1 ? 1 : 0;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(C_::THREADS);
+    cfg.blockDim = dim3(C_::threads(G2));
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = r->stream;
     cudaLaunchAttribute attr[2];
@@ -133,10 +133,14 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
     if (!r) return PEAK_ERR_INVALID_VALUE;
     r->cuda_error = 0;
     if (in_elem(r->dtype) == Elem::F32 || r->M < 1 || r->N < 1 || r->K < 1) return PEAK_ERR_UNSUPPORTED;
+    // two groups of epilogue warps when the launch is at most two waves of 512 x 256 super-tiles long (the
+    // last tile's epilogue is then a visible part of the run time)
+    const int64_t super_tiles = ((r->M + 511) / 512) * ((r->N + 255) / 256);
+    const bool g2 = r->epilogue_warps ? r->epilogue_warps == 2 : super_tiles <= 64;
     switch (out_elem(r->dtype)) {
-        case Elem::F32: return launch_mc<float>(r);
-        case Elem::F16: return launch_mc<__half>(r);
-        case Elem::BF16: return launch_mc<__nv_bfloat16>(r);
+        case Elem::F32: return g2 ? launch_mc<float, true>(r) : launch_mc<float, false>(r);
+        case Elem::F16: return g2 ? launch_mc<__half, true>(r) : launch_mc<__half, false>(r);
+        case Elem::BF16: return g2 ? launch_mc<__nv_bfloat16, true>(r) : launch_mc<__nv_bfloat16, false>(r);
     }
     return PEAK_ERR_INVALID_VALUE;
 }

@@ -24,6 +24,7 @@ SPACE_16BIT = {
     3: [1, 2],                   # PEAK_TUNE_EPILOGUE
     10: [1, 2],                  # PEAK_TUNE_MULTICAST
     0: [0, 2, 16],               # PEAK_TUNE_RASTER_GROUP
+    12: [1, 2],                  # PEAK_TUNE_EPILOGUE_WARPS
 }
 SPACE_F32 = {
     "variant": ["sgemm"],
@@ -31,7 +32,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 12
+NUM_KEYS = 13
 
 
 def candidates(space: dict, quick: bool = False):

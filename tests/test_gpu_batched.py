@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(12):
+    for key in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(key, 0)
 
 

@@ -32,7 +32,7 @@ def k_major(dtype, M, N, K, **kw):
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(12):
+    for key in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(key, 0)
 
 

@@ -19,7 +19,7 @@ LIP = {P.PEAK_ACT_NONE: 1.0, P.PEAK_ACT_RELU: 1.0, P.PEAK_ACT_GELU: 1.13}
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(12):
+    for key in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(key, 0)
 
 
@@ -80,7 +80,7 @@ def test_fused_tail_code_paths(act, reset_tuning):
     if P.peak_multicast_available():
         settings.append({P.PEAK_TUNE_MULTICAST: 2})
     for knobs in settings:
-        for key in range(12):
+        for key in range(P.PEAK_TUNE_COUNT):
             P.peak_set_tuning(key, knobs.get(key, 0))
         dc = run_fused(c, P.PEAK_VARIANT_UMMA_2CTA, bias, act)
         check_fused(dc, bias, act, f"knobs {knobs} act={act}")

@@ -256,7 +256,7 @@ def test_launch_counter_moves():
 @pytest.fixture
 def reset_tuning():
     yield
-    for key in range(12):
+    for key in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(key, 0)
 
 
@@ -521,3 +521,30 @@ def test_inf_nan_propagate_and_outputs_overflow_to_inf(variant, dtype):
         want = W.to_float64(oracle.round_to(R.OT[c.out_type], ref), c.out_type)
         assert np.isinf(want).any() and np.array_equal(np.isinf(got), np.isinf(want))
         assert np.array_equal(np.sign(got[np.isinf(got)]), np.sign(want[np.isinf(want)]))
+
+
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("warps", [1, 2])
+@pytest.mark.parametrize("tile_n", [128, 256])
+def test_umma_epilogue_warp_groups(variant, warps, tile_n, reset_tuning):
+    """One or two groups of epilogue warps on one-slot tiles: same bits (integers), same tolerance (reals),
+    for every output type, with ragged edges, alpha/beta, a k-split and both store paths."""
+    P.peak_set_tuning(P.PEAK_TUNE_EPILOGUE_WARPS, warps)
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, tile_n)
+    for dtype in PAIRS_16:
+        for (ta, tb, M, N, K, split) in [(0, 0, 384, 520, 200, 0), (1, 1, 200, 328, 264, 2), (0, 1, 130, 257, 136, 0)]:
+            P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+            pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+            ci = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.25, beta=-1.0, pad_a=pa, pad_b=pb, case=tile_n + warps)
+            di = R.DeviceCase(ci)
+            di.run(variant)
+            ref, _ = di.oracle_full()
+            want = oracle.round_to(R.OT[ci.out_type], ref)
+            got = di.result()
+            if ci.out_type == "f32":
+                got = got.view(np.uint32)
+            assert np.array_equal(got, want), f"{ci.name} warps={warps} tile_n={tile_n} split={split}"
+            cr = ci.with_(dist="uniform", alpha=0.5, beta=2.0)
+            dr = R.DeviceCase(cr)
+            dr.run(variant)
+            R.check_full(dr, what=f"{cr.name} warps={warps} tile_n={tile_n} split={split}")
