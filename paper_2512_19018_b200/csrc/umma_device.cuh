@@ -725,9 +725,14 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
     int64_t tm, tn;
     tile_coord(gt - bz * tiles_per_batch, tiles_m, tiles_n, group, tm, tn);
     const int vec_per_row = bn / 4;
-    const int total_vec = rows_t * vec_per_row;
+    const int64_t rows_left = (int64_t)M - tm * rows_t;  // rows of this tile that exist
+    const int total_vec = (int)(rows_left < rows_t ? rows_left : rows_t) * vec_per_row;
     const int64_t block_elems = (int64_t)rows_t * bn;
     const float *base = ws + (int64_t)t * splits * block_elems;
+    // launched as a programmatic dependent of the GEMM kernel: everything above overlapped its tail; the
+    // partial tiles may be read only once that kernel has completed
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < total_vec; e += blocks_per_tile * blockDim.x) {
         const int r = e / vec_per_row, c4 = e - r * vec_per_row;
         const int64_t i = tm * rows_t + r;

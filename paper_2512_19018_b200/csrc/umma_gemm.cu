@@ -205,12 +205,21 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 
     // second kernel: add the slices of the split tiles in order, apply alpha/beta
     const int split_tiles = tiles - plan.full_tiles;
-    dim3 rgrid((unsigned)split_tiles, split_tiles >= 64 ? 2u : 8u);
-    splitk_reduce_kernel<TOut><<<rgrid, 256, 0, g.stream>>>(ws, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
-                                                            p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C,
-                                                            g.ldc, g.strideC, p.vec_ok, g.bias, g.act);
+    cudaLaunchConfig_t rcfg = {};
+    rcfg.gridDim = dim3((unsigned)split_tiles, split_tiles >= 64 ? 2u : 8u);
+    rcfg.blockDim = dim3(256);
+    rcfg.dynamicSmemBytes = 0;
+    rcfg.stream = g.stream;
+    cudaLaunchAttribute rattr[1];
+    rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    rattr[0].val.programmaticStreamSerializationAllowed = 1;
+    rcfg.attrs = rattr;
+    rcfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 0 : 1;
+    const float *ws_c = ws;
+    e = cudaLaunchKernelEx(&rcfg, splitk_reduce_kernel<TOut>, ws_c, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
+                           p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C, g.ldc, g.strideC, p.vec_ok,
+                           g.bias, g.act);
     count_launch();
-    e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
