@@ -136,6 +136,7 @@ int gemm_impl(int variant, int dtype, int transA, int transB, int64_t M, int64_t
 struct Staging {
     void *ptr = nullptr;
     size_t bytes = 0;
+    int device = -1;  // the device the buffer lives on
 };
 Staging g_stage[3];
 
@@ -151,11 +152,16 @@ HostPipeline g_pipe;
 std::mutex g_stage_mutex;
 
 int ensure(Staging &s, size_t need) {
-    if (need <= s.bytes) return PEAK_OK;
-    if (s.ptr) { cudaFree(s.ptr); s.ptr = nullptr; s.bytes = 0; }
-    cudaError_t e = cudaMalloc(&s.ptr, need);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    if (need <= s.bytes && (s.device == dev || s.bytes == 0)) return PEAK_OK;
+    if (s.ptr) { cudaFree(s.ptr); s.ptr = nullptr; s.bytes = 0; }  // too small, or on another device
+    if (need == 0) return PEAK_OK;
+    e = cudaMalloc(&s.ptr, need);
     if (e != cudaSuccess) { set_cuda_error(e); s.ptr = nullptr; return PEAK_ERR_NO_MEMORY; }
     s.bytes = need;
+    s.device = dev;
     return PEAK_OK;
 }
 

@@ -181,6 +181,7 @@ int launch_scale(const GemmArgs &g) {
         case Elem::F32: return run_scale<float>(g);
         case Elem::F16: return run_scale<__half>(g);
         case Elem::BF16: return run_scale<__nv_bfloat16>(g);
+        default: break;  // outputs are never 8-bit
     }
     return PEAK_ERR_INVALID_VALUE;
 }

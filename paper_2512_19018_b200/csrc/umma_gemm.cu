@@ -258,6 +258,7 @@ template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, 
             if constexpr (BN != 512)
                 if (g2) return launch_kernel<CG, BN, __nv_bfloat16, false, false, true>(g, plan, units, ws);
             return launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);
+        default: break;  // outputs are never 8-bit
     }
     return PEAK_ERR_INVALID_VALUE;
 }

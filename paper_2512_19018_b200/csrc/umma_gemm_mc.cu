@@ -141,6 +141,7 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
         case Elem::F32: return g2 ? launch_mc<float, true>(r) : launch_mc<float, false>(r);
         case Elem::F16: return g2 ? launch_mc<__half, true>(r) : launch_mc<__half, false>(r);
         case Elem::BF16: return g2 ? launch_mc<__nv_bfloat16, true>(r) : launch_mc<__nv_bfloat16, false>(r);
+        default: break;  // outputs are never 8-bit
     }
     return PEAK_ERR_INVALID_VALUE;
 }
