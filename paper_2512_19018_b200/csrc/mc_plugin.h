@@ -25,6 +25,7 @@ struct peak_mc_request {
     const float *bias;      // fused epilogue: fp32 value per column (device) or NULL
     int activation;         // fused epilogue: a peak_activation_t
     int epilogue_warps;     // PEAK_TUNE_EPILOGUE_WARPS value
+    int tile_n;             // 256 (512 x 256 super-tiles) or 512 (512 x 512 super-tiles of two-half tiles)
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

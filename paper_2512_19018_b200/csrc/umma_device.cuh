@@ -419,7 +419,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    static_assert(MC == 0 || (CG == 2 && BN == 256), "the multicast build pairs CTAs and uses 256-wide tiles");
+    static_assert(MC == 0 || (CG == 2 && BN >= 256), "the multicast build pairs CTAs and uses 256- or 512-wide tiles");
     constexpr int CLUSTER = MC ? 4 : CG;       // CTAs that work on one (super-)tile together
     const uint32_t crank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
     const uint32_t rank = crank & 1u;          // position inside the CTA pair
@@ -506,9 +506,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // this CTA's quarter (64 of the pair-wide tile's 256 columns) goes to itself and to the
                         // CTA of the same parity in the other pair; both layouts use 64 x 64 boxes of 8 KiB
                         const uint16_t mask = (uint16_t)((1u << crank) | (1u << (crank ^ 2u)));
-                        const int n_q = n_cta + 64 * (int)pair;
-                        McOps<MC>::load_b_quarter(b_dst + pair * ATOM_BYTES, &tmB, p.b_mn ? n_q : k0, p.b_mn ? k0 : n_q,
-                                                  bz, bar, mask);
+#pragma unroll
+                        for (int hf = 0; hf < C_::HALVES; ++hf) {
+                            const int n_q = n_cta + hf * C_::SLOT_N + 64 * (int)pair;
+                            McOps<MC>::load_b_quarter(b_dst + hf * C_::HROWS * 128 + pair * ATOM_BYTES, &tmB,
+                                                      p.b_mn ? n_q : k0, p.b_mn ? k0 : n_q, bz, bar, mask);
+                        }
                     } else if (!p.b_mn) {
 #pragma unroll
                         for (int hf = 0; hf < C_::HALVES; ++hf) {

@@ -396,16 +396,21 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // tile is half as long, the wide tile wins (bf16 4096^3: 1231 against 1244-1249), and from 2.7e11 flop on
     // the plug-in loses 3-6 % (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
+    // With a 16-bit output the wide tile is preferred, and the plug-in then shares its 512-wide B tile between
+    // the two pairs of a cluster (512 x 512 super-tiles): bf16 4096^3 1222 -> 1248 in the bench protocol; at
+    // 8192^3, beyond the plug-in's size limit, it would lose (1251 against 1327: only 33 clusters fit).
     const bool wide_first = wide && elem_bytes(out_elem(g.dtype)) == 2;
-    if (whole256 && mc_mode != 1 && (mc_mode == 2 || !wide_first) && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
-        const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + 255) / 256);
+    const bool whole512 = cta_group == 2 && plan.bn == 512 && plan.tail_splits == 1 && mc_mode == 2;  // forced
+    if ((whole256 || whole512) && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
+        const int mc_tile_n = (whole512 || wide_first) ? 512 : 256;
+        const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + mc_tile_n - 1) / mc_tile_n);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
         if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {
             peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
                               tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act,
-                              tuning(PEAK_TUNE_EPILOGUE_WARPS), 0};
+                              tuning(PEAK_TUNE_EPILOGUE_WARPS), mc_tile_n, 0};
             if (!r.status) return PEAK_ERR_CUDA;
             const int rc = mc_entry()(&r);
             if (rc == PEAK_OK) { count_launch(); return rc; }

@@ -7,9 +7,9 @@
 // Clusters of four CTAs = two CTA pairs stacked in M work on a 512 x 256 super-tile.  Both pairs need the
 // same 256-column B tile for every k-block; each CTA fetches one 64-column quarter of it and the copy engine
 // delivers that quarter to the CTA itself and to the CTA of the same parity in the other pair.  L2 reads per
-// super-tile k-block drop from 128 KiB to 96 KiB.  Measured motivation: under the 1 kW power cap the
-// L2 -> shared-memory traffic is a large part of the energy budget (cutting a quarter of it raised the
-// sustained throughput of the plain kernel by 24-31 %).
+// super-tile k-block drop from 128 KiB to 96 KiB (512 x 512 super-tiles of two-half tiles: from 192 to 128).
+// Motivation: one SM's L2 port sustains 40-57 bytes per cycle, a 256 x 256 pair tile asks for 64, and under
+// the 1 kW power cap operand traffic is part of the energy budget (measured gains: a few per cent).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -52,8 +52,8 @@ int tuning(int) { return 0; }
 namespace {
 using namespace umma;
 
-template <typename TOut, bool G2> int launch_mc(peak_mc_request *r) {
-    constexpr int CG = 2, BN = 256;
+template <typename TOut, bool G2, int BN = 256> int launch_mc(peak_mc_request *r) {
+    constexpr int CG = 2;
     using C_ = Cfg<CG, BN>;
     auto kernel = umma_gemm_kernel<CG, BN, TOut, 1, false, false, G2>;
     static cudaError_t attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
@@ -78,7 +78,7 @@ template <typename TOut, bool G2> int launch_mc(peak_mc_request *r) {
     p.a_mn = a_mn; p.b_mn = b_mn;
     const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
+              ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = r->alpha; p.beta = r->beta;
     p.C = r->C; p.ldc = r->ldc;
     p.bias = r->bias; p.act = r->activation;
@@ -137,6 +137,15 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
     // last tile's epilogue is then a visible part of the run time)
     const int64_t super_tiles = ((r->M + 511) / 512) * ((r->N + 255) / 256);
     const bool g2 = r->epilogue_warps ? r->epilogue_warps == 2 : super_tiles <= 64;
+    if (r->tile_n == 512) {  // two-half tiles: 512 x 512 super-tiles
+        switch (out_elem(r->dtype)) {
+            case Elem::F32: return launch_mc<float, false, 512>(r);
+            case Elem::F16: return launch_mc<__half, false, 512>(r);
+            case Elem::BF16: return launch_mc<__nv_bfloat16, false, 512>(r);
+            default: break;
+        }
+        return PEAK_ERR_INVALID_VALUE;
+    }
     switch (out_elem(r->dtype)) {
         case Elem::F32: return g2 ? launch_mc<float, true>(r) : launch_mc<float, false>(r);
         case Elem::F16: return g2 ? launch_mc<__half, true>(r) : launch_mc<__half, false>(r);

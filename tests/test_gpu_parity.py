@@ -384,14 +384,16 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant, reset_tuning
     R.check_full(dc)
 
 
+@pytest.mark.parametrize("tile_n", [256, 512])
 @pytest.mark.parametrize("dtype", [W.PEAK_BF16_BF16, W.PEAK_F16_F32])
 @pytest.mark.parametrize("ta,tb", LAYOUTS)
-def test_multicast_plugin_matches_oracle(dtype, ta, tb, reset_tuning):
+def test_multicast_plugin_matches_oracle(dtype, ta, tb, tile_n, reset_tuning):
     """The optional cluster-multicast plug-in (four-CTA clusters sharing B tiles), forced on: exact on integer
     inputs for every layout, within the bounds on real inputs with alpha/beta and ragged edges, and identical
     to the plain kernel's output bit for bit on the integer cases."""
     if not P.peak_multicast_available():
         pytest.skip("libpeak_gemm_mc.so is not present (multi-GPU runs leave it out)")
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, tile_n)      # 512 x 256 or 512 x 512 super-tiles
     for idx, (M, N, K) in enumerate([(512, 256, 64), (1024, 512, 448), (700, 328, 264), (1536, 1280, 1024)]):
         pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8     # TMA needs pitches that are multiples of 8
         ci = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.125, beta=-1.0, case=idx, pad_a=pa, pad_b=pb, pad_c=8)
