@@ -399,10 +399,11 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // With a 16-bit output the wide tile is preferred, and the plug-in then shares its 512-wide B tile between
     // the two pairs of a cluster (512 x 512 super-tiles): bf16 4096^3 1222 -> 1248 in the bench protocol; at
     // 8192^3, beyond the plug-in's size limit, it would lose (1251 against 1327: only 33 clusters fit).
+    // (8-bit inputs, 256-wide tiles only: 2048^3 1295 -> 1415, 4096^3 unchanged, larger problems excluded as above)
     const bool wide_first = wide && elem_bytes(out_elem(g.dtype)) == 2;
     const bool whole512 = cta_group == 2 && plan.bn == 512 && plan.tail_splits == 1 && mc_mode == 2;  // forced
-    if ((whole256 || whole512) && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && !in8 && mc_entry()) {
-        const int mc_tile_n = (whole512 || wide_first) ? 512 : 256;
+    if ((whole256 || whole512) && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && mc_entry()) {
+        const int mc_tile_n = ((whole512 || wide_first) && !in8) ? 512 : 256;
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + mc_tile_n - 1) / mc_tile_n);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
         if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {

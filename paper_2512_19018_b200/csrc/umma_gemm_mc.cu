@@ -52,23 +52,25 @@ int tuning(int) { return 0; }
 namespace {
 using namespace umma;
 
-template <typename TOut, bool G2, int BN = 256> int launch_mc(peak_mc_request *r) {
+template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(peak_mc_request *r) {
     constexpr int CG = 2;
+    constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block (8-bit inputs: 128 per 128-byte row)
     using C_ = Cfg<CG, BN>;
-    auto kernel = umma_gemm_kernel<CG, BN, TOut, 1, false, false, G2>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 1, false, IN8, G2>;
     static cudaError_t attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
     if (attr_err != cudaSuccess) { r->cuda_error = (int)attr_err; return PEAK_ERR_CUDA; }
 
     const Elem ein = in_elem(r->dtype), eout = out_elem(r->dtype);
     const int a_mn = r->transA ? 1 : 0, b_mn = r->transB ? 0 : 1;
     CUtensorMap tmA, tmB, tmC;
-    bool ok = a_mn ? make_map(&tmA, ein, r->A, r->M, r->K, r->lda, 64, BK) : make_map(&tmA, ein, r->A, r->K, r->M, r->lda, BK, 128);
-    ok = ok && (b_mn ? make_map(&tmB, ein, r->B, r->N, r->K, r->ldb, 64, BK) : make_map(&tmB, ein, r->B, r->K, r->N, r->ldb, BK, 64));
+    if (IN8 && (a_mn || b_mn)) return PEAK_ERR_UNSUPPORTED;  // 8-bit operands: K-major only
+    bool ok = a_mn ? make_map(&tmA, ein, r->A, r->M, r->K, r->lda, 64, BK) : make_map(&tmA, ein, r->A, r->K, r->M, r->lda, BKE, 128);
+    ok = ok && (b_mn ? make_map(&tmB, ein, r->B, r->N, r->K, r->ldb, 64, BK) : make_map(&tmB, ein, r->B, r->K, r->N, r->ldb, BKE, 64));
     if (!ok) return PEAK_ERR_CUDA;
 
     UmmaParams p;
     p.M = (int)r->M; p.N = (int)r->N; p.K = (int)r->K;
-    p.num_kb = (int)((r->K + BK - 1) / BK);
+    p.num_kb = (int)((r->K + BKE - 1) / BKE);
     p.tiles_m = (int)((r->M + 4 * BM - 1) / (4 * BM));  // 512-row super-tiles
     p.tiles_n = (int)((r->N + BN - 1) / BN);
     p.group = r->raster_group > 0 ? r->raster_group : 2;  // super-tile rows per raster group (measured best)
@@ -76,7 +78,7 @@ template <typename TOut, bool G2, int BN = 256> int launch_mc(peak_mc_request *r
     p.tiles_per_batch = tiles; p.stride_c = 0;
     p.full_tiles = tiles; p.tail_splits = 1; p.kb_per_split = p.num_kb; p.total_items = tiles;
     p.a_mn = a_mn; p.b_mn = b_mn;
-    const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
+    const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = r->alpha; p.beta = r->beta;
@@ -137,6 +139,15 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
     // last tile's epilogue is then a visible part of the run time)
     const int64_t super_tiles = ((r->M + 511) / 512) * ((r->N + 255) / 256);
     const bool g2 = r->epilogue_warps ? r->epilogue_warps == 2 : super_tiles <= 64;
+    if (is_fp8(in_elem(r->dtype))) {  // 8-bit inputs: 256-wide tiles, bf16 or fp32 output
+        switch (out_elem(r->dtype)) {
+            case Elem::F32: return g2 ? launch_mc<float, true, 256, true>(r) : launch_mc<float, false, 256, true>(r);
+            case Elem::BF16:
+                return g2 ? launch_mc<__nv_bfloat16, true, 256, true>(r) : launch_mc<__nv_bfloat16, false, 256, true>(r);
+            default: break;
+        }
+        return PEAK_ERR_INVALID_VALUE;
+    }
     if (r->tile_n == 512) {  // two-half tiles: 512 x 512 super-tiles
         switch (out_elem(r->dtype)) {
             case Elem::F32: return launch_mc<float, false, 512>(r);

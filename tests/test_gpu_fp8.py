@@ -163,3 +163,28 @@ def test_fp8_fused_bias_activation(act):
         bias = (rng.standard_normal(c.N) * 2).astype(np.float32)
         dc = run_fused(c, variant, bias, act)
         check_fused(dc, bias, act, f"fp8 fused act={act} {P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32])
+def test_fp8_multicast_plugin(dtype, reset_tuning):
+    """8-bit inputs through the single-GPU multicast plug-in (forced on): integers bit for bit and identical
+    to the plain kernel, reals within the bounds."""
+    if not P.peak_multicast_available():
+        pytest.skip("libpeak_gemm_mc.so is not present (multi-GPU runs leave it out)")
+    for idx, (M, N, K) in enumerate([(512, 256, 128), (1024, 512, 896), (700, 328, 272), (1536, 1280, 2048)]):
+        ci = k_major(dtype, M, N, K, dist="smallint", alpha=0.125, beta=-1.0, pad_c=8, case=idx)
+        outs = []
+        for mode in (2, 1):
+            P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, mode)
+            dc = R.DeviceCase(ci)
+            n0 = P.peak_kernel_launches()
+            dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+            outs.append(dc.result().copy())
+            if mode == 2:
+                assert_bits_equal(ci, dc, f"{ci.name} multicast")
+        assert np.array_equal(outs[0], outs[1])
+        P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, 2)
+        cr = k_major(dtype, M, N, K, alpha=0.5, beta=2.0, dist="uniform", case=idx)
+        dr = R.DeviceCase(cr)
+        dr.run(P.PEAK_VARIANT_UMMA_2CTA)
+        R.check_full(dr, what=f"{cr.name} multicast")
