@@ -566,7 +566,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     ptx::tc_fence_after_sync();
                 }
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                // A two-half tile ends with its last k-blocks taken apart: half 0 finishes them first and is
+                // handed to its epilogue warps while the tensor cores still work on half 1, which shortens the
+                // exposed epilogue by that much.  The stages involved stay unreleased until half 1 has read them,
+                // so at most STAGES - 1 k-blocks can be treated this way.
+                const int kb_tail = (C_::HALVES == 2) ? max(kb0 + 1, kb1 - (STAGES - 1)) : kb1;
+                for (int kb = kb0; kb < kb_tail; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
                         report_timeout(p, abort_flag, 4, s);
@@ -604,11 +609,39 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     else ptx::umma_commit_pair(empty0 + 8 * s, MC ? 0xF : 3);
                 }
                 if (!ok) break;
+                if (C_::HALVES == 2) {
+#pragma unroll 1
+                    for (int hf = 0; hf < 2 && ok; ++hf) {
+                        uint32_t jt = it;
+                        for (int kb = kb_tail; kb < kb1; ++kb, ++jt) {
+                            const uint32_t s = jt % STAGES, ph = (jt / STAGES) & 1u;
+                            if (hf == 0) {
+                                if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
+                                    report_timeout(p, abort_flag, 4, s);
+                                    ok = false;
+                                    break;
+                                }
+                                ptx::tc_fence_after_sync();
+                            }
+                            const uint32_t a_base = stage_base + s * C_::STAGE_BYTES;
+                            const uint32_t bh_base = a_base + A_STAGE_BYTES + hf * C_::HROWS * 128;
+                            const uint32_t d_tmem = tmem_base + (uint32_t)hf * C_::SLOT_N;
 #pragma unroll
-                for (int hf = 0; hf < C_::HALVES; ++hf) {
-                    const uint32_t slot = (C_::HALVES == 1) ? b : (uint32_t)hf;
-                    if (CG == 1) ptx::umma_commit_1cta(accfull0 + 8 * slot);
-                    else ptx::umma_commit_pair(accfull0 + 8 * slot, (uint16_t)(3u << leader_crank));
+                            for (int k = 0; k < BK / UMMA_K; ++k) {
+                                const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
+                                const uint64_t bd = smem_desc(bh_base + k * b_kstep, b_lbo, 1024u);
+                                if (IN8) ptx::umma_f8<CG>(d_tmem, ad, bd, p.idesc, 1u);
+                                else ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, 1u);
+                            }
+                            if (hf == 1) ptx::umma_commit_pair(empty0 + 8 * s, MC ? 0xF : 3);  // two-half tiles are pairs
+                        }
+                        if (ok) ptx::umma_commit_pair(accfull0 + 8 * hf, (uint16_t)(3u << leader_crank));
+                    }
+                    if (!ok) break;
+                    it += (uint32_t)(kb1 - kb_tail);
+                } else {
+                    if (CG == 1) ptx::umma_commit_1cta(accfull0 + 8 * b);
+                    else ptx::umma_commit_pair(accfull0 + 8 * b, (uint16_t)(3u << leader_crank));
                 }
             }
         }
