@@ -140,6 +140,11 @@ template <int N> __device__ __forceinline__ void tma_store_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// ask for the 128-byte line at `p` to be brought into L2 (no register, no wait)
+__device__ __forceinline__ void prefetch_l2(const void *p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 // ---- programmatic dependent launch ------------------------------------------------------------
 // wait: returns once the kernels this launch depends on have completed and their writes are visible
 // (immediately when the launch carries no programmatic dependency)

@@ -230,18 +230,23 @@ __device__ __forceinline__ void unstage_row32(uint32_t buf, int lane, int h, flo
 
 // Old-C prefetch of one epilogue warp (beta != 0 with TMA stores): chunk c of a tile is loaded by TMA into
 // staging buffer c & 1, where the result later overwrites it in place and leaves by a TMA store.
+// With two staging buffers per warp (one-group kernels) chunk c uses buffer and barrier c & 1 and the load of
+// chunk c + 1 overlaps the work on chunk c; with one buffer per warp (two-group kernels: `single`) the next
+// chunk is requested as soon as the store of the current one has read the buffer.
 struct CFetch {
-    uint32_t bar0;    // two mbarriers of this warp, 8 bytes apart
+    uint32_t bar0;    // mbarrier(s) of this warp, 8 bytes apart
     uint32_t phases;  // bit b: parity the next wait on barrier b uses
     bool on;
+    bool single;
 };
 template <typename T, bool MAP3D>
 __device__ __forceinline__ void cfetch_issue(const CFetch &cf, uint32_t my_stage, int c, const CUtensorMap *tm, int x0,
                                              int y0, int z0) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);
-    const uint32_t bar = cf.bar0 + 8u * (uint32_t)(c & 1);
+    const uint32_t slot = cf.single ? 0u : (uint32_t)(c & 1);
+    const uint32_t bar = cf.bar0 + 8u * slot;
     ptx::mbar_arrive_expect_tx(bar, (uint32_t)EPI_BUF_BYTES);
-    const uint32_t dst = my_stage + (uint32_t)(c & 1) * EPI_BUF_BYTES;
+    const uint32_t dst = my_stage + slot * EPI_BUF_BYTES;
     if (MAP3D) ptx::tma_load_3d(dst, tm, x0 + c * CHUNK_COLS, y0, z0, bar);
     else ptx::tma_load_2d(dst, tm, x0 + c * CHUNK_COLS, y0, bar);
 }
@@ -281,7 +286,7 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
         const int col0 = cbase + c * CHUNK_COLS;
         if (col0 >= ncols) break;  // warp-uniform
-        const uint32_t buf = my_stage + (cf.on ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
+        const uint32_t buf = my_stage + ((cf.on && !cf.single) ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
         // the whole chunk is requested from tensor memory before the first wait
         uint32_t r[CHUNK_COLS / 32][32];
 #pragma unroll
@@ -291,13 +296,13 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
             // chunks 0 and 1 were requested before the accumulator was waited for; chunk c + 1 (c >= 1) goes
             // into the buffer chunk c - 1 left by a store, which has had this chunk's tensor-memory load to
             // finish reading it
-            if (c >= 1 && c + 1 < BN / CHUNK_COLS && cbase + (c + 1) * CHUNK_COLS < ncols) {
+            if (!cf.single && c >= 1 && c + 1 < BN / CHUNK_COLS && cbase + (c + 1) * CHUNK_COLS < ncols) {
                 if (lane == 0) {
                     ptx::tma_store_wait_read<0>();
                     cfetch_issue<T, MAP3D>(cf, my_stage, c + 1, tm, x0, y0, z0);
                 }
             }
-            const uint32_t b = (uint32_t)(c & 1);
+            const uint32_t b = cf.single ? 0u : (uint32_t)(c & 1);
             const bool got = ptx::mbar_wait<false>(cf.bar0 + 8u * b, (cf.phases >> b) & 1u, abort_flag, wait_cycles);
             cf.phases ^= 1u << b;
             if (!__all_sync(0xffffffffu, got)) return false;
@@ -359,6 +364,10 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                 if (MAP3D) ptx::tma_store_3d(tm, x0 + c * CHUNK_COLS, y0, z0, buf);
                 else ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
                 ptx::tma_store_commit();
+                if (cf.on && cf.single && c + 1 < BN / CHUNK_COLS && cbase + (c + 1) * CHUNK_COLS < ncols) {
+                    ptx::tma_store_wait_read<0>();  // the one buffer: its store must have read it
+                    cfetch_issue<T, MAP3D>(cf, my_stage, c + 1, tm, x0, y0, z0);
+                }
             }
         }
     }
@@ -657,8 +666,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         constexpr bool ONE_GROUP = C_::HALVES == 1 && !G2;
         const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (ONE_GROUP ? 2u : 1u) * EPI_BUF_BYTES;
         const bool vec = p.vec_ok != 0;
-        CFetch cf{cbar0 + 16u * (uint32_t)((warp - 2) & 3), 0u, ONE_GROUP && p.c_prefetch != 0};
-        CFetch no_cf{0u, 0u, false};
+        CFetch cf{ONE_GROUP ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
+                  p.c_prefetch != 0, !ONE_GROUP};
+        CFetch no_cf{0u, 0u, false, false};
         uint32_t tl = 0;
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
@@ -676,10 +686,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (cf.on && live && w.ws_block < 0) {
                     // old C of the first two chunks is requested while the main loop still runs
                     constexpr int CC = 128 / (int)sizeof(TOut);
+                    const int c0 = n0 + ((C_::HALVES == 2) ? hf * C_::SLOT_N : (SPLIT_COLS ? grp * W : 0));
                     if (lane == 0) {
-                        ptx::tma_store_wait_read<0>();  // the previous tile's stores have read both buffers
-                        cfetch_issue<TOut, BATCHED>(cf, my_stage, 0, &tmC, n0, row0, bz);
-                        if (n0 + CC < p.N && CC < C_::SLOT_N) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, n0, row0, bz);
+                        ptx::tma_store_wait_read<0>();  // the previous tile's stores have read the buffer(s)
+                        cfetch_issue<TOut, BATCHED>(cf, my_stage, 0, &tmC, c0, row0, bz);
+                        if (!cf.single && c0 + CC < p.N && CC < W) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, c0, row0, bz);
+                    }
+                    if (cf.single) {
+                        // the later chunks are fetched one by one between stores: have them wait in L2
+                        const int r = row0 + lane;
+                        if (r < p.M) {
+                            const TOut *row_ptr = reinterpret_cast<const TOut *>(p.C) +
+                                                  (BATCHED ? (int64_t)bz * p.stride_c : 0) + (int64_t)r * p.ldc + c0;
+#pragma unroll
+                            for (int c = CC; c < W; c += CC)
+                                if (c0 + c < p.N) ptx::prefetch_l2(row_ptr + c);
+                        }
                     }
                     __syncwarp();
                 }
