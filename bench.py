@@ -39,9 +39,9 @@ SM_COUNT, SM_MAX_MHZ = 148, 1965.0
 # DRAM bytes per launch (read + write) of the dominant kernel from the ncu capture summarised under
 # profiles/; None where no capture exists for the workload.
 NCU_TRAFFIC_BYTES = {
-    "bf16_4096_nn": 85.5e6,     # profiles/umma_gemm_multicast512_bf16_4096_nn.md (73.8 MB read + 11.7 MB written)
-    "bf16_8192_nn": 0.971e9,    # profiles/umma_gemm_2cta_512wide_bf16_8192_nn.md (0.851 GB read + 0.121 GB written)
-    "e4m3_8192_nt": 0.459e9,    # profiles/umma_gemm_2cta_e4m3_8192_nt.md (0.343 GB read + 0.116 GB written)
+    "bf16_4096_nn": 86.8e6,     # profiles/umma_gemm_multicast512_bf16_4096_nn.md (74.4 MB read + 12.4 MB written)
+    "bf16_8192_nn": 0.986e9,    # profiles/umma_gemm_2cta_512wide_bf16_8192_nn.md (0.866 GB read + 0.120 GB written)
+    "e4m3_8192_nt": 0.461e9,    # profiles/umma_gemm_2cta_e4m3_8192_nt.md (0.344 GB read + 0.117 GB written)
     "fp32_8192_nn": 3.553e9,    # profiles/sgemm_async_fp32_8192_nn.md (3.281 GB read + 0.272 GB written)
 }
 
