@@ -550,3 +550,40 @@ def test_umma_epilogue_warp_groups(variant, warps, tile_n, reset_tuning):
             dr = R.DeviceCase(cr)
             dr.run(variant)
             R.check_full(dr, what=f"{cr.name} warps={warps} tile_n={tile_n} split={split}")
+
+
+def test_two_host_threads_two_streams():
+    """Distinct streams from distinct host threads at the same time (the binding releases the GIL inside the
+    library): different shapes and kernel families, a k-split among them; every result must match the oracle."""
+    import threading
+    jobs = [mk(W.PEAK_BF16_BF16, 0, 0, 520, 776, 264, alpha=0.5, beta=2.0, case=1),
+            mk(W.PEAK_F16_F32, 1, 0, 96, 1032, 1544, alpha=1.0, beta=1.0, pad_a=0, case=2),      # k-split path
+            mk(W.PEAK_F32_F32, 0, 0, 256, 256, 128, alpha=-1.0, beta=0.5, case=3),               # SGEMM
+            mk(W.PEAK_BF16_F32, 0, 1, 1000, 264, 520, alpha=2.0, beta=0.0, case=4)]
+    cases = [R.DeviceCase(c) for c in jobs]
+    errors = []
+
+    def worker(idx):
+        try:
+            st = torch.cuda.Stream()
+            for rep in range(20):
+                for k in range(idx, len(cases), 2):
+                    dc = cases[k]
+                    dc.reset_c()
+                    st.wait_stream(torch.cuda.current_stream())     # the upload of C ran on the default stream
+                    c = dc.case
+                    P.peak_gemm(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta,
+                                dc.C, c.ldc, st)
+                    rc, detail = P.peak_check(st)
+                    assert rc == P.PEAK_OK, hex(detail)
+                    if rep == 19:
+                        R.check_full(dc, what=f"thread {idx} {c.name}")
+        except Exception as exc:                                     # reported by the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[0]
