@@ -377,15 +377,15 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // cap (sustained, random inputs): with 16-bit inputs and beta = 0 they win from 48 k-blocks on (+1..2 % at
     // 8192x8192x3072, +2 % at 8192x8192x4096, +5 % at 8192^3, +9 % at fp16 8192^3 TN), with beta != 0 (the epilogue also reads C)
     // only from 128 k-blocks on (-7 % at 16384x14336x4096, +3 % at 16384x4096x14336); 8-bit inputs, whose
-    // k-blocks take the same time but whose 256-wide tiles are less starved, from 128 k-blocks (K = 16384)
-    // on (+3 %).  They must fill the grid as well as the 256-wide tiles do (4096x8192x4096: 3.46 waves
+    // k-blocks take the same time but hold twice the K, from 96 k-blocks (K = 12288) on (a tie at 64 k-blocks,
+    // +2.6 % at 96, +3..5 % at 128).  They must fill the grid as well as the 256-wide tiles do (4096x8192x4096: 3.46 waves
     // against 6.9, -3 %).
     bool wide = false;
     if (whole256 && !tuning(PEAK_TUNE_TILE_N)) {
         const int bke = in8 ? 2 * BK : BK;
         const int64_t num_kb = (g.K + bke - 1) / bke;
         const bool light_tail = g.beta == 0.0f && g.act != PEAK_ACT_GELU;
-        const int64_t min_kb = (!in8 && light_tail) ? 48 : 128;
+        const int64_t min_kb = !light_tail ? 128 : (in8 ? 96 : 48);
         auto fill = [&](int64_t tiles) { return (double)tiles / (double)(((tiles + units - 1) / units) * units); };
         const int64_t t512 = tiles_of(g, 2, 512), t256 = tiles_of(g, 2, 256);
         wide = num_kb >= min_kb && t512 >= units && fill(t512) >= fill(t256) - 0.02;
