@@ -1,4 +1,5 @@
-// Tensor-core GEMM for 16-bit inputs on sm_100a: device code (kernel, epilogue, split-K reduction).
+// Tensor-core GEMM for 16-bit (and 8-bit float) inputs on sm_100a: device code (kernel, epilogue, split-K
+// reduction).
 //
 // One persistent CTA (or CTA pair) per SM walks work items -- output tiles, or (tile, k-slice) pairs when
 // K is split -- in a grouped order (the paper's block swizzle).  Inside a CTA three roles run concurrently
@@ -9,22 +10,27 @@
 //               warp tiling / tensor-core steps), two accumulator buffers so that the next tile's main
 //               loop overlaps this tile's epilogue,
 //   warps 2..5  epilogue: tcgen05.ld -> alpha/beta in fp32 -> one rounding -> swizzled shared-memory
-//               staging -> TMA store (coalesced, clipped at the matrix edge); a direct vector / scalar
-//               store path serves outputs whose base or pitch is not 16-byte aligned.
+//   (or 2..9)   staging -> TMA store (coalesced, clipped at the matrix edge); with beta != 0 old C comes in by
+//               TMA through the same buffers; a direct vector / scalar path serves outputs whose base or
+//               pitch is not 16-byte aligned.  Two-half tiles, and one-slot tiles of short launches, have a
+//               second group of four epilogue warps.
 // mbarriers connect the roles (full/empty per stage, full/empty per accumulator).  Every wait is bounded.
 //
 // Tile: 128 x BN x 64 per CTA (CTA_GROUP 1) or 256 x BN x 64 per CTA pair (CTA_GROUP 2: each CTA stages its
 // 128 rows of A and its BN/2-column half of B; the leader CTA issues MMAs for both).  BN is 128, 256, or --
 // CTA pairs only -- 512: a 256 x 512 tile is computed as two 256-column halves that occupy both accumulator
 // slots, so a quarter fewer operand bytes reach each SM per flop (what limits the sustained rate under the
-// power cap) at the price of an epilogue that overlaps the next main loop only half by half.
+// power cap) at the price of an epilogue that is exposed once per tile: the two halves are drained at the
+// same time by the two warp groups, and the last k-blocks of the tile are issued half by half so that half 0
+// reaches its warps early.
 //
 // Split-K (the paper's Split-K transformation, section 4.1).  The first `full_tiles` tiles are computed
 // whole; each remaining tile has its k-blocks divided among `tail_splits` work items that store fp32 partial
 // tiles to a workspace, and a second kernel adds a tile's slices in slice order and applies alpha/beta, so
 // the result does not depend on scheduling.  Two uses: shapes with too few tiles to fill the GPU split every
 // tile (full_tiles = 0); shapes whose tile count is not a multiple of the SM (pair) count split only the
-// tiles of the last, partly filled wave, so that the wave finishes in a fraction of a tile time.
+// tiles of the last, partly filled wave, so that the wave finishes in a fraction of a tile time (opt-in: it
+// measured no gain under the power cap).
 #pragma once
 #include <type_traits>
 #include <cuda.h>

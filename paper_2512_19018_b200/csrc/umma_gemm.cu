@@ -1,4 +1,5 @@
-// Tensor-core GEMM for 16-bit inputs on sm_100a: host side (plan, launch, workspace, entry points).
+// Tensor-core GEMM for 16-bit (and 8-bit float) inputs on sm_100a: host side (plan, dispatch rules, launch,
+// workspace, entry points).
 // The kernels are in umma_device.cuh.
 #include <cuda.h>
 
