@@ -41,7 +41,7 @@ def check_fused(dc, bias_h, act, what):
     c0 = R.c0_values(dc) if c.beta != 0 else 0.0
     sp = R.s_prime(c, S, c.alpha, c.beta, c0)
     tol = LIP[act] * (4 * max(c.K, 1) * 2.0 ** -24 * sp + 2.0 ** -22 * (0 if bias_h is None else np.abs(bias_h)[None, :])) \
-        + 2.0 ** -21 * np.abs(prebias) + 2 * R.U_OUT[c.out_type] * np.abs(ref) + 1e-37
+        + 2.0 ** -21 * np.abs(prebias) + 2 * R.U_OUT[c.out_type] * np.abs(ref) + R.SUB_OUT[c.out_type]
     got = W.to_float64(dc.result(), c.out_type)
     err = np.abs(got - ref)
     assert not np.isnan(got).any(), what
