@@ -693,7 +693,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // old C of the first two chunks is requested while the main loop still runs
                     constexpr int CC = 128 / (int)sizeof(TOut);
                     const int c0 = n0 + ((C_::HALVES == 2) ? hf * C_::SLOT_N : (SPLIT_COLS ? grp * W : 0));
-                    if (lane == 0) {
+                    // (a group whose columns start beyond N has no chunk in this tile: nothing to request, or the
+                    // barrier would be armed for a wait that never comes)
+                    if (lane == 0 && c0 < p.N) {
                         ptx::tma_store_wait_read<0>();  // the previous tile's stores have read the buffer(s)
                         cfetch_issue<TOut, BATCHED>(cf, my_stage, 0, &tmC, c0, row0, bz);
                         if (!cf.single && c0 + CC < p.N && CC < W) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, c0, row0, bz);

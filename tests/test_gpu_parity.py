@@ -587,3 +587,23 @@ def test_two_host_threads_two_streams():
     for t in threads:
         t.join()
     assert not errors, errors[0]
+
+
+@pytest.mark.parametrize("dtype", [W.PEAK_F16_F32, W.PEAK_BF16_BF16])
+@pytest.mark.parametrize("knobs", [{"tile": 512, "warps": 0, "mc": 1}, {"tile": 256, "warps": 2, "mc": 1},
+                                   {"tile": 512, "warps": 0, "mc": 2}, {"tile": 256, "warps": 2, "mc": 2}])
+def test_old_c_by_tma_with_a_group_that_has_no_columns(dtype, knobs, reset_tuning):
+    """beta != 0 on kernels with two groups of epilogue warps, several tiles per CTA, and a last tile column so
+    narrow that the second group's columns lie beyond N: that group must request nothing (a request without
+    its wait left a barrier armed and the next tile's wait ran out)."""
+    if knobs["mc"] == 2 and not P.peak_multicast_available():
+        pytest.skip("libpeak_gemm_mc.so is not present")
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, knobs["tile"])
+    P.peak_set_tuning(P.PEAK_TUNE_EPILOGUE_WARPS, knobs["warps"])
+    P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, knobs["mc"])
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 50)
+    for (M, N, K) in [(3840, 2056, 192), (4480, 1544, 128), (2944, 4992, 128)]:
+        c = mk(dtype, 0, 1, M, N, K, alpha=0.5, beta=2.0, case=N)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+        R.check_sampled(dc, tile_m=128, tile_n=128, budget_macs=2e7, what=f"{c.name} {knobs}")
