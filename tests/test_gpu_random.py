@@ -66,3 +66,40 @@ def test_random_cases_against_the_oracle(seed):
         for k in range(P.PEAK_TUNE_COUNT):
             P.peak_set_tuning(k, 0)
     assert done > 250
+
+
+def test_random_multi_wave_cases_sampled():
+    """The same idea at sizes of several tiles per CTA (ragged in every dimension, beta != 0 in half of the
+    cases, back-to-back launches), compared with the oracle on a sampled grid that touches every tile."""
+    rng = np.random.default_rng(21)
+    types = [W.PEAK_F16_F32, W.PEAK_BF16_BF16, W.PEAK_F16_F16, W.PEAK_BF16_F32, W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32]
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 200)       # a lost hand-over shows up quickly instead of after seconds
+    try:
+        for n in range(80):
+            dt = types[rng.integers(len(types))]
+            in8 = W.IN_TYPE[dt] in ("e4m3", "e5m2")
+            ta, tb = (0, 1) if in8 else (int(rng.integers(2)), int(rng.integers(2)))
+            M = int(rng.integers(1, 40)) * 128 + int(rng.choice([0, 0, 8, 56]))
+            N = int(rng.integers(1, 40)) * 128 + int(rng.choice([0, 0, 8, 72]))
+            K = int(rng.integers(1, 40)) * 64 + int(rng.choice([0, 0, 16, 40]))
+            unit = 16 if in8 else 8
+            c = W.GemmCase(f"m{n}", dt, bool(ta), bool(tb), M, N, K, float(rng.choice([1.0, 0.5])),
+                           float(rng.choice([0.0, 0.0, 1.0, 2.0])), "uniform", pad_a=(-(M if ta else K)) % unit,
+                           pad_b=(-(K if tb else N)) % unit, pad_c=int(rng.choice([0, 0, 8])), case=5000 + n)
+            knobs = {P.PEAK_TUNE_TILE_N: int(rng.choice([0, 0, 0, 256, 512])),
+                     P.PEAK_TUNE_EPILOGUE: int(rng.choice([0, 0, 0, 1, 3])),
+                     P.PEAK_TUNE_EPILOGUE_WARPS: int(rng.choice([0, 0, 1, 2])),
+                     P.PEAK_TUNE_MULTICAST: int(rng.choice([0, 0, 1, 2])),
+                     P.PEAK_TUNE_RASTER_GROUP: int(rng.choice([0, 0, 2, 16])),
+                     P.PEAK_TUNE_BALANCED_GRID: int(rng.choice([0, 1])),
+                     P.PEAK_TUNE_DEPENDENT_LAUNCH: int(rng.choice([0, 0, 1]))}
+            for k, v in knobs.items():
+                P.peak_set_tuning(k, v)
+            dc = R.DeviceCase(c)
+            for _ in range(2):
+                dc.reset_c()
+                dc.run(P.PEAK_VARIANT_AUTO)
+            R.check_sampled(dc, tile_m=128, tile_n=128, budget_macs=2e7, what=f"{c} knobs={knobs}")
+    finally:
+        for k in range(P.PEAK_TUNE_COUNT):
+            P.peak_set_tuning(k, 0)
