@@ -607,3 +607,31 @@ def test_old_c_by_tma_with_a_group_that_has_no_columns(dtype, knobs, reset_tunin
         dc = R.DeviceCase(c)
         dc.run(P.PEAK_VARIANT_UMMA_2CTA)
         R.check_sampled(dc, tile_m=128, tile_n=128, budget_macs=2e7, what=f"{c.name} {knobs}")
+
+
+def test_cuda_graph_with_k_split_and_several_calls():
+    """A captured sequence: a k-split problem (pooled workspace allocated and freed inside the capture, reduce
+    kernel launched as a programmatic dependent), a beta != 0 problem and a wide-tile problem, replayed twice."""
+    cases = [mk(W.PEAK_BF16_BF16, 1, 0, 16, 1024, 2048, alpha=0.5, beta=2.0, case=1),        # split-K
+             mk(W.PEAK_F16_F32, 0, 1, 520, 776, 264, alpha=1.0, beta=1.0, case=2),
+             mk(W.PEAK_BF16_BF16, 0, 0, 512, 1024, 4096, case=3)]
+    dcs = [R.DeviceCase(c) for c in cases]
+    stream = torch.cuda.Stream()
+    for dc in dcs:
+        dc.run(stream=None)                                    # first-use set-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for dc in dcs:
+                c = dc.case
+                P.peak_gemm(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta,
+                            dc.C, c.ldc, stream)
+    for rep in range(2):
+        for dc in dcs:                                          # restore C0 in place (the graph holds the pointers)
+            dc.Cfull.copy_(R.to_device(dc.Cfull_h, dc.case.out_type))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert P.peak_check()[0] == P.PEAK_OK
+        for dc in dcs:
+            R.check_full(dc, what=f"graph replay {rep} {dc.case.name}")
