@@ -192,4 +192,11 @@ def check_sampled(dc: DeviceCase, tile_m=128, tile_n=256, what="", budget_macs=1
     ref, S = dc.oracle_sub(rows, cols)
     got = dc.result()[np.ix_(rows, cols)]
     c0 = c0_values(dc, rows, cols) if c.beta != 0 else 0.0
-    return check_values(c, got, ref, S, c0, what=what or c.name)
+    worst = check_values(c, got, ref, S, c0, what=what or c.name)
+    # scattered single elements off the grid (the listed-points entry point: one k-loop per element)
+    rng = np.random.default_rng(c.seed + 4242)
+    n_pts = int(min(512, max(16, 2e8 // max(c.K, 1))))
+    si, sj = rng.integers(0, c.M, n_pts), rng.integers(0, c.N, n_pts)
+    ref_p, S_p = dc.oracle_points(si, sj)
+    c0_p = c0_values(dc)[si, sj] if c.beta != 0 else 0.0
+    return max(worst, check_values(c, dc.result()[si, sj], ref_p, S_p, c0_p, what=(what or c.name) + " (points)"))

@@ -290,6 +290,48 @@ def test_layout_consistency_and_entry_points_agree(oracle):
     assert np.array_equal(rp.reshape(rs.shape), rs) and np.array_equal(sp.reshape(ss.shape), ss)
 
 
+@pytest.mark.parametrize("t", ["bf16", "f16", "f32"])
+@pytest.mark.parametrize("ta,tb", [(1, 0), (0, 1), (0, 0), (1, 1)])
+def test_indexed_entry_points_with_old_c(oracle, t, ta, tb):
+    """The sub-grid and listed-point entry points with beta != 0: their gather of old C (padded pitch, stored
+    output type) must give the full-matrix result bit for bit, and agree with numpy's float64
+    alpha * (op(A) @ op(B)) + beta * C0 at the same places -- a wrong row/column index, a missing pitch or a
+    dropped beta term in the indexed paths fails here.  Small-integer inputs make the second check exact."""
+    M, N, K = 37, 53, 41
+    rng = np.random.default_rng(77 + 2 * ta + tb)
+    rows = np.array([36, 0, 5, 5, 20, 1])          # unsorted, with a repeat
+    cols = np.array([52, 3, 0, 17, 51, 3, 30])
+    for dist, (alpha, beta) in [("uniform", (0.5, 2.0)), ("uniform", (1.0, 1.0)), ("smallint", (2.0, -3.0))]:
+        c = _case(t, ta, tb, M, N, K, dist=dist, pad_a=3, pad_b=1, pad_c=5, alpha=alpha, beta=beta,
+                  case=int(rng.integers(1 << 20)))
+        A, B, C0 = W.make_inputs(c)
+        assert c.ldc == N + 5 and C0.shape == (M, N + 5)
+        full, Sfull = _run(oracle, c, A, B, C0)
+        a = W.to_float64(A[:, :c.a_shape[1]], c.in_type)
+        b = W.to_float64(B[:, :c.b_shape[1]], c.in_type)
+        c0 = W.to_float64(C0[:, :N], c.out_type)
+        opA, opB = (a.T if ta else a), (b.T if tb else b)
+        want = (alpha * (opA @ opB) + beta * c0)[np.ix_(rows, cols)]
+        scale = (abs(alpha) * (np.abs(opA) @ np.abs(opB)) + np.abs(beta * c0))[np.ix_(rows, cols)]
+        rs, ss = oracle.gemm_submatrix(T[c.in_type], T[c.out_type], ta, tb, M, N, K, alpha, A, c.lda, B,
+                                       c.ldb, beta, C0, c.ldc, rows, cols)
+        assert np.array_equal(rs, full[np.ix_(rows, cols)]) and np.array_equal(ss, Sfull[np.ix_(rows, cols)])
+        ii, jj = np.meshgrid(rows, cols, indexing="ij")
+        rp, sp = oracle.gemm_points(T[c.in_type], T[c.out_type], ta, tb, M, N, K, alpha, A, c.lda, B, c.ldb, beta, C0, c.ldc,
+                                    ii.ravel(), jj.ravel())
+        assert np.array_equal(rp.reshape(rs.shape), rs) and np.array_equal(sp.reshape(ss.shape), ss)
+        if dist == "smallint":
+            assert np.array_equal(rs, want)
+        else:
+            assert np.all(np.abs(rs - want) <= 1e-13 * scale + 1e-300)
+        # beta really enters: dropping the old-C term would change the answer
+        r0, _ = oracle.gemm_submatrix(T[c.in_type], T[c.out_type], ta, tb, M, N, K, alpha, A, c.lda, B, c.ldb, 0.0,
+                                      None, c.ldc, rows, cols)
+        if dist == "smallint":
+            assert np.array_equal(rs - r0, beta * c0[np.ix_(rows, cols)])
+        assert not np.array_equal(rs, r0)
+
+
 def test_rectangular_not_transposed(oracle):
     """A deliberately asymmetric case: mixing up M/N, or transposing an operand, changes the answer."""
     M, N, K = 3, 5, 2
