@@ -239,6 +239,11 @@ int peak_tile_coord(int64_t tile, int64_t tiles_m, int64_t tiles_n, int64_t grou
  * peak_check: synchronises `stream`, then reads and clears the device status word that kernels set
  * when a bounded wait (on an mbarrier) gives up.  Returns PEAK_OK, PEAK_ERR_TIMEOUT or PEAK_ERR_CUDA.
  * `detail`, if not NULL, receives the raw status word (role and barrier that gave up).
+ * There is ONE status word per device, not one per stream: a wait that gave up in a kernel on any stream of
+ * the current device is reported to whichever caller checks first, and the read clears it.  A process that
+ * runs GEMMs on several streams and wants to attribute a timeout should check after each stream's work, or
+ * treat a report as "some call on this device since the last check".  (The paper's validators, section 3.3,
+ * check results after a run; this is the run-time half: a stuck pipeline is reported, never a hang.)
  */
 int peak_check(void *stream, uint32_t *detail);
 
@@ -284,6 +289,24 @@ int64_t peak_kernel_launches(void);
 
 /* The cudaError_t of the most recent failing CUDA call made by this thread's last entry-point call. */
 int peak_last_cuda_error(void);
+
+/*
+ * peak_last_kernel: which kernel this host thread's most recent GEMM call launched, and with which launch
+ * configuration, as text: the kernel's name with its template arguments, written the way profilers print
+ * it, followed by key=value pairs (grid, work items, k-slices, ...).  The paper's performance evaluator
+ * (section 3.3) records which candidate produced a measurement; this is that record for a dispatcher that
+ * chooses among kernels by shape.  `buf` (host) receives at most len - 1 characters and a terminator; the
+ * text is empty before the first launch.  Returns PEAK_OK, or PEAK_ERR_INVALID_VALUE for a null buffer.
+ */
+int peak_last_kernel(char *buf, size_t len);
+
+/*
+ * peak_selftest_per_device_once: host-only self-check of the library's once-per-device bookkeeping (a
+ * kernel's shared-memory attribute and similar context state are set the first time EACH device runs a
+ * kernel, not once per process).  Touches no device.  Returns 0, or the number of the failed check.  (No
+ * counterpart in the paper: test support.)
+ */
+int peak_selftest_per_device_once(void);
 
 const char *peak_status_string(int status);
 const char *peak_variant_string(int variant);

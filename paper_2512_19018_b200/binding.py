@@ -24,7 +24,7 @@ _lib = None
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
            "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available", "peak_gemm_fused",
-           "peak_gemm_fused_variant", "peak_gemm_strided_batched"]
+           "peak_gemm_fused_variant", "peak_gemm_strided_batched", "peak_last_kernel", "peak_selftest_per_device_once"]
 
 
 class PeakError(RuntimeError):
@@ -83,6 +83,10 @@ def load():
     lib.peak_kernel_launches.argtypes = []
     lib.peak_last_cuda_error.restype = i
     lib.peak_last_cuda_error.argtypes = []
+    lib.peak_last_kernel.restype = i
+    lib.peak_last_kernel.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
+    lib.peak_selftest_per_device_once.restype = i
+    lib.peak_selftest_per_device_once.argtypes = []
     lib.peak_status_string.restype = ctypes.c_char_p
     lib.peak_status_string.argtypes = [i]
     lib.peak_variant_string.restype = ctypes.c_char_p
@@ -231,6 +235,17 @@ def peak_kernel_launches() -> int:
 
 def peak_last_cuda_error() -> int:
     return load().peak_last_cuda_error()
+
+
+def peak_last_kernel() -> str:
+    """Name and launch configuration of the kernel this thread's last GEMM call launched."""
+    buf = ctypes.create_string_buffer(256)
+    _raise(load().peak_last_kernel(buf, 256), "peak_last_kernel")
+    return buf.value.decode()
+
+
+def peak_selftest_per_device_once() -> int:
+    return load().peak_selftest_per_device_once()
 
 
 def peak_status_string(status: int) -> str:

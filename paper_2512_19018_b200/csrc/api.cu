@@ -2,6 +2,9 @@
 // small amount of process state (launch counter, last CUDA error, per-device status word, staging buffers).
 #include <atomic>
 #include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -16,7 +19,6 @@ thread_local int t_last_cuda_error = 0;
 // a code into it when a bounded wait gives up; peak_check() reads and clears it.
 __device__ uint32_t g_status_word[4];
 
-constexpr int kMaxDevices = 64;
 uint32_t *g_status_ptr[kMaxDevices] = {};
 std::mutex g_status_mutex;
 }  // namespace
@@ -27,6 +29,15 @@ std::atomic<int> g_tuning[PEAK_TUNE_COUNT_];
 int tuning(int key) { return (key >= 0 && key < PEAK_TUNE_COUNT_) ? g_tuning[key].load(std::memory_order_relaxed) : 0; }
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+namespace {
+thread_local char t_last_kernel[256] = "";
+}
+void note_kernel(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_last_kernel, sizeof(t_last_kernel), fmt, ap);
+    va_end(ap);
+}
 void set_cuda_error(cudaError_t e) { t_last_cuda_error = (int)e; }
 
 uint32_t *device_status_word() {
@@ -138,7 +149,7 @@ struct Staging {
     size_t bytes = 0;
     int device = -1;  // the device the buffer lives on
 };
-Staging g_stage[3];
+Staging g_stage_of[kMaxDevices][3];  // per device: a process may call from several GPUs in turn
 
 // Streams and events of the host-buffer entry point's copy / compute pipeline (created on first use, for the
 // device that is current then; guarded by g_stage_mutex like the staging buffers).
@@ -148,7 +159,7 @@ struct HostPipeline {
     cudaEvent_t start = nullptr, out_done = nullptr, in_done[kHostPanels] = {}, mm_done[kHostPanels] = {};
     int device = -1;
 };
-HostPipeline g_pipe;
+HostPipeline g_pipe_of[kMaxDevices];
 std::mutex g_stage_mutex;
 
 int ensure(Staging &s, size_t need) {
@@ -165,7 +176,7 @@ int ensure(Staging &s, size_t need) {
     return PEAK_OK;
 }
 
-void release_pipeline() {
+void release_pipeline(HostPipeline &g_pipe) {
     if (g_pipe.in) cudaStreamDestroy(g_pipe.in);
     if (g_pipe.out) cudaStreamDestroy(g_pipe.out);
     if (g_pipe.start) cudaEventDestroy(g_pipe.start);
@@ -177,12 +188,10 @@ void release_pipeline() {
     g_pipe = HostPipeline{};
 }
 
-int ensure_pipeline() {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+int ensure_pipeline(HostPipeline &g_pipe, int dev) {
+    cudaError_t e = cudaSuccess;
     if (g_pipe.in && g_pipe.device == dev) return PEAK_OK;
-    release_pipeline();
+    release_pipeline(g_pipe);
     e = cudaStreamCreateWithFlags(&g_pipe.in, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&g_pipe.out, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_pipe.start, cudaEventDisableTiming);
@@ -191,7 +200,7 @@ int ensure_pipeline() {
         e = cudaEventCreateWithFlags(&g_pipe.in_done[i], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_pipe.mm_done[i], cudaEventDisableTiming);
     }
-    if (e != cudaSuccess) { set_cuda_error(e); release_pipeline(); return PEAK_ERR_CUDA; }
+    if (e != cudaSuccess) { set_cuda_error(e); release_pipeline(g_pipe); return PEAK_ERR_CUDA; }
     g_pipe.device = dev;
     return PEAK_OK;
 }
@@ -280,7 +289,11 @@ int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int6
     const size_t b_bytes = need_ab ? span_bytes(transB ? N : K, transB ? K : N, ldb, ib) : 0;
     const size_t c_bytes = span_bytes(M, N, ldc, ob);
     cudaStream_t st = (cudaStream_t)stream;
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return PEAK_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_stage_mutex);
+    Staging *g_stage = g_stage_of[dev];
+    HostPipeline &g_pipe = g_pipe_of[dev];
     if ((rc = ensure(g_stage[0], a_bytes)) || (rc = ensure(g_stage[1], b_bytes)) || (rc = ensure(g_stage[2], c_bytes)))
         return rc;
     // C travels to the device when its old values are needed, or when the pitch leaves gaps that the
@@ -297,27 +310,33 @@ int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int6
     // multiply panel i.  Copies in run on one internal stream (B first, then the panels in order), the
     // products on the caller's stream, copies out on a second internal stream; events order them.
     const int64_t panels = need_ab ? std::max<int64_t>(1, std::min<int64_t>(kHostPanels, M / 512)) : 1;
-    if (panels > 1 && (rc = ensure_pipeline()) != PEAK_OK) return rc;
+    if (panels > 1 && (rc = ensure_pipeline(g_pipe, dev)) != PEAK_OK) return rc;
     if (panels == 1) {
         if (a_bytes) e = cudaMemcpyAsync(dA, A, a_bytes, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess && b_bytes) e = cudaMemcpyAsync(dB, B, b_bytes, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess && c_in) e = cudaMemcpyAsync(dC, C, c_bytes, cudaMemcpyHostToDevice, st);
+        // on any error the stream is still drained, so that no copy uses the caller's buffers after the return
+        if (e == cudaSuccess)
+            rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, dA, lda, dB, ldb, beta, dC, ldc, stream);
+        const int rc_cuda = peak_last_cuda_error();
+        if (e == cudaSuccess && rc == PEAK_OK) e = cudaMemcpyAsync(C, dC, c_bytes, cudaMemcpyDeviceToHost, st);
+        const cudaError_t es = cudaStreamSynchronize(st);
+        if (rc != PEAK_OK) { t_last_cuda_error = rc_cuda; return rc; }
         if (e != cudaSuccess) return fail(e);
-        rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, dA, lda, dB, ldb, beta, dC, ldc, stream);
-        if (rc != PEAK_OK) return rc;
-        e = cudaMemcpyAsync(C, dC, c_bytes, cudaMemcpyDeviceToHost, st);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-        if (e != cudaSuccess) return fail(e);
+        if (es != cudaSuccess) return fail(es);
         return PEAK_OK;
     }
     cudaStream_t s_in = g_pipe.in, s_out = g_pipe.out;
     // the internal streams start after whatever the caller's stream already holds
+    // Nothing is in flight on the internal streams yet, so a failure here may return at once; from the first
+    // copy on, every failure leaves the loop into the common tail below, which drains all three streams.
     if ((e = cudaEventRecord(g_pipe.start, st)) != cudaSuccess) return fail(e);
     if ((e = cudaStreamWaitEvent(s_in, g_pipe.start, 0)) != cudaSuccess) return fail(e);
     if ((e = cudaStreamWaitEvent(s_out, g_pipe.start, 0)) != cudaSuccess) return fail(e);
-    if ((e = cudaMemcpyAsync(dB, B, b_bytes, cudaMemcpyHostToDevice, s_in)) != cudaSuccess) return fail(e);
+    e = cudaMemcpyAsync(dB, B, b_bytes, cudaMemcpyHostToDevice, s_in);
     const int64_t rows_per = ((M + panels - 1) / panels + 127) / 128 * 128;  // whole 128-row tiles per panel
-    for (int64_t i = 0; i < panels; ++i) {
+    int rc_cuda = 0;
+    for (int64_t i = 0; i < panels && e == cudaSuccess; ++i) {
         const int64_t m0 = i * rows_per, mp = std::min(rows_per, M - m0);
         if (mp <= 0) break;
         const size_t c_off = (size_t)m0 * (size_t)ldc * (size_t)ob;
@@ -333,23 +352,25 @@ int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int6
         if (e == cudaSuccess && c_in) e = cudaMemcpyAsync(dC + c_off, hC + c_off, c_len, cudaMemcpyHostToDevice, s_in);
         if (e == cudaSuccess) e = cudaEventRecord(g_pipe.in_done[i], s_in);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(st, g_pipe.in_done[i], 0);
-        if (e != cudaSuccess) return fail(e);
+        if (e != cudaSuccess) break;
         const char *a_panel = transA ? dA + (size_t)m0 * ib : dA + (size_t)m0 * (size_t)lda * ib;
         rc = gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, mp, N, K, alpha, a_panel, lda, dB, ldb, beta, dC + c_off,
                        ldc, stream);
-        if (rc != PEAK_OK) break;
-        if ((e = cudaEventRecord(g_pipe.mm_done[i], st)) != cudaSuccess) return fail(e);
-        if ((e = cudaStreamWaitEvent(s_out, g_pipe.mm_done[i], 0)) != cudaSuccess) return fail(e);
-        if ((e = cudaMemcpyAsync(hC + c_off, dC + c_off, c_len, cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
-            return fail(e);
+        if (rc != PEAK_OK) { rc_cuda = peak_last_cuda_error(); break; }
+        if ((e = cudaEventRecord(g_pipe.mm_done[i], st)) != cudaSuccess) break;
+        if ((e = cudaStreamWaitEvent(s_out, g_pipe.mm_done[i], 0)) != cudaSuccess) break;
+        e = cudaMemcpyAsync(hC + c_off, dC + c_off, c_len, cudaMemcpyDeviceToHost, s_out);
     }
-    // everything rejoins the caller's stream, which is then drained (also when a panel's product was refused, so
-    // that no copy is still in flight when the caller gets its buffers back)
+    // everything rejoins the caller's stream, and all three streams are drained -- also after a refused product
+    // or a failed CUDA call, so that no copy is still in flight when the caller gets its buffers back
     cudaError_t e1 = cudaEventRecord(g_pipe.out_done, s_out);
     if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(st, g_pipe.out_done, 0);
     cudaError_t e2 = cudaStreamSynchronize(s_in);
+    cudaError_t e4 = cudaStreamSynchronize(s_out);
     cudaError_t e3 = cudaStreamSynchronize(st);
-    if (rc != PEAK_OK) return rc;
+    if (rc != PEAK_OK) { t_last_cuda_error = rc_cuda; return rc; }
+    if (e != cudaSuccess) return fail(e);
+    if (e4 != cudaSuccess) return fail(e4);
     if (e1 != cudaSuccess) return fail(e1);
     if (e2 != cudaSuccess) return fail(e2);
     if (e3 != cudaSuccess) return fail(e3);
@@ -358,12 +379,21 @@ int peak_gemm_host(int dtype, int transA, int transB, int64_t M, int64_t N, int6
 
 int peak_release_staging(void) {
     std::lock_guard<std::mutex> lock(g_stage_mutex);
-    for (auto &s : g_stage) {
-        if (s.ptr) cudaFree(s.ptr);
-        s.ptr = nullptr;
-        s.bytes = 0;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    for (int dev = 0; dev < kMaxDevices; ++dev) {
+        bool any = g_pipe_of[dev].in != nullptr;
+        for (auto &s : g_stage_of[dev]) any = any || s.ptr != nullptr;
+        if (!any) continue;
+        cudaSetDevice(dev);  // buffers, streams and events are released with their own device current
+        for (auto &s : g_stage_of[dev]) {
+            if (s.ptr) cudaFree(s.ptr);
+            s.ptr = nullptr;
+            s.bytes = 0;
+        }
+        release_pipeline(g_pipe_of[dev]);
     }
-    release_pipeline();
+    if (prev >= 0) cudaSetDevice(prev);
     return PEAK_OK;
 }
 
@@ -424,6 +454,30 @@ int peak_multicast_available(void) { return umma_multicast_available() ? 1 : 0; 
 int64_t peak_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int peak_last_cuda_error(void) { return t_last_cuda_error; }
+
+int peak_last_kernel(char *buf, size_t len) {
+    if (!buf || len == 0) return PEAK_ERR_INVALID_VALUE;
+    strncpy(buf, t_last_kernel, len - 1);
+    buf[len - 1] = '\0';
+    return PEAK_OK;
+}
+
+int peak_selftest_per_device_once(void) {
+    // host-only check of the once-per-device bookkeeping behind the kernels' context set-up
+    PerDeviceOnce once;
+    int calls[4] = {0, 0, 0, 0};
+    auto run = [&](int dev, cudaError_t result) {
+        return once.run(dev, [&] { ++calls[dev < 0 || dev > 2 ? 3 : dev]; return result; });
+    };
+    if (run(0, cudaSuccess) != cudaSuccess || run(0, cudaErrorUnknown) != cudaSuccess || calls[0] != 1) return 1;
+    if (run(1, cudaErrorInvalidValue) != cudaErrorInvalidValue || calls[1] != 1) return 2;  // device 1 set up itself
+    if (run(1, cudaSuccess) != cudaErrorInvalidValue || calls[1] != 1) return 3;            // and its result is kept
+    if (run(2, cudaSuccess) != cudaSuccess || calls[2] != 1 || calls[0] != 1) return 4;
+    if (run(kMaxDevices - 1, cudaSuccess) != cudaSuccess) return 5;
+    run(-1, cudaSuccess); run(-1, cudaSuccess); run(kMaxDevices, cudaSuccess);  // outside the table: no memory
+    if (calls[3] != 4) return 6;
+    return 0;
+}
 
 const char *peak_status_string(int status) {
     switch (status) {

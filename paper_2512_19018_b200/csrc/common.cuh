@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/peak_gemm.h"
 
 namespace peak {
@@ -61,6 +63,9 @@ __device__ __forceinline__ float finish_f32(float x, const float *bias, int64_t 
 
 // ---- host-side bookkeeping (api.cu owns the definitions) ---------------------------------------
 void count_launch(int n = 1);
+// Remembers, for this host thread, which kernel the entry point launched last and how (printf-style; the
+// kernel's name is written the way profilers print it); read back through peak_last_kernel().
+void note_kernel(const char *fmt, ...);
 void set_cuda_error(cudaError_t e);
 uint32_t *device_status_word();  // address of the per-device status word (nullptr on failure)
 int tuning(int key);             // value set through peak_set_tuning (0 = library default)
@@ -79,6 +84,32 @@ struct GemmArgs {
     int64_t strideA, strideB, strideC;  // elements between consecutive matrices of the batch
     int64_t nbatch() const { return batch > 1 ? batch : 1; }
 };
+
+// One-time set-up that belongs to a device's context rather than to the process (a kernel's
+// cudaFuncAttributeMaxDynamicSharedMemorySize, an occupancy query): done the first time each device runs the
+// code, with that device current, and remembered per device.  A process that drives several GPUs therefore
+// gets every one of them set up, not just the first.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    std::mutex m;
+    bool done[kMaxDevices] = {};
+    cudaError_t err[kMaxDevices] = {};
+    // Runs fn() once for device `dev` (its later callers get the remembered result).  A device index outside
+    // the table is served without memory: fn() runs every time.
+    template <typename Fn> cudaError_t run(int dev, Fn fn) {
+        if (dev < 0 || dev >= kMaxDevices) return fn();
+        std::lock_guard<std::mutex> lock(m);
+        if (!done[dev]) {
+            err[dev] = fn();
+            done[dev] = true;
+        }
+        return err[dev];
+    }
+};
+inline int current_device() {
+    int dev = 0;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
 
 // kernel-family launchers; each returns a peak_status_t
 int launch_fallback(const GemmArgs &g);

@@ -114,6 +114,7 @@ template <typename TIn, typename TOut> int run_fallback(const GemmArgs &g) {
         g.transA, g.transB, g.M, g.N, g.K, g.alpha, (const TIn *)g.A, g.lda, (const TIn *)g.B, g.ldb, g.beta,
         (TOut *)g.C, g.ldc, g.bias, g.act);
     count_launch();
+    note_kernel("fallback_gemm_kernel grid=%ux%u", grid.x, grid.y);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
@@ -139,6 +140,7 @@ template <typename TOut> int run_scale(const GemmArgs &g) {
     if (blocks > 148 * 16) blocks = 148 * 16;
     scale_kernel<TOut><<<(unsigned)blocks, 256, 0, g.stream>>>(g.M, g.N, g.beta, (TOut *)g.C, g.ldc, g.bias, g.act);
     count_launch();
+    note_kernel("scale_kernel grid=%u", (unsigned)blocks);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;

@@ -1,6 +1,12 @@
 // Interface between the main library and its optional single-GPU accelerator plug-in
 // (libpeak_gemm_mc.so): the tensor-core GEMM run by clusters of four CTAs that share B tiles.
 // Plain C structs and one entry point, so that the two shared objects need nothing else from each other.
+//
+// Contract: the plug-in is for single-GPU processes.  Its tensor maps must cover memory of the GPU it runs on
+// and nothing else; the entry point verifies that A and B are ordinary device allocations of the current
+// device (first and last byte of each) and answers PEAK_ERR_UNSUPPORTED otherwise, in which case the main
+// library runs its own kernel.  Multi-rank jobs switch the plug-in off (PEAK_TUNE_MULTICAST = 1) and do not
+// ship it.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>

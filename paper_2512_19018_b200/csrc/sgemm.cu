@@ -272,7 +272,10 @@ sgemm_async_kernel(int M, int N, int K, float alpha, const float *__restrict__ A
 
 template <bool TA, bool TB, bool PACKED> int run_sgemm_async(const GemmArgs &g) {
     auto kernel = sgemm_async_kernel<TA, TB, PACKED>;
-    static cudaError_t attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SA_SMEM_BYTES);
+    static PerDeviceOnce attr_once;  // once per device, not per process
+    const cudaError_t attr_err = attr_once.run(current_device(), [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SA_SMEM_BYTES);
+    });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err); return PEAK_ERR_CUDA; }
     const int tiles_m = (int)(g.M / SG_BM), tiles_n = (int)(g.N / SG_BN);
     const int group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 8;
@@ -280,6 +283,7 @@ template <bool TA, bool TB, bool PACKED> int run_sgemm_async(const GemmArgs &g) 
         (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
         (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
     count_launch();
+    note_kernel("sgemm_async_kernel<%d, %d, %d> grid=%d", (int)TA, (int)TB, (int)PACKED, tiles_m * tiles_n);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
@@ -302,6 +306,8 @@ template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
             (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
             (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
     count_launch();
+    note_kernel("sgemm_kernel<%d, %d, %d> grid=%d", (int)TA, (int)TB, (int)(tuning(PEAK_TUNE_SGEMM_FMA) != 1),
+                tiles_m * tiles_n);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;

@@ -110,10 +110,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     using C_ = Cfg<CG, BN>;
     constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block
     auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8, G2>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+    static PerDeviceOnce attr_once;  // the attribute belongs to the device's context: once per device
+    const cudaError_t attr_err = attr_once.run(current_device(), [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err); return PEAK_ERR_CUDA; }
 
@@ -201,6 +200,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, tmW, ws, p);
     count_launch();
+    note_kernel("umma_gemm_kernel<%d, %d, %s, 0, %d, %d, %d> grid=%d items=%d splits=%d", CG, BN,
+                sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"),
+                (int)BATCHED, (int)IN8, (int)G2, units * CG, p.total_items, plan.tail_splits);
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     if (plan.full_tiles == tiles) return PEAK_OK;
 
@@ -415,7 +417,13 @@ int launch_umma(const GemmArgs &g, int cta_group) {
                               tuning(PEAK_TUNE_EPILOGUE_WARPS), mc_tile_n, 0};
             if (!r.status) return PEAK_ERR_CUDA;
             const int rc = mc_entry()(&r);
-            if (rc == PEAK_OK) { count_launch(); return rc; }
+            if (rc == PEAK_OK) {
+                count_launch();
+                const Elem eo = out_elem(g.dtype);
+                note_kernel("umma_gemm_kernel<2, %d, %s, 1, 0, %d, *> (cluster-multicast plug-in)", mc_tile_n,
+                            eo == Elem::F32 ? "float" : (eo == Elem::F16 ? "__half" : "__nv_bfloat16"), (int)in8);
+                return rc;
+            }
             if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
             if (rc != PEAK_ERR_UNSUPPORTED) return rc;
         }

@@ -45,6 +45,7 @@ template <> struct McOps<1> {
 
 // The plug-in does not use the main library's bookkeeping; these satisfy common.cuh's declarations.
 void count_launch(int) {}
+void note_kernel(const char *, ...) {}
 void set_cuda_error(cudaError_t) {}
 uint32_t *device_status_word() { return nullptr; }
 int tuning(int) { return 0; }
@@ -52,12 +53,23 @@ int tuning(int) { return 0; }
 namespace {
 using namespace umma;
 
+// True when `p` lies in an ordinary device allocation (cudaMalloc, a memory pool) of the CURRENT device.
+bool local_device_memory(const void *p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice && at.device == current_device();
+}
+
 template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(peak_mc_request *r) {
     constexpr int CG = 2;
     constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block (8-bit inputs: 128 per 128-byte row)
     using C_ = Cfg<CG, BN>;
     auto kernel = umma_gemm_kernel<CG, BN, TOut, 1, false, IN8, G2>;
-    static cudaError_t attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+    const int dev = current_device();
+    static PerDeviceOnce attr_once;  // once per device, not per process
+    const cudaError_t attr_err = attr_once.run(dev, [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+    });
     if (attr_err != cudaSuccess) { r->cuda_error = (int)attr_err; return PEAK_ERR_CUDA; }
 
     const Elem ein = in_elem(r->dtype), eout = out_elem(r->dtype);
@@ -106,13 +118,18 @@ template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     // how many 4-CTA clusters the device can hold at once (GPC boundaries may leave some SMs out)
-    static int max_clusters = 0;
-    if (max_clusters == 0) {
+    static PerDeviceOnce occ_once;
+    static int max_clusters_of[kMaxDevices] = {};
+    int queried = 0;
+    occ_once.run(dev, [&] {
         cfg.gridDim = dim3(4 * 37);
         int n = 0;
         cudaError_t oe = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
-        max_clusters = (oe == cudaSuccess && n > 0) ? n : 32;
-    }
+        queried = (oe == cudaSuccess && n > 0) ? n : 32;
+        if (dev >= 0 && dev < kMaxDevices) max_clusters_of[dev] = queried;
+        return cudaSuccess;
+    });
+    const int max_clusters = (dev >= 0 && dev < kMaxDevices) ? max_clusters_of[dev] : queried;
     int clusters = max_clusters < tiles ? max_clusters : tiles;
     if (r->balanced_grid != 1) {  // the fewest clusters that finish in the same number of waves
         const int waves = (tiles + clusters - 1) / clusters;
@@ -135,6 +152,18 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
     if (!r) return PEAK_ERR_INVALID_VALUE;
     r->cuda_error = 0;
     if (in_elem(r->dtype) == Elem::F32 || r->M < 1 || r->N < 1 || r->K < 1) return PEAK_ERR_UNSUPPORTED;
+    // The multicast loads below may only ever read this GPU's own memory: both operands must be plain device
+    // allocations of the current device over their whole extent (first and last byte are looked up); a peer
+    // GPU's buffer, managed or host memory sends the caller back to its own kernel.
+    {
+        const int ib = elem_bytes(in_elem(r->dtype));
+        const int64_t a_rows = r->transA ? r->K : r->M, a_cols = r->transA ? r->M : r->K;
+        const int64_t b_rows = r->transB ? r->N : r->K, b_cols = r->transB ? r->K : r->N;
+        const char *a0 = static_cast<const char *>(r->A), *b0 = static_cast<const char *>(r->B);
+        if (!local_device_memory(a0) || !local_device_memory(a0 + ((a_rows - 1) * r->lda + a_cols) * ib - 1) ||
+            !local_device_memory(b0) || !local_device_memory(b0 + ((b_rows - 1) * r->ldb + b_cols) * ib - 1))
+            return PEAK_ERR_UNSUPPORTED;
+    }
     // two groups of epilogue warps when the launch is at most two waves of 512 x 256 super-tiles long (the
     // last tile's epilogue is then a visible part of the run time)
     const int64_t super_tiles = ((r->M + 511) / 512) * ((r->N + 255) / 256);

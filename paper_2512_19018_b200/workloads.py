@@ -255,11 +255,14 @@ def bench_workload() -> GemmCase:
     return config1()
 
 
-def fp8_workload(n: int, in_type: str = "e4m3") -> GemmCase:
-    """8-bit float inputs, bf16 output, n^3, K-major operands (A row-major, B stored N x K): uniform[-1, 1]
-    values so that the operands use the formats' range (normal / sqrt(K) would fall into the subnormals)."""
+def fp8_workload(n: int, in_type: str = "e4m3", layout: str = "NT") -> GemmCase:
+    """8-bit float inputs, bf16 output, n^3 (default NT: A row-major, B stored N x K, both with K innermost):
+    uniform[-1, 1] values so that the operands use the formats' range (normal / sqrt(K) would fall into the
+    subnormals)."""
     dt = PEAK_E4M3_BF16 if in_type == "e4m3" else PEAK_E5M2_BF16
-    return GemmCase(f"{in_type}_{n}_nt", dt, False, True, n, n, n, 1.0, 0.0, "uniform", config=5, case=n)
+    ta, tb = layout[0] == "T", layout[1] == "T"
+    return GemmCase(f"{in_type}_{n}_{layout.lower()}", dt, ta, tb, n, n, n, 1.0, 0.0, "uniform", config=5,
+                    case=n + (0 if layout == "NT" else 1 + 2 * ta + tb))
 
 
 def target_workload() -> GemmCase:

@@ -157,3 +157,34 @@ def test_tuner_enumerates_and_prunes():
     # a k-split cannot have more slices than k-blocks
     assert not tune.prune("umma_2cta", {1: 256, 2: 8, 3: 2, 10: 1, 0: 0}, 256, 256, 128)
     assert len(list(tune.candidates(tune.SPACE_F32, quick=True))) == 8
+
+
+def test_per_device_once_bookkeeping():
+    """Context set-up (a kernel's shared-memory attribute, occupancy queries) is remembered per device, so a
+    second GPU used by the same process is set up as well; the library checks its own bookkeeping on the host."""
+    assert P.peak_selftest_per_device_once() == 0
+
+
+def test_last_kernel_is_text_and_needs_a_buffer():
+    assert isinstance(P.peak_last_kernel(), str)
+    assert P.load().peak_last_kernel(None, 16) == P.PEAK_ERR_INVALID_VALUE
+
+
+def test_bench_traffic_is_read_from_the_profile_of_the_launched_kernel():
+    """bench.py quotes DRAM traffic from the ncu summary under profiles/ only when that summary covers the kernel
+    that was launched; a different kernel (or an unprofiled workload) gives null and a reason."""
+    import bench
+    t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 512, __nv_bfloat16, 0, 0, 0, 0> grid=148 items=512 splits=1")
+    assert t is not None and 0.3e9 < t < 3e9 and "profiles/" in src
+    t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 256, __nv_bfloat16, 0, 0, 0, 0> grid=148")
+    assert t is None and "differs" in src
+    t, src = bench.profile_traffic("no_such_workload", "x_kernel<1>")
+    assert t is None and "no ncu summary" in src
+
+
+def test_bench_rotation_rule():
+    import bench
+    table = bench.workloads_table()
+    assert bench.rotation_sets(table["bf16_8192_nn"]) == 1 and "larger than L2" in bench.l2_note(table["bf16_8192_nn"])
+    n = bench.rotation_sets(table["bf16_4096_nn"])
+    assert n >= 4 and n * bench.set_bytes(table["bf16_4096_nn"]) > 3 * bench.L2_BYTES
