@@ -107,9 +107,9 @@ typedef enum peak_variant {
  *   lda, ldb, ldc  row pitches in elements
  *   stream         cudaStream_t
  * The fastest variant whose preconditions hold is chosen: the tensor-core path needs 16-byte aligned
- * base pointers and row pitches that are multiples of 16 bytes, and for the 8-bit input types also
- * transA = 0, transB = 1 (both operands stored with K innermost); anything else runs on the fallback
- * kernel with the same result contract.  Returns after enqueueing; never synchronises.
+ * base pointers and row pitches that are multiples of 16 bytes (all four layouts, for 16-bit and 8-bit
+ * inputs alike); anything else runs on the fallback kernel with the same result contract.  Returns after
+ * enqueueing; never synchronises.
  */
 int peak_gemm(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
               int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream);

@@ -404,8 +404,12 @@ template <> struct McOps<0> {
 };
 
 // IN8: the inputs are 8-bit floats.  A k-block is still one 128-byte swizzle row per matrix row, so it holds
-// 128 elements instead of 64, every byte count and descriptor stays as it is, and the MMA is the f8f6f4 kind
-// with K = 32 per instruction.  Both operands must be K-major (A not transposed, B transposed).
+// 128 elements instead of 64, every byte count and descriptor of a K-major operand stays as it is, and the MMA
+// is the f8f6f4 kind with K = 32 per instruction.  An MN-major 8-bit operand (A transposed, B not transposed)
+// is described to the MMA exactly like a 16-bit one -- major bit in the instruction descriptor, 128-byte
+// swizzle, 8-row groups 1 KiB apart -- with every count taken in bytes: a swizzle row holds 128 elements of
+// M (or N), a k-block has 128 k-rows, so one box is 128 x 128 bytes = 16 KiB, the boxes of a tile lie 16 KiB
+// apart (leading-dimension offset) and one K = 32 instruction advances 32 rows = 4 KiB.
 // G2: a one-slot tile is drained by two groups of four epilogue warps, each taking half of the columns.  The
 // epilogue of such a tile hides behind the next tile's main loop, so the second group only pays when there is
 // no next tile: problems of at most two waves, where it shortens the exposed tail of the launch.
@@ -432,6 +436,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t accempty0 = accfull0 + 16;
     const uint32_t cbar0 = accempty0 + 16;  // old-C barriers: two per epilogue warp of a one-group kernel
 
+    // MN-major operands: elements of M / N per 128-byte swizzle row, and bytes of one box (all k-rows of a
+    // k-block under that row)
+    constexpr int MN_ELEMS = IN8 ? 128 : 64;
+    constexpr int MN_ATOM = IN8 ? 2 * ATOM_BYTES : ATOM_BYTES;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     static_assert(MC == 0 || (CG == 2 && BN >= 256), "the multicast build pairs CTAs and uses 256- or 512-wide tiles");
@@ -513,8 +521,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         load_tile<CG, BATCHED>(a_dst, &tmA, k0, m_cta, bz, bar);
                     } else {
 #pragma unroll
-                        for (int h = 0; h < BM / 64; ++h) {
-                            load_tile<CG, BATCHED>(a_dst + h * ATOM_BYTES, &tmA, m_cta + 64 * h, k0, bz, bar);
+                        for (int h = 0; h < BM / MN_ELEMS; ++h) {
+                            load_tile<CG, BATCHED>(a_dst + h * MN_ATOM, &tmA, m_cta + MN_ELEMS * h, k0, bz, bar);
                         }
                     }
                     if (MC) {
@@ -541,9 +549,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                         for (int hf = 0; hf < C_::HALVES; ++hf) {
 #pragma unroll
-                            for (int h = 0; h < C_::HROWS / 64; ++h) {
-                                const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * ATOM_BYTES;
-                                const int n = n_cta + hf * C_::SLOT_N + 64 * h;
+                            for (int h = 0; h < C_::HROWS / MN_ELEMS; ++h) {  // (8-bit: HROWS >= 128, host-checked)
+                                const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * MN_ATOM;
+                                const int n = n_cta + hf * C_::SLOT_N + MN_ELEMS * h;
                                 load_tile<CG, BATCHED>(d, &tmB, n, k0, bz, bar);
                             }
                         }
@@ -565,8 +573,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0 && leader) {
             uint32_t it = 0, tl = 0;
             bool ok = true;
-            const uint32_t a_lbo = p.a_mn ? (uint32_t)ATOM_BYTES : 16u, b_lbo = p.b_mn ? (uint32_t)ATOM_BYTES : 16u;
-            const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+            const uint32_t a_lbo = p.a_mn ? (uint32_t)MN_ATOM : 16u, b_lbo = p.b_mn ? (uint32_t)MN_ATOM : 16u;
+            // one instruction's K: 32 bytes along a K-major row, or 16 (8-bit: 32) k-rows of 128 bytes
+            constexpr uint32_t MN_KSTEP = IN8 ? 4096u : 2048u;
+            const uint32_t a_kstep = p.a_mn ? MN_KSTEP : 32u, b_kstep = p.b_mn ? MN_KSTEP : 32u;
             for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
                 const Item w = decode_item(p, item);
                 const int kb0 = w.kb0, kb1 = w.kb1;

@@ -66,6 +66,8 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     for (int bn : {512, 256, 128}) {
         if (force_bn ? bn != force_bn : bn == 512) continue;  // 512-wide tiles only on request (see launch_umma)
         if (bn == 512 && cg != 2) continue;
+        // an 8-bit B stored K x N is fetched 128 columns at a time: a pair's 128-wide tile (64 per CTA) is out
+        if (bn == 128 && cg == 2 && is_fp8(in_elem(g.dtype)) && !g.transB) continue;
         const int64_t tiles = tiles_of(g, cg, bn);
         const double kb_cycles = fmax(2.0 * bn, (128.0 + bn / cg) * 128.0 / kL2BytesPerClk);
         const double item_ovh = 1500.0;
@@ -102,6 +104,7 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
             }
         }
     }
+    if (best_cost == 1e300) best = Plan{256, (int)tiles_of(g, cg, 256), 1};  // a forced width nothing above accepts
     return best;
 }
 
@@ -121,10 +124,13 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const int b_mn = g.transB ? 0 : 1;  // B stored K x N: N is the contiguous index
     CUtensorMap tmA, tmB, tmC, tmW;
     const int64_t nb = g.nbatch();
-    if (IN8 && (a_mn || b_mn)) return PEAK_ERR_UNSUPPORTED;  // 8-bit operands: K-major only
-    bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, 64, BK, nb, g.strideA)
+    // An MN-major operand is fetched in boxes of one 128-byte swizzle row of M / N (64 16-bit or 128 8-bit
+    // elements) by all k-rows of a k-block; an 8-bit B of that kind needs at least 128 columns per CTA.
+    constexpr int MNE = IN8 ? 128 : 64;
+    if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
+    bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, MNE, BKE, nb, g.strideA)
                    : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, 128, nb, g.strideA);
-    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, 64, BK, nb, g.strideB)
+    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, MNE, BKE, nb, g.strideB)
                      : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS, nb, g.strideB));
     if (!ok) return nb > 1 ? PEAK_ERR_UNSUPPORTED : PEAK_ERR_CUDA;  // e.g. a batch stride TMA cannot express
 
@@ -352,7 +358,6 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
     if (g.M >= (1ll << 31) - 512 || g.N >= (1ll << 31) - 512 || g.K >= (1ll << 31) - 512) return false;
     if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16) return false;
     const bool in8 = is_fp8(in_elem(g.dtype));
-    if (in8 && (g.transA || !g.transB)) return false;  // 8-bit operands: K-major only (A as is, B transposed)
     const int pitch_unit = in8 ? 16 : 8;               // TMA: row pitch must be a multiple of 16 bytes
     if (g.lda % pitch_unit || g.ldb % pitch_unit) return false;
     if (g.lda >= (1ll << 38) || g.ldb >= (1ll << 38) || g.ldc >= (1ll << 38)) return false;

@@ -1,6 +1,8 @@
 """GPU parity for 8-bit floating-point inputs (E4M3 / E5M2 operands, bf16 or fp32 output) against the CPU
-oracle, whose decoders are written from the bit layout and pinned separately.  The tensor-core path takes
-K-major operands only (A as stored, B transposed); the other layouts run on the portable kernel."""
+oracle, whose decoders are written from the bit layout and pinned separately.  The tensor-core path takes all
+four layouts (a K-major operand as one 128-byte swizzle row of K per matrix row, an MN-major one through the
+major bit of the instruction descriptor); pitches that are not multiples of 16 bytes run on the portable
+kernel."""
 import numpy as np
 import pytest
 
@@ -27,6 +29,13 @@ def pad16(n):
 def k_major(dtype, M, N, K, **kw):
     """A row-major M x K, B stored N x K (transB), pitches padded to 16 bytes as the TMA path needs."""
     return mk(dtype, 0, 1, M, N, K, pad_a=pad16(K), pad_b=pad16(K), **kw)
+
+
+def any_layout(dtype, ta, tb, M, N, K, **kw):
+    """Any layout with the pitches padded to 16 bytes, as the TMA path needs."""
+    a_cols = M if ta else K
+    b_cols = K if tb else N
+    return mk(dtype, ta, tb, M, N, K, pad_a=pad16(a_cols), pad_b=pad16(b_cols), **kw)
 
 
 @pytest.fixture
@@ -108,13 +117,80 @@ def test_umma_fp8_ragged_alpha_beta(variant, dtype):
         R.check_full(dc, what=f"{c.name} {P.peak_variant_string(variant)}")
 
 
-@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32])
-def test_fp8_tensor_core_variant_refuses_other_layouts(dtype):
-    c = mk(dtype, 1, 0, 256, 256, 256)
+@pytest.mark.parametrize("variant", UMMA)
+@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_F32, W.PEAK_E5M2_BF16])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_umma_fp8_every_layout_exact_small_integers(variant, dtype, ta, tb):
+    """All four layouts on the tensor cores: small integers, so that a wrong box, k-step or leading-dimension
+    offset of an MN-major 8-bit operand (a dropped, repeated or misplaced k-row or column) changes the exact
+    result.  Sizes cover one tile, several tiles and k-blocks, and ragged M, N and K."""
+    for (M, N, K) in [(128, 256, 128), (256, 512, 384), (384, 256, 512), (200, 328, 208), (130, 72, 48),
+                      (1000, 1100, 1300)]:
+        c = any_layout(dtype, ta, tb, M, N, K, dist="smallint", case=K + 3 * ta + 5 * tb)
+        if c.out_type != "f32":
+            c = c.with_(alpha=0.125)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        assert_bits_equal(c, dc, f"{c.name} {c.layout} {P.peak_variant_string(variant)}")
+
+
+@pytest.mark.parametrize("dtype", PAIRS_8)
+@pytest.mark.parametrize("ta,tb", [(0, 0), (1, 0), (1, 1)])
+def test_umma_fp8_mn_major_real_values(dtype, ta, tb, reset_tuning):
+    """Real-valued inputs, alpha / beta, several tile widths and a k-split on the layouts with an MN-major
+    operand; the dispatcher must pick a tensor-core kernel for them."""
+    for tile_n, split in [(0, 0), (128, 0), (256, 3), (512, 0)]:
+        P.peak_set_tuning(P.PEAK_TUNE_TILE_N, tile_n)
+        P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+        c = any_layout(dtype, ta, tb, 520, 1032, 3000 + 8, dist="uniform", alpha=0.75, beta=0.5, pad_c=8,
+                       case=tile_n + split)
+        for variant in UMMA + [P.PEAK_VARIANT_AUTO]:
+            dc = R.DeviceCase(c)
+            v = P.peak_query_variant(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb,
+                                     c.beta, dc.C, c.ldc)
+            assert v in UMMA, f"{c.layout}: dispatcher chose {P.peak_variant_string(v)}"
+            dc.run(variant)
+            assert "umma_gemm_kernel" in P.peak_last_kernel()
+            R.check_full(dc, what=f"{c.name} {c.layout} bn{tile_n} split{split} {P.peak_variant_string(variant)}")
+
+
+def test_fp8_every_bit_pattern_every_layout():
+    """All finite bit patterns of both formats as A (one per row) against B = e_0, in every layout, on the
+    tensor cores: the MN-major paths decode exactly as the oracle does."""
+    import torch
+    for dtype, t in [(W.PEAK_E4M3_F32, "e4m3"), (W.PEAK_E5M2_F32, "e5m2")]:
+        bits = np.arange(256, dtype=np.uint8)
+        vals = oracle.decode(R.OT[t], bits)
+        keep = np.isfinite(vals)
+        a = np.zeros((256, 32), dtype=np.uint8)          # op(A): 256 x 32, column 5 carries the patterns
+        a[:, 5] = np.where(keep, bits, 0)
+        one = W.encode(np.ones((1, 1), np.float32), t)[0, 0]
+        b = np.zeros((32, 48), dtype=np.uint8)           # op(B): 32 x 48 with B[5, 7] = 1
+        b[5, 7] = one
+        want = np.where(keep, vals, 0.0)
+        for ta, tb in LAYOUTS:
+            As = np.ascontiguousarray(a.T if ta else a)
+            Bs = np.ascontiguousarray(b.T if tb else b)
+            A, B = torch.from_numpy(As).cuda(), torch.from_numpy(Bs).cuda()
+            for variant in UMMA:
+                C = torch.full((256, 48), float("nan"), dtype=torch.float32, device="cuda")
+                P.peak_gemm_variant(variant, dtype, ta, tb, 256, 48, 32, 1.0, A, As.shape[1], B, Bs.shape[1], 0.0, C,
+                                    48, None)
+                rc, _ = P.peak_check(None)
+                assert rc == P.PEAK_OK
+                got = C.cpu().numpy().astype(np.float64)
+                assert np.array_equal(got[:, 7], want), f"{t} {ta}{tb} {P.peak_variant_string(variant)}"
+                got[:, 7] = 0
+                assert (got == 0).all()
+
+
+def test_fp8_unaligned_pitch_still_runs_on_the_portable_kernel():
+    c = mk(W.PEAK_E4M3_BF16, 1, 0, 256, 256, 256, pad_a=3)
     dc = R.DeviceCase(c)
     with pytest.raises(P.PeakError):
         dc.run(P.PEAK_VARIANT_UMMA_2CTA)
-    dc.run(P.PEAK_VARIANT_AUTO)      # the dispatcher routes it to the portable kernel instead
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "fallback" in P.peak_last_kernel()
     R.check_full(dc)
 
 
@@ -130,10 +206,11 @@ def test_umma_fp8_tiles_and_split_k(dtype, tile_n, split, reset_tuning):
         R.check_full(dc, what=f"{c.name} bn{tile_n} split{split} {P.peak_variant_string(variant)}")
 
 
-@pytest.mark.parametrize("dtype", [W.PEAK_E4M3_BF16, W.PEAK_E4M3_F32])
-def test_fp8_full_size_sampled(dtype):
-    """8192^3 K-major in the launch configuration the benchmark times, on a sampled sub-grid."""
-    c = k_major(dtype, 8192, 8192, 8192, dist="uniform")
+@pytest.mark.parametrize("dtype,ta,tb", [(W.PEAK_E4M3_BF16, 0, 1), (W.PEAK_E4M3_F32, 0, 1), (W.PEAK_E4M3_BF16, 0, 0),
+                                         (W.PEAK_E5M2_BF16, 1, 0), (W.PEAK_E4M3_BF16, 1, 1)])
+def test_fp8_full_size_sampled(dtype, ta, tb):
+    """8192^3 in the launch configuration the benchmark times, on a sampled sub-grid."""
+    c = any_layout(dtype, ta, tb, 8192, 8192, 8192, dist="uniform")
     dc = R.DeviceCase(c)
     dc.run(P.PEAK_VARIANT_AUTO)
     R.check_sampled(dc, tile_m=256, tile_n=256, budget_macs=6e8)

@@ -78,7 +78,7 @@ def test_random_multi_wave_cases_sampled():
         for n in range(80):
             dt = types[rng.integers(len(types))]
             in8 = W.IN_TYPE[dt] in ("e4m3", "e5m2")
-            ta, tb = (0, 1) if in8 else (int(rng.integers(2)), int(rng.integers(2)))
+            ta, tb = int(rng.integers(2)), int(rng.integers(2))
             M = int(rng.integers(1, 40)) * 128 + int(rng.choice([0, 0, 8, 56]))
             N = int(rng.integers(1, 40)) * 128 + int(rng.choice([0, 0, 8, 72]))
             K = int(rng.integers(1, 40)) * 64 + int(rng.choice([0, 0, 16, 40]))

@@ -88,11 +88,11 @@ def test_dispatch_choices(lib):
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 1.0, al, 64) == P.PEAK_VARIANT_NONE
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 0.0, al, 64) == P.PEAK_VARIANT_SCALE
     assert q(9, 0, 0, 64, 64, 64, 1.0, al, 64, al, 64, 0.0, al, 64) == -P.PEAK_ERR_INVALID_VALUE
-    # 8-bit float inputs: tensor cores only for K-major operands (A as stored, B transposed), 16-byte pitches
+    # 8-bit float inputs: tensor cores for every layout, given 16-byte pitches
     for dt in (P.PEAK_E4M3_BF16, P.PEAK_E4M3_F32, P.PEAK_E5M2_BF16, P.PEAK_E5M2_F32):
-        assert q(dt, 0, 1, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_2CTA
-        for ta, tb in [(0, 0), (1, 0), (1, 1)]:
-            assert q(dt, ta, tb, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
+        for ta, tb in [(0, 1), (0, 0), (1, 0), (1, 1)]:
+            assert q(dt, ta, tb, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_2CTA
+        assert q(dt, 1, 0, 4096, 4096, 4096, 1.0, al, 4100, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
         assert q(dt, 0, 1, 4096, 4096, 1000, 1.0, al, 1000, al, 1000, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
         assert q(dt, 0, 1, 4096, 4096, 1000, 1.0, al, 1008, al, 1008, 0.0, al, 4096) == P.PEAK_VARIANT_UMMA_2CTA
     # few tiles: single-CTA tiles spread the problem over more SMs than 256-row pair tiles would
