@@ -261,7 +261,9 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_SGEMM_FMA = 4,    /* SGEMM inner product: 1 = scalar fp32 FMA, 2 = two-wide fp32 FMA (default) */
     PEAK_TUNE_TAIL_SPLIT = 5,   /* 2 = split the tiles of the last, partly filled wave whenever possible (off by default) */
     PEAK_TUNE_DEPENDENT_LAUNCH = 6, /* 1 = launch the tensor-core kernel without programmatic dependent launch */
-    PEAK_TUNE_SGEMM_COPY = 7,   /* SGEMM tile loads: 1 = staged through registers, 2 = asynchronous copies */
+    PEAK_TUNE_SGEMM_COPY = 7,   /* SGEMM tile loads: 1 = staged through registers, 2 = cp.async ring (both: whole
+                                   128 x 128 x 16 tiles only), 3 = TMA + mbarrier ring (any shape; the default
+                                   except for whole-tile problems with B transposed) */
     PEAK_TUNE_WAIT_MS = 8,      /* budget of each device-side barrier wait in ms at 2 GHz (default 2000) */
     PEAK_TUNE_INJECT_STALL = 9, /* test hook, 1 = one CTA leaves one pipeline stage unfilled so that the bounded
                                    waits run out: the call's result is then wrong by design and peak_check()

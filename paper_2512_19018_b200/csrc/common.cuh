@@ -117,6 +117,8 @@ int launch_scale(const GemmArgs &g);
 int launch_xcheck_f64(const GemmArgs &g, const void *C0, double *Cref, int64_t ldcref);
 int launch_sgemm(const GemmArgs &g);
 bool sgemm_supports(const GemmArgs &g);
+int launch_sgemm_tma(const GemmArgs &g);        // TMA-fed SGEMM: any shape, 16-byte aligned operands
+bool sgemm_tma_supports(const GemmArgs &g);
 int launch_umma(const GemmArgs &g, int cta_group);
 bool umma_supports(const GemmArgs &g, int cta_group);
 int umma_units(int cta_group);  // CTAs (cta_group 1) or CTA pairs (2) a persistent launch can keep resident

@@ -315,7 +315,8 @@ template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
 
 }  // namespace
 
-bool sgemm_supports(const GemmArgs &g) {
+// The earlier kernels (block-wide barriers, no edge handling): whole 128 x 128 x 16 tiles only.
+static bool sgemm_aligned_supports(const GemmArgs &g) {
     if (g.dtype != PEAK_F32_F32) return false;
     if (g.M < SG_BM || g.N < SG_BN || g.K < SG_BK) return false;
     if (g.M % SG_BM || g.N % SG_BN || g.K % SG_BK) return false;
@@ -328,11 +329,20 @@ bool sgemm_supports(const GemmArgs &g) {
     return true;
 }
 
+bool sgemm_supports(const GemmArgs &g) { return sgemm_tma_supports(g) || sgemm_aligned_supports(g); }
+
 int launch_sgemm(const GemmArgs &g) {
     if (!sgemm_supports(g)) return PEAK_ERR_UNSUPPORTED;
-    // The asynchronous-copy kernel wins unless both operands need the 4-byte transposing copies (A not
-    // transposed and B transposed: measured 52 vs 57 TFLOP/s at 4096^3), where register staging is kept.
-    const int copy = tuning(PEAK_TUNE_SGEMM_COPY);  // 1 = registers, 2 = asynchronous copies, 0 = by layout
+    // Default: the TMA-fed kernel (any shape).  PEAK_TUNE_SGEMM_COPY = 1 / 2 selects the earlier kernels for
+    // A/B measurements, on shapes made of whole tiles: 1 = tiles staged through registers, 2 = cp.async ring.
+    // With B transposed (k-contiguous rows of B, sixteen different ones per warp) the TMA-fed kernel is slower
+    // than the earlier kernels (4096^3: NT 34 against 53, TT 43 against 57 TFLOP/s), so whole-tile shapes of
+    // those layouts stay on them; PEAK_TUNE_SGEMM_COPY = 3 forces the TMA-fed kernel.
+    const int copy = tuning(PEAK_TUNE_SGEMM_COPY);
+    const bool aligned = sgemm_aligned_supports(g);
+    const bool want_tma = copy == 3 || !aligned || (copy == 0 && !g.transB);
+    if (want_tma && sgemm_tma_supports(g)) return launch_sgemm_tma(g);
+    if (!aligned) return PEAK_ERR_UNSUPPORTED;
     const bool both_k_contiguous = !g.transA && g.transB;
     if (copy == 2 || (copy == 0 && !both_k_contiguous))
         return tuning(PEAK_TUNE_SGEMM_FMA) != 1 ? dispatch_sgemm_async<true>(g) : dispatch_sgemm_async<false>(g);

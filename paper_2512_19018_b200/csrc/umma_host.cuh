@@ -29,8 +29,9 @@ inline EncodeTiledFn encode_fn() {
 // Tensor map over a stack of `batch` row-major 2-D arrays `batch_stride` elements apart: `inner` contiguous
 // elements per row, `outer` rows, `pitch` elements between rows; box = box_inner x box_outer x 1, 128-byte
 // swizzle, zero fill.  batch <= 1 gives a two-dimensional map of the one matrix.
+// `swizzle_bytes`: 128 (the tensor-core tiles), 64, or 0 for a dense box.
 inline bool encode_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch,
-                       int box_inner, int box_outer, int64_t batch, int64_t batch_stride) {
+                       int box_inner, int box_outer, int64_t batch, int64_t batch_stride, int swizzle_bytes = 128) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const CUtensorMapDataType dt = e == Elem::F16    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
@@ -43,8 +44,11 @@ inline bool encode_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner,
     cuuint64_t strides[2] = {(cuuint64_t)pitch * eb, (cuuint64_t)batch_stride * eb};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(tm, dt, rank, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUtensorMapSwizzle sw = swizzle_bytes == 128  ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                        : CU_TENSOR_MAP_SWIZZLE_NONE;
+    CUresult r = fn(tm, dt, rank, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -55,10 +59,11 @@ inline bool encode_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner,
 struct MapKey {
     const void *base;
     int64_t inner, outer, pitch, batch, batch_stride;
-    int elem, box_inner, box_outer;
+    int elem, box_inner, box_outer, swizzle;
     bool operator==(const MapKey &o) const {
         return base == o.base && inner == o.inner && outer == o.outer && pitch == o.pitch && batch == o.batch &&
-               batch_stride == o.batch_stride && elem == o.elem && box_inner == o.box_inner && box_outer == o.box_outer;
+               batch_stride == o.batch_stride && elem == o.elem && box_inner == o.box_inner &&
+               box_outer == o.box_outer && swizzle == o.swizzle;
     }
 };
 constexpr int kMapCacheSlots = 64;
@@ -73,12 +78,12 @@ inline MapCache &map_cache() {
     return c;
 }
 inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, int64_t outer, int64_t pitch, int box_inner,
-                     int box_outer, int64_t batch = 1, int64_t batch_stride = 0) {
-    const MapKey k{base, inner, outer, pitch, batch, batch_stride, (int)e, box_inner, box_outer};
+                     int box_outer, int64_t batch = 1, int64_t batch_stride = 0, int swizzle_bytes = 128) {
+    const MapKey k{base, inner, outer, pitch, batch, batch_stride, (int)e, box_inner, box_outer, swizzle_bytes};
     uint64_t h = (uint64_t)reinterpret_cast<uintptr_t>(base) >> 4;
     h ^= (uint64_t)inner * 0x9E3779B97F4A7C15ull;
     h ^= ((uint64_t)outer + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
-    h ^= (uint64_t)(box_outer * 131 + box_inner) * 0x165667B19E3779F9ull;
+    h ^= (uint64_t)(box_outer * 131 + box_inner + swizzle_bytes * 7919) * 0x165667B19E3779F9ull;
     h ^= h >> 29;
     MapCache &c = map_cache();
     const int slot = (int)(h % kMapCacheSlots);
@@ -87,7 +92,7 @@ inline bool make_map(CUtensorMap *tm, Elem e, const void *base, int64_t inner, i
         ++c.hits;
         return true;
     }
-    if (!encode_map(tm, e, base, inner, outer, pitch, box_inner, box_outer, batch, batch_stride)) return false;
+    if (!encode_map(tm, e, base, inner, outer, pitch, box_inner, box_outer, batch, batch_stride, swizzle_bytes)) return false;
     c.key[slot] = k;
     c.map[slot] = *tm;
     c.used[slot] = true;

@@ -181,7 +181,30 @@ def test_sgemm_parity(ta, tb):
     assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref))
 
 
-@pytest.mark.parametrize("copy", [1, 2])
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_sgemm_ragged_shapes_run_the_fast_kernel(ta, tb, reset_tuning):
+    """Shapes that are not made of whole tiles (ragged M, N, a K tail, one-row and one-column problems) run on the
+    TMA-fed SGEMM kernel, whose copies zero-fill the edges: exact on integers, within the fp32 bounds on reals,
+    guard bands and pitch padding untouched."""
+    shapes = [(1000, 1000, 1000), (129, 257, 33), (1, 300, 50), (300, 1, 7), (131, 131, 16), (500, 300, 250)]
+    for idx, (M, N, K) in enumerate(shapes):
+        pa, pb = (-(M if ta else K)) % 4, (-(K if tb else N)) % 4        # the copy engine wants 16-byte pitches
+        for pc in (0, 3):                                                # aligned and unaligned rows of C
+            ci = mk(W.PEAK_F32_F32, ta, tb, M, N, K, dist="smallint", alpha=2.0, beta=-1.0, pad_a=pa, pad_b=pb,
+                    pad_c=pc, case=idx)
+            dc = R.DeviceCase(ci)
+            dc.run(P.PEAK_VARIANT_SGEMM)
+            assert "sgemm_tma_kernel" in P.peak_last_kernel()
+            ref, _ = dc.oracle_full()
+            assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref)), f"{ci}"
+        cr = mk(W.PEAK_F32_F32, ta, tb, M, N, K, alpha=0.5, beta=2.0, pad_a=pa + 4, pad_b=pb, pad_c=1, case=idx)
+        dr = R.DeviceCase(cr)
+        dr.run(P.PEAK_VARIANT_AUTO)
+        assert "sgemm_tma_kernel" in P.peak_last_kernel()
+        R.check_full(dr)
+
+
+@pytest.mark.parametrize("copy", [1, 2, 3])
 @pytest.mark.parametrize("fma", [1, 2])
 def test_sgemm_kernel_variants_agree_with_oracle(copy, fma, reset_tuning):
     """Register-staged vs asynchronous-copy tile loads, scalar vs two-wide FMA: every combination exact on
@@ -201,7 +224,7 @@ def test_sgemm_kernel_variants_agree_with_oracle(copy, fma, reset_tuning):
 
 
 def test_sgemm_unsupported_shape_is_reported_not_faulted():
-    c = mk(W.PEAK_F32_F32, 0, 0, 100, 128, 16)
+    c = mk(W.PEAK_F32_F32, 0, 0, 100, 128, 16, pad_a=1)      # a pitch the copy engine cannot take, not whole tiles
     dc = R.DeviceCase(c)
     rc = P.peak_gemm_variant(P.PEAK_VARIANT_SGEMM, c.dtype, 0, 0, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb, 0.0,
                              dc.C, c.ldc, check=False)

@@ -82,7 +82,8 @@ def test_dispatch_choices(lib):
     assert q(P.PEAK_BF16_BF16, 0, 0, 100, 100, 100, 1.0, al, 100, al, 100, 0.0, al, 100) == P.PEAK_VARIANT_FALLBACK
     assert q(P.PEAK_BF16_BF16, 0, 0, 128, 128, 128, 1.0, al + 2, 128, al, 128, 0.0, al, 128) == P.PEAK_VARIANT_FALLBACK
     assert q(P.PEAK_F32_F32, 0, 0, 4096, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_SGEMM
-    assert q(P.PEAK_F32_F32, 0, 0, 100, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
+    assert q(P.PEAK_F32_F32, 0, 0, 100, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_SGEMM
+    assert q(P.PEAK_F32_F32, 0, 0, 100, 4096, 4096, 1.0, al, 4098, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_FALLBACK
     assert q(P.PEAK_F32_F32, 0, 0, 0, 4096, 4096, 1.0, al, 4096, al, 4096, 0.0, al, 4096) == P.PEAK_VARIANT_NONE
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 0, 1.0, None, 1, None, 64, 0.5, al, 64) == P.PEAK_VARIANT_SCALE
     assert q(P.PEAK_F32_F32, 0, 0, 64, 64, 64, 0.0, al, 64, al, 64, 1.0, al, 64) == P.PEAK_VARIANT_NONE
