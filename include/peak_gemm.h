@@ -143,6 +143,29 @@ int peak_gemm_fused_variant(int variant, int dtype, int transA, int transB, int6
                             int64_t ldc, const float *bias, int activation, void *stream);
 
 /*
+ * peak_gemm_fused_residual: the fused tail with a residual operand,
+ *     C = act( alpha*op(A)*op(B) + beta*C + bias ) + R,
+ * the third operation that commonly follows a linear layer (a skip connection); like bias and activation it
+ * is fused into the producing kernel's epilogue instead of costing another pass over C (paper sections 1 and
+ * 3.2 on fusing neighbouring operations).
+ *   R    device pointer to an M x N row-major matrix of the OUTPUT storage type of `dtype`, or NULL for none
+ *   ldr  row pitch of R in elements, >= N when R is given
+ * R is only read; it must not overlap C (with R == C the result is unspecified: use beta instead).  The
+ * residual is converted to fp32 and added after the activation; the sum is rounded once to the output type.
+ * R may have any alignment (16-byte aligned bases and pitches are read with vector loads).  Everything else
+ * -- kernels, layouts, quick returns (K == 0 or alpha == 0: C = act(beta*C + bias) + R), asynchrony, errors --
+ * is as for peak_gemm_fused.  The _variant form names the kernel family.
+ */
+int peak_gemm_fused_residual(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
+                             const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C,
+                             int64_t ldc, const float *bias, int activation, const void *R, int64_t ldr,
+                             void *stream);
+int peak_gemm_fused_residual_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N,
+                                     int64_t K, float alpha, const void *A, int64_t lda, const void *B,
+                                     int64_t ldb, float beta, void *C, int64_t ldc, const float *bias,
+                                     int activation, const void *R, int64_t ldr, void *stream);
+
+/*
  * peak_gemm_strided_batched: `batch` independent GEMMs of one shape,
  *     C_b = alpha * op(A_b) * op(B_b) + beta * C_b,   X_b = X + b * strideX   (strides in elements),
  * the second half of the paper's fusion / specialisation motive (sections 1, 3.1: kernels are specialised

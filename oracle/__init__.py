@@ -68,6 +68,8 @@ def _load():
         lib.oracle_gemm_submatrix.argtypes = common + [i64, vp, i64, vp, vp, vp]
         lib.oracle_bias_act.restype = ci
         lib.oracle_bias_act.argtypes = [vp, i64, i64, vp, ci]
+        lib.oracle_residual_add.restype = ci
+        lib.oracle_residual_add.argtypes = [vp, i64, i64, ci, vp, i64]
         _lib = lib
     return _lib
 
@@ -202,6 +204,22 @@ def bias_act(ref, bias=None, act=ACT_NONE) -> np.ndarray:
     if rc:
         raise ValueError(f"oracle_bias_act failed: {rc}")
     return x
+
+
+def residual_add(x, R, r_type: int, ldr: int) -> np.ndarray:
+    """x (2-D float64) + the residual matrix R (stored bits of type r_type, row pitch ldr); returns a new array."""
+    lib = _load()
+    out = np.array(x, dtype=np.float64, order="C", copy=True)
+    if out.ndim != 2:
+        raise ValueError("x must be 2-D")
+    Rb = _store(R, r_type)
+    rows, cols = out.shape
+    if rows and Rb.size < (rows - 1) * ldr + cols:
+        raise ValueError("R too small for its shape / ldr")
+    rc = lib.oracle_residual_add(_ptr(out), rows, cols, int(r_type), _ptr(Rb), int(ldr))
+    if rc:
+        raise ValueError(f"oracle_residual_add failed: {rc}")
+    return out
 
 
 def num_threads() -> int:

@@ -20,7 +20,8 @@
  *     opB(k,j) = transB ? B[j*ldb + k] : B[k*ldb + j]
  *     C0(i,j)  = C0[i*ldc + j]
  *
- * oracle_bias_act() applies the fused tail, ref + bias[j] followed by ReLU or GELU, on top of that.
+ * oracle_bias_act() applies the fused tail, ref + bias[j] followed by ReLU or GELU, on top of that, and
+ * oracle_residual_add() the residual matrix that may follow the activation.
  *
  * Stored elements (binary16, bfloat16, binary32) are decoded to double by the
  * bit-level decoders below, exactly; nothing here includes a CUDA header.
@@ -381,6 +382,19 @@ int oracle_bias_act(double *x, int64_t rows, int64_t cols, const double *bias, i
                 v = 0.5 * v * (1.0 + erf(v * 0.70710678118654752440));
             x[i * cols + j] = v;
         }
+    return ORACLE_OK;
+}
+
+/* Residual operand of the fused tail (an addition beyond the paper, like the tail itself): after bias and
+ * activation, x(i,j) += R(i,j), with R an M x N row-major matrix of storage type r_type and pitch ldr, decoded
+ * exactly; the sum stays in fp64 (the caller rounds once). */
+int oracle_residual_add(double *x, int64_t rows, int64_t cols, int r_type, const void *R, int64_t ldr)
+{
+    if (rows < 0 || cols < 0 || r_type < ORACLE_F16 || r_type > ORACLE_F32 || (rows * cols > 0 && (!x || !R)) || ldr < cols)
+        return ORACLE_BAD_ARG;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j)
+            x[i * cols + j] += load_elem(r_type, R, i * ldr + j);
     return ORACLE_OK;
 }
 

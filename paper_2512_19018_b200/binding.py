@@ -24,7 +24,8 @@ _lib = None
 EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_staging", "peak_gemm_xcheck_f64",
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
            "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available", "peak_gemm_fused",
-           "peak_gemm_fused_variant", "peak_gemm_strided_batched", "peak_last_kernel", "peak_selftest_per_device_once"]
+           "peak_gemm_fused_variant", "peak_gemm_strided_batched", "peak_last_kernel", "peak_selftest_per_device_once",
+           "peak_gemm_fused_residual", "peak_gemm_fused_residual_variant"]
 
 
 class PeakError(RuntimeError):
@@ -62,6 +63,10 @@ def load():
     lib.peak_gemm_fused.argtypes = gemm_args[:-1] + [vp, i, vp]
     lib.peak_gemm_fused_variant.restype = i
     lib.peak_gemm_fused_variant.argtypes = [i] + gemm_args[:-1] + [vp, i, vp]
+    lib.peak_gemm_fused_residual.restype = i
+    lib.peak_gemm_fused_residual.argtypes = gemm_args[:-1] + [vp, i, vp, i64, vp]
+    lib.peak_gemm_fused_residual_variant.restype = i
+    lib.peak_gemm_fused_residual_variant.argtypes = [i] + gemm_args[:-1] + [vp, i, vp, i64, vp]
     lib.peak_gemm_strided_batched.restype = i
     lib.peak_gemm_strided_batched.argtypes = [i, i, i, i64, i64, i64, f, vp, i64, i64, vp, i64, i64, f, vp, i64, i64,
                                               i64, vp]
@@ -174,6 +179,26 @@ def peak_gemm_fused_variant(variant, dtype, transA, transB, M, N, K, alpha, A, l
                             activation, stream=None, check=True):
     return peak_gemm_fused(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation,
                            stream, check, variant)
+
+
+def peak_gemm_fused_residual(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation, R,
+                             ldr, stream=None, check=True, variant=None):
+    """C = act(alpha*op(A)*op(B) + beta*C + bias) + R; `variant` (optional) names the kernel family."""
+    lib = load()
+    if variant is None:
+        rc = lib.peak_gemm_fused_residual(dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A), lda, _ptr(B), ldb,
+                                          beta, _ptr(C), ldc, _ptr(bias), int(activation), _ptr(R), ldr, _stream(stream))
+    else:
+        rc = lib.peak_gemm_fused_residual_variant(int(variant), dtype, int(transA), int(transB), M, N, K, alpha, _ptr(A),
+                                                  lda, _ptr(B), ldb, beta, _ptr(C), ldc, _ptr(bias), int(activation),
+                                                  _ptr(R), ldr, _stream(stream))
+    return _raise(rc, "peak_gemm_fused_residual") if check else rc
+
+
+def peak_gemm_fused_residual_variant(variant, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias,
+                                     activation, R, ldr, stream=None, check=True):
+    return peak_gemm_fused_residual(dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, bias, activation,
+                                    R, ldr, stream, check, variant)
 
 
 def peak_gemm_strided_batched(dtype, transA, transB, M, N, K, alpha, A, lda, strideA, B, ldb, strideB, beta, C, ldc,

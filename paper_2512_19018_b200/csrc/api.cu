@@ -75,7 +75,7 @@ int validate(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K,
 // The dispatcher's choice, as a peak_variant_t (arguments already validated).
 int choose_variant(const GemmArgs &g) {
     if (g.M == 0 || g.N == 0) return PEAK_VARIANT_NONE;
-    const bool fused = g.bias != nullptr || g.act != PEAK_ACT_NONE;
+    const bool fused = g.bias != nullptr || g.act != PEAK_ACT_NONE || g.R != nullptr;
     if (g.K == 0 || g.alpha == 0.0f) return (g.beta == 1.0f && !fused) ? PEAK_VARIANT_NONE : PEAK_VARIANT_SCALE;
     if (in_elem(g.dtype) == Elem::F32) return sgemm_supports(g) ? PEAK_VARIANT_SGEMM : PEAK_VARIANT_FALLBACK;
     // CTA pairs (256-row tiles, B shared between the two SMs) win whenever there is more than one
@@ -124,13 +124,16 @@ int run_variant(int variant, const GemmArgs &g) {
 
 int gemm_impl(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,
               const void *A, int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, void *stream,
-              const float *bias = nullptr, int act = PEAK_ACT_NONE) {
+              const float *bias = nullptr, int act = PEAK_ACT_NONE, const void *R = nullptr, int64_t ldr = 0) {
     t_last_cuda_error = 0;
     int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
     if (rc != PEAK_OK) return rc;
     if (variant < PEAK_VARIANT_AUTO || variant > PEAK_VARIANT_NONE) return PEAK_ERR_INVALID_VALUE;
     if (act < PEAK_ACT_NONE || act > PEAK_ACT_GELU) return PEAK_ERR_INVALID_VALUE;
+    if (R && ldr < N) return PEAK_ERR_INVALID_VALUE;
     GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, C, lda, ldb, ldc, (cudaStream_t)stream, bias, act};
+    g.R = R;
+    g.ldr = ldr;
     const int chosen = choose_variant(g);
     int v = chosen;
     if (variant != PEAK_VARIANT_AUTO && chosen != PEAK_VARIANT_NONE && chosen != PEAK_VARIANT_SCALE) {
@@ -240,6 +243,21 @@ int peak_gemm_fused_variant(int variant, int dtype, int transA, int transB, int6
                             const float *bias, int activation, void *stream) {
     return gemm_impl(variant, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, stream, bias,
                      activation);
+}
+
+int peak_gemm_fused_residual(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const void *A,
+                             int64_t lda, const void *B, int64_t ldb, float beta, void *C, int64_t ldc, const float *bias,
+                             int activation, const void *R, int64_t ldr, void *stream) {
+    return gemm_impl(PEAK_VARIANT_AUTO, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, stream, bias,
+                     activation, R, ldr);
+}
+
+int peak_gemm_fused_residual_variant(int variant, int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K,
+                                     float alpha, const void *A, int64_t lda, const void *B, int64_t ldb, float beta,
+                                     void *C, int64_t ldc, const float *bias, int activation, const void *R, int64_t ldr,
+                                     void *stream) {
+    return gemm_impl(variant, dtype, transA, transB, M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, stream, bias,
+                     activation, R, ldr);
 }
 
 int peak_gemm_strided_batched(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha,

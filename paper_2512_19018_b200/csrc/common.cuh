@@ -60,6 +60,10 @@ __device__ __forceinline__ float finish_f32(float x, const float *bias, int64_t 
     if (bias) x += __ldg(bias + col);
     return activate_f32(x, act);
 }
+// ... and the residual operand, added after the activation (fp32, before the one output rounding)
+template <typename T> __device__ __forceinline__ float add_residual(float x, const T *R, int64_t idx) {
+    return R ? x + to_f32(R[idx]) : x;
+}
 
 // ---- host-side bookkeeping (api.cu owns the definitions) ---------------------------------------
 void count_launch(int n = 1);
@@ -82,6 +86,10 @@ struct GemmArgs {
     int act;            // fused epilogue: a peak_activation_t
     int64_t batch;      // strided batch: number of independent problems (0 or 1: a single GEMM)
     int64_t strideA, strideB, strideC;  // elements between consecutive matrices of the batch
+    // fused epilogue: residual matrix added after the activation (device, the output's storage type, M x N with
+    // pitch ldr), or nullptr
+    const void *R = nullptr;
+    int64_t ldr = 0;
     int64_t nbatch() const { return batch > 1 ? batch : 1; }
 };
 

@@ -15,7 +15,7 @@ template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(FB_THREADS)
 fallback_gemm_kernel(int transA, int transB, int64_t M, int64_t N, int64_t K, float alpha, const TIn *__restrict__ A,
                      int64_t lda, const TIn *__restrict__ B, int64_t ldb, float beta, TOut *__restrict__ C,
-                     int64_t ldc, const float *__restrict__ bias, int act) {
+                     int64_t ldc, const float *__restrict__ bias, int act, const TOut *__restrict__ R, int64_t ldr) {
     __shared__ float As[FB_BK][FB_TILE + 1];  // As[k][m]
     __shared__ float Bs[FB_BK][FB_TILE + 1];  // Bs[k][n]
     const int tid = threadIdx.x;
@@ -70,7 +70,8 @@ fallback_gemm_kernel(int transA, int transB, int64_t M, int64_t N, int64_t K, fl
             if (n >= N) continue;
             TOut *p = C + m * ldc + n;
             const float c_old = (beta != 0.0f) ? to_f32(*p) : 0.0f;
-            *p = from_f32<TOut>(finish_f32(epilogue_f32(alpha, acc[i][j], beta, c_old), bias, n, act));
+            *p = from_f32<TOut>(add_residual(finish_f32(epilogue_f32(alpha, acc[i][j], beta, c_old), bias, n, act), R,
+                                             m * ldr + n));
         }
     }
 }
@@ -98,12 +99,12 @@ __global__ void xcheck_f64_kernel(int transA, int transB, int64_t M, int64_t N, 
 // C = beta * C (beta == 0 stores zeros without reading C).
 template <typename TOut>
 __global__ void scale_kernel(int64_t M, int64_t N, float beta, TOut *__restrict__ C, int64_t ldc,
-                             const float *__restrict__ bias, int act) {
+                             const float *__restrict__ bias, int act, const TOut *__restrict__ R, int64_t ldr) {
     const int64_t total = M * N;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         TOut *p = C + (e / N) * ldc + (e % N);
         const float x = (beta == 0.0f) ? 0.0f : beta * to_f32(*p);
-        *p = from_f32<TOut>(finish_f32(x, bias, e % N, act));
+        *p = from_f32<TOut>(add_residual(finish_f32(x, bias, e % N, act), R, (e / N) * ldr + (e % N)));
     }
 }
 
@@ -112,7 +113,7 @@ template <typename TIn, typename TOut> int run_fallback(const GemmArgs &g) {
     if (grid.y > 65535u) return PEAK_ERR_UNSUPPORTED;
     fallback_gemm_kernel<TIn, TOut><<<grid, FB_THREADS, 0, g.stream>>>(
         g.transA, g.transB, g.M, g.N, g.K, g.alpha, (const TIn *)g.A, g.lda, (const TIn *)g.B, g.ldb, g.beta,
-        (TOut *)g.C, g.ldc, g.bias, g.act);
+        (TOut *)g.C, g.ldc, g.bias, g.act, (const TOut *)g.R, g.ldr);
     count_launch();
     note_kernel("fallback_gemm_kernel grid=%ux%u", grid.x, grid.y);
     cudaError_t e = cudaGetLastError();
@@ -138,7 +139,8 @@ template <typename TOut> int run_scale(const GemmArgs &g) {
     const int64_t total = g.M * g.N;
     int64_t blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    scale_kernel<TOut><<<(unsigned)blocks, 256, 0, g.stream>>>(g.M, g.N, g.beta, (TOut *)g.C, g.ldc, g.bias, g.act);
+    scale_kernel<TOut><<<(unsigned)blocks, 256, 0, g.stream>>>(g.M, g.N, g.beta, (TOut *)g.C, g.ldc, g.bias, g.act,
+                                                               (const TOut *)g.R, g.ldr);
     count_launch();
     note_kernel("scale_kernel grid=%u", (unsigned)blocks);
     cudaError_t e = cudaGetLastError();

@@ -32,6 +32,8 @@ struct peak_mc_request {
     int activation;         // fused epilogue: a peak_activation_t
     int epilogue_warps;     // PEAK_TUNE_EPILOGUE_WARPS value
     int tile_n;             // 256 (512 x 256 super-tiles) or 512 (512 x 512 super-tiles of two-half tiles)
+    const void *R;          // fused epilogue: residual matrix (output type, device) or NULL
+    int64_t ldr;
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

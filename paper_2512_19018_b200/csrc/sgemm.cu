@@ -51,7 +51,7 @@ template <bool TA, bool TB, bool PACKED>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
              int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int group,
-             const float *__restrict__ bias, int act) {
+             const float *__restrict__ bias, int act, const float *__restrict__ R, int64_t ldr) {
     __shared__ __align__(16) float As[2][SG_BK][SG_LD];
     __shared__ __align__(16) float Bs[2][SG_BK][SG_LD];
     const int tid = threadIdx.x;
@@ -132,6 +132,10 @@ sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int6
             r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), bias, n + 1, act);
             r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), bias, n + 2, act);
             r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), bias, n + 3, act);
+            if (R) {
+                const float4 q = *reinterpret_cast<const float4 *>(R + m * ldr + n);
+                r.x += q.x; r.y += q.y; r.z += q.z; r.w += q.w;
+            }
             *dst = r;
         }
     }
@@ -185,7 +189,8 @@ template <bool TA, bool TB, bool PACKED>
 __global__ void __launch_bounds__(SG_THREADS, 2)
 sgemm_async_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, float beta, float *__restrict__ C, int64_t ldc, int tiles_m,
-                   int tiles_n, int group, const float *__restrict__ bias, int act) {
+                   int tiles_n, int group, const float *__restrict__ bias, int act, const float *__restrict__ R,
+                   int64_t ldr) {
     extern __shared__ __align__(16) float sg_smem[];
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
@@ -265,6 +270,10 @@ sgemm_async_kernel(int M, int N, int K, float alpha, const float *__restrict__ A
             r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), bias, n + 1, act);
             r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), bias, n + 2, act);
             r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), bias, n + 3, act);
+            if (R) {
+                const float4 q = *reinterpret_cast<const float4 *>(R + m * ldr + n);
+                r.x += q.x; r.y += q.y; r.z += q.z; r.w += q.w;
+            }
             *dst = r;
         }
     }
@@ -281,7 +290,7 @@ template <bool TA, bool TB, bool PACKED> int run_sgemm_async(const GemmArgs &g) 
     const int group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 8;
     kernel<<<(unsigned)(tiles_m * tiles_n), SG_THREADS, SA_SMEM_BYTES, g.stream>>>(
         (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-        (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
+        (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act, (const float *)g.R, g.ldr);
     count_launch();
     note_kernel("sgemm_async_kernel<%d, %d, %d> grid=%d", (int)TA, (int)TB, (int)PACKED, tiles_m * tiles_n);
     cudaError_t e = cudaGetLastError();
@@ -300,11 +309,11 @@ template <bool TA, bool TB> int run_sgemm(const GemmArgs &g) {
     if (tuning(PEAK_TUNE_SGEMM_FMA) == 1)
         sgemm_kernel<TA, TB, false><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
             (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act, (const float *)g.R, g.ldr);
     else
         sgemm_kernel<TA, TB, true><<<(unsigned)(tiles_m * tiles_n), SG_THREADS, 0, g.stream>>>(
             (int)g.M, (int)g.N, (int)g.K, g.alpha, (const float *)g.A, g.lda, (const float *)g.B, g.ldb, g.beta,
-            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act);
+            (float *)g.C, g.ldc, tiles_m, tiles_n, group, g.bias, g.act, (const float *)g.R, g.ldr);
     count_launch();
     note_kernel("sgemm_kernel<%d, %d, %d> grid=%d", (int)TA, (int)TB, (int)(tuning(PEAK_TUNE_SGEMM_FMA) != 1),
                 tiles_m * tiles_n);
@@ -326,6 +335,7 @@ static bool sgemm_aligned_supports(const GemmArgs &g) {
     if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16 ||
         reinterpret_cast<uintptr_t>(g.C) % 16)
         return false;
+    if (g.R && (reinterpret_cast<uintptr_t>(g.R) % 16 || g.ldr % 4)) return false;  // read in 16-byte pieces
     return true;
 }
 

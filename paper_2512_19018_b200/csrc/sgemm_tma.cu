@@ -37,7 +37,9 @@ struct SgemmParams {
     int tiles_m, tiles_n, group;
     const float *bias;
     int act;
-    int vec_ok;  // C base and pitch allow 16-byte accesses
+    const float *R;  // residual added after the activation, or nullptr
+    int64_t ldr;
+    int vec_ok;  // C (and R) base and pitch allow 16-byte accesses
     long long wait_cycles;
     uint32_t *status;
 };
@@ -246,13 +248,18 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), p.bias, n + 1, p.act);
                     r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), p.bias, n + 2, p.act);
                     r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), p.bias, n + 3, p.act);
+                    if (p.R) {
+                        const float4 q = *reinterpret_cast<const float4 *>(p.R + (int64_t)m * p.ldr + n);
+                        r.x += q.x; r.y += q.y; r.z += q.z; r.w += q.w;
+                    }
                     *dst = r;
                 } else {
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         if (n + q < p.N) {
                             const float o = (beta != 0.0f) ? crow[n + q] : 0.0f;
-                            crow[n + q] = finish_f32(epilogue_f32(alpha, acc[i][4 * h + q], beta, o), p.bias, n + q, p.act);
+                            crow[n + q] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][4 * h + q], beta, o), p.bias, n + q, p.act),
+                                                       p.R, (int64_t)m * p.ldr + n + q);
                         }
                     }
                 }
@@ -263,7 +270,8 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n = n0 + tx + 16 * j;
                 if (n < p.N) {
                     const float o = (beta != 0.0f) ? crow[n] : 0.0f;
-                    crow[n] = finish_f32(epilogue_f32(alpha, acc[i][j], beta, o), p.bias, n, p.act);
+                    crow[n] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][j], beta, o), p.bias, n, p.act), p.R,
+                                           (int64_t)m * p.ldr + n);
                 }
             }
         }
@@ -296,7 +304,9 @@ template <bool A_KC, bool B_KC, int KG> int run_sgemm_tma(const GemmArgs &g) {
     p.tiles_n = (int)((g.N + ST_BN - 1) / ST_BN);
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 8;
     p.bias = g.bias; p.act = g.act;
-    p.vec_ok = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0 && g.ldc % 4 == 0) ? 1 : 0;
+    p.R = (const float *)g.R; p.ldr = g.ldr;
+    p.vec_ok = (reinterpret_cast<uintptr_t>(g.C) % 16 == 0 && g.ldc % 4 == 0 &&
+                (!g.R || (reinterpret_cast<uintptr_t>(g.R) % 16 == 0 && g.ldr % 4 == 0))) ? 1 : 0;
     const int wait_ms = tuning(PEAK_TUNE_WAIT_MS);
     p.wait_cycles = wait_ms > 0 ? (long long)wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
     p.status = device_status_word();

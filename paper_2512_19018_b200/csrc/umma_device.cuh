@@ -100,6 +100,9 @@ struct UmmaParams {
     int c_prefetch;        // beta != 0: old C chunks arrive by TMA in the staging buffers (one-slot tiles only)
     const float *bias;     // fused epilogue: fp32 value per column of C, or nullptr
     int act;               // fused epilogue: a peak_activation_t
+    const void *R;         // fused epilogue: residual (output type, M x N, pitch ldr) added after the activation
+    int64_t ldr;
+    int r_vec;             // R base and pitch allow 16-byte vector loads
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;
@@ -286,7 +289,8 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
                                               bool vec, float alpha, float beta, const float *bias, int act,
-                                              CFetch &cf, volatile uint32_t *abort_flag, long long wait_cycles) {
+                                              const T *rbase, int64_t ldr, bool rvec, CFetch &cf,
+                                              volatile uint32_t *abort_flag, long long wait_cycles) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
@@ -352,6 +356,13 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
             } else if (act == PEAK_ACT_GELU) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = activate_f32(v[i], PEAK_ACT_GELU);
+            }
+            if (rbase != nullptr && row < nrows && valid > 0) {
+                // residual: each thread reads its own row's contiguous run (the same access as old C without TMA)
+                float rr[32];
+                load_row32<T>(rbase + (int64_t)row * ldr + col, rr, valid, rvec);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] += rr[i];
             }
             if (tma) {
                 if (h == 0 && !cf.on) {
@@ -743,7 +754,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;
                     if (!epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc, row0 + lane, row0, p.M,
                                                          nh, p.N, &tmC, nh, row0, bz, p.tma_store != 0, vec, p.alpha,
-                                                         p.beta, p.bias, p.act, cf, abort_flag, p.wait_cycles)) {
+                                                         p.beta, p.bias, p.act, reinterpret_cast<const TOut *>(p.R),
+                                                         p.ldr, p.r_vec != 0, cf, abort_flag, p.wait_cycles)) {
                         if (lane == 0) report_timeout(p, abort_flag, 6, b);
                         ok = false;
                         break;
@@ -753,7 +765,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const int wrow0 = w.ws_block * (BM * CG) + (int)rank * BM + q * 32;
                     epilogue_tile<float, W>(t_addr, my_stage, lane, ws, (int64_t)BN, wrow0 + lane, wrow0,
                                             0x7fffffff, co, BN, &tmW, co, wrow0, 0, true, true, 1.0f, 0.0f, nullptr, 0,
-                                            no_cf, abort_flag, p.wait_cycles);
+                                            nullptr, 0, false, no_cf, abort_flag, p.wait_cycles);
                 }
                 // hand the accumulator slot back to the MMA issuer
                 ptx::tc_fence_before_sync();
@@ -791,7 +803,8 @@ template <typename TOut>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
                      int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
-                     int64_t stride_c, int vec_ok, const float *__restrict__ bias, int act) {
+                     int64_t stride_c, int vec_ok, const float *__restrict__ bias, int act,
+                     const TOut *__restrict__ R, int64_t ldr) {
     const int blocks_per_tile = gridDim.y;
     const int t = blockIdx.x;  // split tile number
     const int tiles_per_batch = tiles_m * tiles_n;
@@ -838,7 +851,8 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
             }
             float rr[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) rr[k] = finish_f32(epilogue_f32(alpha, a4[k], beta, o[k]), bias, j + k, act);
+            for (int k = 0; k < 4; ++k)
+                rr[k] = add_residual(finish_f32(epilogue_f32(alpha, a4[k], beta, o[k]), bias, j + k, act), R, i * ldr + j + k);
             if constexpr (sizeof(TOut) == 4) {
                 *reinterpret_cast<float4 *>(dst) = make_float4(rr[0], rr[1], rr[2], rr[3]);
             } else {
@@ -849,7 +863,8 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
             for (int k = 0; k < 4; ++k) {
                 if (j + k < N) {
                     const float c_old = (beta != 0.0f) ? to_f32(dst[k]) : 0.0f;
-                    dst[k] = from_f32<TOut>(finish_f32(epilogue_f32(alpha, a4[k], beta, c_old), bias, j + k, act));
+                    dst[k] = from_f32<TOut>(add_residual(finish_f32(epilogue_f32(alpha, a4[k], beta, c_old), bias, j + k, act),
+                                                         R, i * ldr + j + k));
                 }
             }
         }

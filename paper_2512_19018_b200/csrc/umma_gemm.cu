@@ -157,6 +157,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.C = g.C; p.ldc = g.ldc;
     p.bias = g.bias; p.act = g.act;
     const int ob = elem_bytes(eout);
+    if (g.R && nb > 1) return PEAK_ERR_UNSUPPORTED;  // no residual on the batched path
+    p.R = g.R; p.ldr = g.ldr;
+    p.r_vec = (g.R && reinterpret_cast<uintptr_t>(g.R) % 16 == 0 && (g.ldr * ob) % 16 == 0) ? 1 : 0;
     p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0 &&
                 (nb == 1 || (g.strideC * ob) % 16 == 0)) ? 1 : 0;
     const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
@@ -227,7 +230,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const float *ws_c = ws;
     e = cudaLaunchKernelEx(&rcfg, splitk_reduce_kernel<TOut>, ws_c, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
                            p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C, g.ldc, g.strideC, p.vec_ok,
-                           g.bias, g.act);
+                           g.bias, g.act, (const TOut *)g.R, g.ldr);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
@@ -419,7 +422,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
                               tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act,
-                              tuning(PEAK_TUNE_EPILOGUE_WARPS), mc_tile_n, 0};
+                              tuning(PEAK_TUNE_EPILOGUE_WARPS), mc_tile_n, g.R, g.ldr, 0};
             if (!r.status) return PEAK_ERR_CUDA;
             const int rc = mc_entry()(&r);
             if (rc == PEAK_OK) {

@@ -97,6 +97,8 @@ template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(
     p.C = r->C; p.ldc = r->ldc;
     p.bias = r->bias; p.act = r->activation;
     const int ob = elem_bytes(eout);
+    p.R = r->R; p.ldr = r->ldr;
+    p.r_vec = (r->R && reinterpret_cast<uintptr_t>(r->R) % 16 == 0 && (r->ldr * ob) % 16 == 0) ? 1 : 0;
     p.vec_ok = ((reinterpret_cast<uintptr_t>(r->C) % 16) == 0 && (r->ldc * ob) % 16 == 0) ? 1 : 0;
     p.tma_store = (p.vec_ok && (r->N * ob) % 16 == 0 && r->epilogue != 1) ? 1 : 0;
     tmC = tmA;

@@ -413,3 +413,32 @@ def test_fp8_gemm_exact_integers(oracle):
         ref, S = oracle.gemm(t, oracle.F32, 0, 1, M, N, K, 1.0, A, K, B, K, 0.0, None, N)
         assert np.array_equal(ref, (a @ b.T).astype(np.float64))
         assert np.array_equal(S, (np.abs(a) @ np.abs(b).T).astype(np.float64))
+
+
+@pytest.mark.parametrize("t", ["f16", "bf16", "f32"])
+def test_residual_add_matches_library_decode(oracle, t):
+    """The residual operand of the fused tail: x + R with R decoded from its stored bits, padded pitch honoured.
+    Checked against numpy addition of library-decoded values (exact: one fp64 addition either way), on random
+    bit patterns that include subnormals and infinities, and against a misplaced pitch."""
+    rng = np.random.default_rng(90)
+    rows, cols, ldr = 13, 21, 29
+    x = rng.standard_normal((rows, cols))
+    if t == "f32":
+        R = rng.standard_normal((rows, ldr)).astype(np.float32)
+        R[0, :4] = [np.float32(1e-42), np.float32(-3e38), np.inf, -0.0]
+        vals = R.astype(np.float64)
+    else:
+        R = rng.integers(0, 1 << 16, size=(rows, ldr), dtype=np.uint64).astype(np.uint16)
+        vals = W.to_float64(R, t)
+    got = oracle.residual_add(x, R, T[t], ldr)
+    with np.errstate(invalid="ignore"):
+        want = x + vals[:, :cols]
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan) and np.array_equal(got[~nan], want[~nan])
+    assert not np.array_equal(np.nan_to_num(got), np.nan_to_num(x))
+    # a wrong pitch would read other elements: the dense copy with ldr = cols must agree as well
+    dense = np.ascontiguousarray(R[:, :cols])
+    got2 = oracle.residual_add(x, dense, T[t], cols)
+    assert np.array_equal(np.isnan(got2), nan) and np.array_equal(got2[~nan], want[~nan])
+    with pytest.raises(ValueError):
+        oracle.residual_add(x, R, T[t], cols - 1)
