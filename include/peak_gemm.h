@@ -302,6 +302,27 @@ typedef enum peak_tuning_key {
 int peak_set_tuning(int key, int value);
 
 /*
+ * Persisted tuning table (the paper's performance evaluator, section 3.3 -- enumerate the tuning-parameter
+ * combinations, prune, keep the best -- with its result kept in a file).  `python -m paper_2512_19018_b200.tune
+ * --sweep` times the candidates for each benchmark shape class and writes tuned_sm100.json; the library reads
+ * that file (beside the shared object, or the file named by the environment variable PEAK_TUNED_TABLE; the
+ * values "off", "0" and "none" disable the table) on first use.  For a problem of the same types, layout and
+ * beta class (zero / non-zero) whose M, N and K each lie within a factor sqrt(2) of an entry's, the entry's
+ * kernel family and knob values replace the dispatcher's built-in rules; knobs set through peak_set_tuning
+ * still win, and results never depend on any of this.
+ *   peak_tuned_table_load     replaces the table with the file at `path` (host string); NULL or "" empties it.
+ *                             Returns the number of entries, -1 if the file is not understood, -2 if it
+ *                             cannot be opened (the current table then stays).
+ *   peak_tuned_table_entries  entries in the table now (loads the default file on first use).
+ *   peak_tuned_lookup         1 and the entry's family (`variant`, 0 = none named) and knob values (`knobs`,
+ *                             PEAK_TUNE_COUNT_ ints) when an entry covers the problem, else 0.  Host only.
+ */
+int peak_tuned_table_load(const char *path);
+int peak_tuned_table_entries(void);
+int peak_tuned_lookup(int dtype, int transA, int transB, int64_t M, int64_t N, int64_t K, float beta, int *variant,
+                      int *knobs);
+
+/*
  * peak_multicast_available: 1 when the optional single-GPU plug-in (libpeak_gemm_mc.so, beside the main
  * library) is present and loaded.  It runs large 16-bit GEMMs with clusters of four CTAs that share B tiles
  * through TMA multicast (the paper's thread-block tiling taken one level up: a cluster-level tile); results

@@ -25,7 +25,8 @@ EXPORTS = ["peak_gemm", "peak_gemm_variant", "peak_gemm_host", "peak_release_sta
            "peak_query_variant", "peak_tile_coord", "peak_set_tuning", "peak_check", "peak_kernel_launches", "peak_last_cuda_error",
            "peak_status_string", "peak_variant_string", "peak_version", "peak_gemm_static_ws", "peak_static_ws_bytes", "peak_multicast_available", "peak_gemm_fused",
            "peak_gemm_fused_variant", "peak_gemm_strided_batched", "peak_last_kernel", "peak_selftest_per_device_once",
-           "peak_gemm_fused_residual", "peak_gemm_fused_residual_variant"]
+           "peak_gemm_fused_residual", "peak_gemm_fused_residual_variant", "peak_tuned_table_load",
+           "peak_tuned_table_entries", "peak_tuned_lookup"]
 
 
 class PeakError(RuntimeError):
@@ -92,6 +93,12 @@ def load():
     lib.peak_last_kernel.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
     lib.peak_selftest_per_device_once.restype = i
     lib.peak_selftest_per_device_once.argtypes = []
+    lib.peak_tuned_table_load.restype = i
+    lib.peak_tuned_table_load.argtypes = [ctypes.c_char_p]
+    lib.peak_tuned_table_entries.restype = i
+    lib.peak_tuned_table_entries.argtypes = []
+    lib.peak_tuned_lookup.restype = i
+    lib.peak_tuned_lookup.argtypes = [i, i, i, i64, i64, i64, f, ctypes.POINTER(i), ctypes.POINTER(i)]
     lib.peak_status_string.restype = ctypes.c_char_p
     lib.peak_status_string.argtypes = [i]
     lib.peak_variant_string.restype = ctypes.c_char_p
@@ -271,6 +278,24 @@ def peak_last_kernel() -> str:
 
 def peak_selftest_per_device_once() -> int:
     return load().peak_selftest_per_device_once()
+
+
+def peak_tuned_table_load(path) -> int:
+    """Replace the tuning table with the JSON file at `path` (None / "" empties it); returns the entry count."""
+    return load().peak_tuned_table_load(None if not path else os.fsencode(path))
+
+
+def peak_tuned_table_entries() -> int:
+    return load().peak_tuned_table_entries()
+
+
+def peak_tuned_lookup(dtype, transA, transB, M, N, K, beta):
+    """(variant, {key: value}) of the table entry that covers the problem, or None."""
+    v = ctypes.c_int(0)
+    knobs = (ctypes.c_int * PEAK_TUNE_COUNT)()
+    if not load().peak_tuned_lookup(dtype, int(transA), int(transB), M, N, K, beta, ctypes.byref(v), knobs):
+        return None
+    return v.value, {k: knobs[k] for k in range(PEAK_TUNE_COUNT) if knobs[k]}
 
 
 def peak_status_string(status: int) -> str:

@@ -15,7 +15,7 @@ LIB = os.path.join(HERE, "libpeak_gemm.so")
 # optional single-GPU plug-in (cluster-multicast loads): built only where its source is present
 MC_SOURCE = os.path.join(CSRC, "umma_gemm_mc.cu")
 MC_LIB = os.path.join(HERE, "libpeak_gemm_mc.so")
-SOURCES = ["api.cu", "fallback_gemm.cu", "sgemm.cu", "sgemm_tma.cu", "umma_gemm.cu"]
+SOURCES = ["api.cu", "fallback_gemm.cu", "sgemm.cu", "sgemm_tma.cu", "tuned_table.cu", "umma_gemm.cu"]
 HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "ptx.cuh", "umma_device.cuh", "umma_host.cuh", "mc_plugin.h")] + [
     os.path.join(os.path.dirname(HERE), "include", "peak_gemm.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

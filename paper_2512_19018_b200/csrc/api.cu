@@ -26,7 +26,11 @@ std::mutex g_status_mutex;
 namespace {
 std::atomic<int> g_tuning[PEAK_TUNE_COUNT_];
 }
-int tuning(int key) { return (key >= 0 && key < PEAK_TUNE_COUNT_) ? g_tuning[key].load(std::memory_order_relaxed) : 0; }
+int tuning(int key) {
+    if (key < 0 || key >= PEAK_TUNE_COUNT_) return 0;
+    const int v = g_tuning[key].load(std::memory_order_relaxed);
+    return v != 0 ? v : tuned_knob(key);  // what the caller set wins; else the tuning table's entry, if any
+}
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 namespace {
@@ -83,6 +87,10 @@ int choose_variant(const GemmArgs &g) {
     // tiles: a problem whose 256 x 256 pair tiles would occupy at most half of the SM pairs runs as
     // single-CTA tiles instead, which spread it over up to four times as many SMs (measured 6-13 % faster
     // from 512^3 to 1536^3, 1024x2048x1024, 256x4096x4096).
+    const int tv = tuned_variant();  // the tuning table's preference, honoured when that family can run the problem
+    if ((tv == PEAK_VARIANT_UMMA_1CTA || tv == PEAK_VARIANT_UMMA_2CTA) && umma_supports(g, tv == PEAK_VARIANT_UMMA_2CTA ? 2 : 1) &&
+        (tv == PEAK_VARIANT_UMMA_1CTA || g.M > 128))
+        return tv;
     if (umma_supports(g, 2) && g.M > 128) {
         const int64_t pair_tiles = ((g.M + 255) / 256) * ((g.N + 255) / 256) * g.nbatch();
         if (2 * pair_tiles > umma_units(2) || !umma_supports(g, 1)) return PEAK_VARIANT_UMMA_2CTA;
@@ -134,6 +142,7 @@ int gemm_impl(int variant, int dtype, int transA, int transB, int64_t M, int64_t
     GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, C, lda, ldb, ldc, (cudaStream_t)stream, bias, act};
     g.R = R;
     g.ldr = ldr;
+    TunedScope tuned(g);
     const int chosen = choose_variant(g);
     int v = chosen;
     if (variant != PEAK_VARIANT_AUTO && chosen != PEAK_VARIANT_NONE && chosen != PEAK_VARIANT_SCALE) {
@@ -436,6 +445,7 @@ int peak_query_variant(int dtype, int transA, int transB, int64_t M, int64_t N, 
     int rc = validate(dtype, transA, transB, M, N, K, A, lda, B, ldb, alpha, beta, C, ldc);
     if (rc != PEAK_OK) return -rc;
     GemmArgs g{dtype, transA, transB, M, N, K, alpha, beta, A, B, const_cast<void *>(C), lda, ldb, ldc, nullptr};
+    TunedScope tuned(g);
     return choose_variant(g);
 }
 

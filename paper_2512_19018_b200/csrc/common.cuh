@@ -119,6 +119,17 @@ inline int current_device() {
     return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
 }
 
+// Persisted tuning table (tuned_table.cu): while a TunedScope lives, tuning() answers knobs the caller left at
+// 0 from the table entry that covers the problem, and tuned_variant() names the family that entry prefers.
+struct TunedScope {
+    explicit TunedScope(const GemmArgs &g);
+    ~TunedScope();
+    TunedScope(const TunedScope &) = delete;
+    TunedScope &operator=(const TunedScope &) = delete;
+};
+int tuned_knob(int key);
+int tuned_variant();
+
 // kernel-family launchers; each returns a peak_status_t
 int launch_fallback(const GemmArgs &g);
 int launch_scale(const GemmArgs &g);

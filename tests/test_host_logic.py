@@ -153,8 +153,9 @@ def test_tuner_enumerates_and_prunes():
     assert len(cands) > 20 and len(set((v, tuple(sorted(k.items()))) for v, k in cands)) == len(cands)
     for v, k in cands:
         assert not (v == "umma_1cta" and k.get(1) == 512)             # wide tiles need CTA pairs
-        assert not (k.get(10) == 2 and k.get(1) != 256)                # the plug-in runs 256-wide tiles only
+        assert not (k.get(10) == 2 and k.get(1) == 128)                # the plug-in runs 256- and 512-wide tiles
         assert not (k.get(2, 1) > 1 and k.get(1) == 512)
+    assert any(k.get(10) == 2 and k.get(1) == 512 for v, k in cands)  # ... so the 512-wide plug-in kernel is timed
     # a k-split cannot have more slices than k-blocks
     assert not tune.prune("umma_2cta", {1: 256, 2: 8, 3: 2, 10: 1, 0: 0}, 256, 256, 128)
     assert len(list(tune.candidates(tune.SPACE_F32, quick=True))) == 8
@@ -189,3 +190,52 @@ def test_bench_rotation_rule():
     assert bench.rotation_sets(table["bf16_8192_nn"]) == 1 and "larger than L2" in bench.l2_note(table["bf16_8192_nn"])
     n = bench.rotation_sets(table["bf16_4096_nn"])
     assert n >= 4 and n * bench.set_bytes(table["bf16_4096_nn"]) > 3 * bench.L2_BYTES
+
+
+def test_tuning_table_is_loaded_matched_and_overridable(tmp_path):
+    """The persisted tuning table: a (fake) table changes the dispatcher's visible choice exactly for the
+    problems its entry covers; knobs it may not set are dropped; emptying it restores the built-in rules;
+    a file that cannot be read or understood leaves the current table alone."""
+    import json
+    al = 1 << 20
+    q = lambda M, N, K, beta=0.0, dt=P.PEAK_BF16_BF16: P.peak_query_variant(dt, 0, 0, M, N, K, 1.0, al, K, al, N, beta, al, N)
+    default_file = os.path.join(os.path.dirname(P.LIB_PATH), "tuned_sm100.json")
+    try:
+        assert P.peak_tuned_table_load(None) == 0 and P.peak_tuned_table_entries() == 0
+        assert q(4096, 4096, 4096) == P.PEAK_VARIANT_UMMA_2CTA
+        fake = {"format": 1, "note": "test", "entries": [
+            {"in": "bf16", "out": "bf16", "layout": "NN", "beta": 0, "M": 4096, "N": 4096, "K": 4096,
+             "variant": "umma_1cta", "knobs": {"1": 128, "0": 4, "8": 5, "9": 1}, "tflops": 1.0},
+            {"in": "bf16", "out": "bf16", "layout": "NX?", "M": 1, "N": 1, "K": 1},          # malformed: skipped
+            {"in": "f32", "out": "f32", "layout": "NN", "beta": 1, "M": 512, "N": 512, "K": 512, "knobs": {"7": 2}}]}
+        path = tmp_path / "table.json"
+        path.write_text(json.dumps(fake))
+        assert P.peak_tuned_table_load(str(path)) == 2 and P.peak_tuned_table_entries() == 2
+        assert q(4096, 4096, 4096) == P.PEAK_VARIANT_UMMA_1CTA           # the entry's family
+        assert q(5000, 3000, 4096) == P.PEAK_VARIANT_UMMA_1CTA           # within sqrt(2) of the entry in every dimension
+        assert q(8192, 8192, 8192) == P.PEAK_VARIANT_UMMA_2CTA           # outside: built-in rule
+        assert q(4096, 4096, 4096, beta=1.0) == P.PEAK_VARIANT_UMMA_2CTA  # other beta class
+        assert q(4096, 4096, 4096, dt=P.PEAK_BF16_F32) == P.PEAK_VARIANT_UMMA_2CTA
+        v, knobs = P.peak_tuned_lookup(P.PEAK_BF16_BF16, 0, 0, 4096, 4096, 4096, 0.0)
+        assert v == P.PEAK_VARIANT_UMMA_1CTA and knobs == {P.PEAK_TUNE_TILE_N: 128, P.PEAK_TUNE_RASTER_GROUP: 4}
+        assert P.peak_tuned_lookup(P.PEAK_BF16_BF16, 0, 0, 4096, 4096, 16384, 0.0) is None
+        v, knobs = P.peak_tuned_lookup(P.PEAK_F32_F32, 0, 0, 600, 400, 512, 2.0)
+        assert v == 0 and knobs == {P.PEAK_TUNE_SGEMM_COPY: 2}
+        bad = tmp_path / "bad.json"
+        bad.write_text("{\"entries\": [1, 2")
+        assert P.peak_tuned_table_load(str(bad)) == -1 and P.peak_tuned_table_entries() == 2
+        assert P.peak_tuned_table_load(str(tmp_path / "missing.json")) == -2 and P.peak_tuned_table_entries() == 2
+        assert P.peak_tuned_table_load("") == 0
+        assert q(4096, 4096, 4096) == P.PEAK_VARIANT_UMMA_2CTA
+    finally:
+        P.peak_tuned_table_load(default_file if os.path.exists(default_file) else None)
+
+
+def test_shipped_tuning_table_parses():
+    """The table that ships with the package (written by the sweep) is understood by the library's reader."""
+    import json
+    path = os.path.join(os.path.dirname(P.LIB_PATH), "tuned_sm100.json")
+    if not os.path.exists(path):
+        pytest.skip("no tuned_sm100.json in the package")
+    n = len(json.load(open(path))["entries"])
+    assert P.peak_tuned_table_load(path) == n
