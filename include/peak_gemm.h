@@ -297,7 +297,10 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_EPILOGUE_WARPS = 12, /* one-slot (128- / 256-wide) tiles: 1 = one group of four epilogue warps, 2 = two
                                       groups that drain half of the columns each (default: two for problems of at
                                       most two waves) */
-    PEAK_TUNE_COUNT_ = 13
+    PEAK_TUNE_K_ORDER = 13,     /* tensor-core kernels: 1 = every tile walks its k-blocks upwards, 2 = every other tile
+                                   of a CTA walks them downwards, so that a wave of tiles starts in the k-range the
+                                   previous wave left in L2 (default: 2 for 512-wide tiles, 1 otherwise) */
+    PEAK_TUNE_COUNT_ = 14
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

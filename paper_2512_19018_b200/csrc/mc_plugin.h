@@ -34,6 +34,7 @@ struct peak_mc_request {
     int tile_n;             // 256 (512 x 256 super-tiles) or 512 (512 x 512 super-tiles of two-half tiles)
     const void *R;          // fused epilogue: residual matrix (output type, device) or NULL
     int64_t ldr;
+    int k_order;            // PEAK_TUNE_K_ORDER value
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

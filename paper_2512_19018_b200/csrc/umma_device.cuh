@@ -103,6 +103,7 @@ struct UmmaParams {
     const void *R;         // fused epilogue: residual (output type, M x N, pitch ldr) added after the activation
     int64_t ldr;
     int r_vec;             // R base and pitch allow 16-byte vector loads
+    int k_alternate;       // 1: every other item of a CTA walks its k-blocks downwards (L2 reuse across waves)
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;
@@ -504,23 +505,30 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, tl = 0;
             bool ok = true;
-            for (int item = unit; item < total_items && ok; item += num_units) {
+            for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
                 const Item w = decode_item(p, item);
+                // Every other item walks k downwards.  All CTAs are at about the same k at any time, so what L2
+                // holds when a wave of tiles ends is the k-range that was read last; a next wave that starts there
+                // (instead of at k = 0, whose panels were read longest ago and are gone) finds the panels it shares
+                // with the previous wave still cached.  The order in which k-blocks are accumulated changes
+                // with it, but it is a fixed function of the launch, so results stay run-to-run identical.
+                const bool rev = p.k_alternate && (tl & 1u);
                 const int bz = BATCHED ? w.tile / p.tiles_per_batch : 0;  // matrix of the batch
                 int64_t tm, tn;
                 tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
                 const int n_cta = (int)tn * BN + (int)rank * C_::HROWS;  // first B row of this CTA (half 0)
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                for (int j = 0, nk = w.kb1 - w.kb0; j < nk; ++j, ++it) {
+                    const int kb = rev ? w.kb1 - 1 - j : w.kb0 + j;
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
                         report_timeout(p, abort_flag, 1, s);
                         ok = false;
                         break;
                     }
-                    if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && kb == w.kb1 - 1)
+                    if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && j == nk - 1)
                         continue;  // test hook: leave this stage empty so that the waits downstream run out
                     uint32_t bar = full0 + 8 * s;
                     if (leader) ptx::mbar_arrive_expect_tx(bar, (uint32_t)(C_::STAGE_BYTES * CG));

@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 13
+NUM_KEYS = 14
 
 
 def candidates(space: dict, quick: bool = False):
@@ -77,6 +77,7 @@ AXES_TENSOR = [
     (2, [0, 1, 2, 3, 4, 8]),        # PEAK_TUNE_SPLIT_K
     (11, [0, 1]),                   # PEAK_TUNE_BALANCED_GRID
     (3, [0, 1, 2]),                 # PEAK_TUNE_EPILOGUE
+    (13, [0, 1, 2]),                # PEAK_TUNE_K_ORDER
 ]
 AXES_F32 = [
     ("variant", ["auto"]),

@@ -658,3 +658,25 @@ def test_cuda_graph_with_k_split_and_several_calls():
         assert P.peak_check()[0] == P.PEAK_OK
         for dc in dcs:
             R.check_full(dc, what=f"graph replay {rep} {dc.case.name}")
+
+
+@pytest.mark.parametrize("variant", UMMA)
+def test_alternating_k_order_is_exact_and_repeatable(variant, reset_tuning):
+    """Every other tile of a CTA walks its k-blocks downwards (PEAK_TUNE_K_ORDER = 2): on integer inputs the
+    result is still exact, whatever the tile width, k-split or layout, on problems of several tiles per CTA with a
+    ragged K tail; and two runs give identical bits."""
+    P.peak_set_tuning(P.PEAK_TUNE_K_ORDER, 2)
+    for idx, (ta, tb, M, N, K, bn, split) in enumerate([(0, 0, 2304, 3328, 1000, 0, 0), (1, 0, 2048, 4096, 712, 128, 0),
+                                                        (0, 1, 3072, 2560, 1544, 512, 0), (1, 1, 1024, 1536, 2056, 256, 3)]):
+        P.peak_set_tuning(P.PEAK_TUNE_TILE_N, bn)
+        P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+        c = mk(W.PEAK_BF16_F32, ta, tb, M, N, K, dist="smallint", alpha=1.0, beta=-1.0, case=idx)
+        dc = R.DeviceCase(c)
+        dc.run(variant)
+        first = dc.result().copy()
+        ref, _ = dc.oracle_sub(*R.sample_grid(c, 128, 128, 3e8))
+        rows, cols = R.sample_grid(c, 128, 128, 3e8)
+        assert np.array_equal(first[np.ix_(rows, cols)].view(np.uint32), oracle.round_to(oracle.F32, ref)), f"{c}"
+        dc.reset_c()
+        dc.run(variant)
+        assert np.array_equal(dc.result(), first)
