@@ -165,8 +165,12 @@ def profile_traffic(workload: str, launched: str):
             continue
         have = _kernel_key(km.group(1))
         seen.append(km.group(1).strip()[:80])
-        same = bool(want and have and want[0] == have[0] and len(want[1]) == len(have[1]) and
-                    all(a == b or "*" in (a, b) for a, b in zip(want[1], have[1])))
+        # template arguments compare position by position ("*" = any); a list that is shorter than the other
+        # (a summary taken before the kernel gained a trailing flag) matches when the extra arguments are 0
+        n = min(len(want[1]), len(have[1])) if want and have else 0
+        same = bool(want and have and want[0] == have[0] and
+                    all(a == b or "*" in (a, b) for a, b in zip(want[1][:n], have[1][:n])) and
+                    all(x in ("0", "*") for x in want[1][n:] + have[1][n:]))
         if same:
             total = float(rd.group(1)) * _UNIT[rd.group(2)] + float(wr.group(1)) * _UNIT[wr.group(2)]
             return total, f"quoted from {os.path.relpath(path, ROOT)} (one ncu capture; not measured in this run)"

@@ -300,7 +300,10 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_K_ORDER = 13,     /* tensor-core kernels: 1 = every tile walks its k-blocks upwards, 2 = every other tile
                                    of a CTA walks them downwards, so that a wave of tiles starts in the k-range the
                                    previous wave left in L2 (default: 2 for 512-wide tiles, 1 otherwise) */
-    PEAK_TUNE_COUNT_ = 14
+    PEAK_TUNE_SWAP_AB = 14,     /* problems with M <= 64 (single-CTA tiles, 16-bit inputs): computed as C^T = op(B)^T
+                                   op(A)^T, so that M is the narrow side of the tensor-core tile, when set to 2
+                                   (default: off -- it measured slower than the plain tiles on B200) */
+    PEAK_TUNE_COUNT_ = 15
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

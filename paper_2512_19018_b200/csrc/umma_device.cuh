@@ -392,6 +392,39 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
     return true;
 }
 
+// Epilogue of a tile computed with the operands exchanged (C^T = op(B)^T op(A)^T: the accumulator's rows are
+// columns n of C, its columns are rows m): each thread owns one n and walks the m of the tile, so for a fixed m
+// the 32 lanes of a warp touch 32 consecutive elements of a row of C -- coalesced without staging.  Bias is
+// per column of C, i.e. one value per thread; the residual is read the same way as old C.
+template <typename T, int W>
+__device__ __forceinline__ void epilogue_tile_swapped(uint32_t t_addr, T *C, int64_t ldc, int n, int n_limit, int m0,
+                                                      int m_limit, float alpha, float beta, const float *bias, int act,
+                                                      const T *R, int64_t ldr) {
+#pragma unroll 1
+    for (int c = 0; c < W / 32; ++c) {
+        const int mc = m0 + c * 32;
+        if (mc >= m_limit) break;  // warp-uniform
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(t_addr + c * 32, r);
+        ptx::tmem_ld_wait();
+        if (n < n_limit) {
+            const float b = bias ? __ldg(bias + n) : 0.0f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int m = mc + i;
+                if (m < m_limit) {
+                    T *dst = C + (int64_t)m * ldc + n;
+                    float x = alpha * __uint_as_float(r[i]);
+                    if (beta != 0.0f) x = fmaf(beta, to_f32(*dst), x);
+                    x = activate_f32(x + b, act);
+                    if (R) x += to_f32(R[(int64_t)m * ldr + n]);
+                    *dst = from_f32<T>(x);
+                }
+            }
+        }
+    }
+}
+
 // Tile copies: a single GEMM uses two-dimensional descriptors, a strided batch three-dimensional ones.  The
 // choice is a template parameter of the kernel: the single-GEMM instantiation carries no trace of the batch
 // (three-dimensional descriptors with a batch of one, or a run-time choice, measured 1-10 % slower).
@@ -425,7 +458,10 @@ template <> struct McOps<0> {
 // G2: a one-slot tile is drained by two groups of four epilogue warps, each taking half of the columns.  The
 // epilogue of such a tile hides behind the next tile's main loop, so the second group only pays when there is
 // no next tile: problems of at most two waves, where it shortens the exposed tail of the launch.
-template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false, bool G2 = false>
+// SWAP: the caller exchanged the operands (the kernel's M is the problem's N and the other way round, see
+// launch_swapped): whole tiles are written transposed, straight from registers.
+template <int CG, int BN, typename TOut, int MC = 0, bool BATCHED = false, bool IN8 = false, bool G2 = false,
+          bool SWAP = false>
 __global__ void __launch_bounds__((Cfg<CG, BN>::threads(G2)), 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmW,
@@ -756,6 +792,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nh = n0 + co;
                 if (!live) {
                     // rows beyond M: the partial-tile reduction and C never look at them
+                } else if (SWAP && w.ws_block < 0) {
+                    // whole tile of C^T: this thread's accumulator row is column n = row0 + lane of C
+                    epilogue_tile_swapped<TOut, W>(t_addr, reinterpret_cast<TOut *>(p.C), p.ldc, row0 + lane, p.M, nh,
+                                                   p.N, p.alpha, p.beta, p.bias, p.act,
+                                                   reinterpret_cast<const TOut *>(p.R), p.ldr);
                 } else if (w.ws_block < 0) {
                     // whole tile: alpha/beta epilogue straight to C
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
@@ -812,7 +853,9 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, int tiles_m, int tiles_n, int group,
                      int rows_t, int bn, int M, int N, float alpha, float beta, TOut *__restrict__ C, int64_t ldc,
                      int64_t stride_c, int vec_ok, const float *__restrict__ bias, int act,
-                     const TOut *__restrict__ R, int64_t ldr) {
+                     const TOut *__restrict__ R, int64_t ldr, int trans) {
+    // trans: the tiles are tiles of C^T (operands exchanged): element (i, j) of the tile grid is C[j][i], the bias
+    // belongs to i, and nothing is vectorised
     const int blocks_per_tile = gridDim.y;
     const int t = blockIdx.x;  // split tile number
     const int tiles_per_batch = tiles_m * tiles_n;
@@ -842,6 +885,18 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
         const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+        if (trans) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (j + k < N) {
+                    TOut *d = C + (j + k) * ldc + i;
+                    const float c_old = (beta != 0.0f) ? to_f32(*d) : 0.0f;
+                    *d = from_f32<TOut>(add_residual(finish_f32(epilogue_f32(alpha, a4[k], beta, c_old), bias, i, act), R,
+                                                     (j + k) * ldr + i));
+                }
+            }
+            continue;
+        }
         TOut *dst = C + i * ldc + j;
         if (vec_ok && j + 4 <= N) {
             float o[4] = {0.f, 0.f, 0.f, 0.f};

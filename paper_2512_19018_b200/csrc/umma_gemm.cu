@@ -3,6 +3,7 @@
 // The kernels are in umma_device.cuh.
 #include <cuda.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "common.cuh"
@@ -108,11 +109,12 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     return best;
 }
 
-template <int CG, int BN, typename TOut, bool BATCHED, bool IN8 = false, bool G2 = false>
+// SWAP: `g` already has its operands exchanged (see launch_swapped); g.C / g.ldc / g.R / g.bias are the caller's.
+template <int CG, int BN, typename TOut, bool BATCHED, bool IN8 = false, bool G2 = false, bool SWAP = false>
 int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws) {
     using C_ = Cfg<CG, BN>;
     constexpr int BKE = IN8 ? 2 * BK : BK;  // elements per k-block
-    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8, G2>;
+    auto kernel = umma_gemm_kernel<CG, BN, TOut, 0, BATCHED, IN8, G2, SWAP>;
     static PerDeviceOnce attr_once;  // the attribute belongs to the device's context: once per device
     const cudaError_t attr_err = attr_once.run(current_device(), [&] {
         return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
@@ -174,7 +176,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const int epi = tuning(PEAK_TUNE_EPILOGUE);  // 0 auto, 1 direct stores, 2 TMA stores
     // TMA stores clip rows exactly but clip the contiguous index only at 16-byte granularity, so they are
     // used when a row of C is a whole number of 16-byte pieces; other widths take the direct-store path
-    p.tma_store = (p.vec_ok && (g.N * ob) % 16 == 0 && epi != 1) ? 1 : 0;
+    p.tma_store = (p.vec_ok && (g.N * ob) % 16 == 0 && epi != 1 && !SWAP) ? 1 : 0;
     tmC = tmA;  // placeholders when unused
     tmW = tmA;
     if (nb > 1 && (g.strideC * ob) % 16 != 0) p.tma_store = 0;  // the batch stride must suit the store map too
@@ -222,9 +224,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, tmW, ws, p);
     count_launch();
-    note_kernel("umma_gemm_kernel<%d, %d, %s, 0, %d, %d, %d> grid=%d items=%d splits=%d", CG, BN,
+    note_kernel("umma_gemm_kernel<%d, %d, %s, 0, %d, %d, %d, %d> grid=%d items=%d splits=%d", CG, BN,
                 sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"),
-                (int)BATCHED, (int)IN8, (int)G2, units * CG, p.total_items, plan.tail_splits);
+                (int)BATCHED, (int)IN8, (int)G2, (int)SWAP, units * CG, p.total_items, plan.tail_splits);
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     if (plan.full_tiles == tiles) return PEAK_OK;
 
@@ -243,7 +245,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     const float *ws_c = ws;
     e = cudaLaunchKernelEx(&rcfg, splitk_reduce_kernel<TOut>, ws_c, plan.tail_splits, plan.full_tiles, p.tiles_m, p.tiles_n,
                            p.group, BM * CG, BN, p.M, p.N, g.alpha, g.beta, (TOut *)g.C, g.ldc, g.strideC, p.vec_ok,
-                           g.bias, g.act, (const TOut *)g.R, g.ldr);
+                           g.bias, g.act, (const TOut *)g.R, g.ldr, SWAP ? 1 : 0);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
@@ -365,6 +367,59 @@ int run_umma_static_ws(const GemmArgs &g, int splits, float *ws) {
     return launch_typed<1, 128>(g, plan, sm_count(), ws);
 }
 
+// ---- exchanged operands for very skinny problems (M <= 64) -----------------------------------------------
+// C^T = op(B)^T op(A)^T: N takes the role of the MMA's M (128-row tiles over N) and M that of its N (one 64-wide
+// tile), so the small operand costs 8 KiB of shared memory and a few hundred bytes of traffic per k-block
+// instead of a 16 KiB box of which all but M rows are padding.  (The paper's Split-K row of its transformation
+// table covers the k-slices; the exchange is the same product written for the other operand order.)
+template <typename TOut> int run_swapped(const GemmArgs &gs, const Plan &plan, int units) {
+    const size_t need = workspace_bytes(gs, 1, plan);
+    if (need == 0) return launch_kernel<1, 64, TOut, false, false, false, true>(gs, plan, units, nullptr);
+    float *ws = nullptr;
+    cudaMemPool_t pool = workspace_pool();
+    if (!pool) return PEAK_ERR_CUDA;
+    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&ws), need, pool, gs.stream);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_NO_MEMORY; }
+    int rc = launch_kernel<1, 64, TOut, false, false, false, true>(gs, plan, units, ws);
+    e = cudaFreeAsync(ws, gs.stream);
+    if (e != cudaSuccess && rc == PEAK_OK) { set_cuda_error(e); rc = PEAK_ERR_CUDA; }
+    return rc;
+}
+
+bool swap_applies(const GemmArgs &g) {
+    // Opt-in (PEAK_TUNE_SWAP_AB = 2, or a tuning-table entry): measured on B200 it is slower than the plain
+    // single-CTA tiles on every skinny shape tried -- 16x4096x4096 TN 15.3 against 14.1 us, NT 13.7 against 13.4,
+    // 8x8192x8192 33.3 against 29.4, 64x8192x8192 35.6 against 33.0, 32x14336x4096 25.7 against 25.1 -- although
+    // each SM receives little more than half the bytes: these launches are bound by their fixed costs and the
+    // latency of a short pipeline, not by operand traffic.
+    const int mode = tuning(PEAK_TUNE_SWAP_AB);
+    if (mode != 2 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype)) || g.M > 64 || g.N < 128) return false;
+    return true;
+}
+
+int launch_swapped(const GemmArgs &g) {
+    GemmArgs gs = g;
+    gs.A = g.B; gs.lda = g.ldb; gs.B = g.A; gs.ldb = g.lda;
+    gs.M = g.N; gs.N = g.M;
+    gs.transA = g.transB ? 0 : 1;
+    gs.transB = g.transA ? 0 : 1;
+    const int units = sm_count();
+    const int64_t num_kb = (g.K + BK - 1) / BK;
+    const int64_t tiles = (gs.M + BM - 1) / BM;
+    // k-slices: fill the SMs once, at least four k-blocks per slice
+    int64_t s = tuning(PEAK_TUNE_SPLIT_K) > 0 ? tuning(PEAK_TUNE_SPLIT_K) : std::min<int64_t>(units / tiles, num_kb / 4);
+    s = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(s, 16), num_kb));
+    while (s > 1 && ((num_kb + s - 1) / s) * (s - 1) >= num_kb) --s;  // no empty last slice
+    const Plan plan{64, s == 1 ? (int)tiles : 0, (int)s};
+    switch (out_elem(g.dtype)) {
+        case Elem::F32: return run_swapped<float>(gs, plan, units);
+        case Elem::F16: return run_swapped<__half>(gs, plan, units);
+        case Elem::BF16: return run_swapped<__nv_bfloat16>(gs, plan, units);
+        default: break;
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
 }  // namespace
 
 bool umma_supports(const GemmArgs &g, int cta_group) {
@@ -392,6 +447,7 @@ int umma_units(int cta_group) { return sm_count() / (cta_group == 2 ? 2 : 1); }
 
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
+    if (cta_group == 1 && swap_applies(g)) return launch_swapped(g);
     const int units = sm_count() / cta_group;
     Plan plan = choose_plan(g, cta_group, units);
     const bool in8 = is_fp8(in_elem(g.dtype));

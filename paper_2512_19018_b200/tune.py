@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 14
+NUM_KEYS = 15
 
 
 def candidates(space: dict, quick: bool = False):
@@ -78,6 +78,7 @@ AXES_TENSOR = [
     (11, [0, 1]),                   # PEAK_TUNE_BALANCED_GRID
     (3, [0, 1, 2]),                 # PEAK_TUNE_EPILOGUE
     (13, [0, 1, 2]),                # PEAK_TUNE_K_ORDER
+    (14, [0, 1, 2]),                # PEAK_TUNE_SWAP_AB
 ]
 AXES_F32 = [
     ("variant", ["auto"]),

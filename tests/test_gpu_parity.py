@@ -680,3 +680,62 @@ def test_alternating_k_order_is_exact_and_repeatable(variant, reset_tuning):
         dc.reset_c()
         dc.run(variant)
         assert np.array_equal(dc.result(), first)
+
+
+# ------------------------------------------------------------------ exchanged operands (M <= 64)
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_swapped_operands_exact_and_selected(ta, tb, reset_tuning):
+    """With PEAK_TUNE_SWAP_AB = 2, problems with M <= 64 are computed as C^T = op(B)^T op(A)^T on single-CTA tiles
+    with a 64-wide MMA N and written back transposed: exact on integers for ragged M, N, K, every output type,
+    alpha / beta, with and without a k-split; without the knob the plain tiles run."""
+    P.peak_set_tuning(P.PEAK_TUNE_SWAP_AB, 2)
+    shapes = [(16, 4096, 1024), (1, 128, 64), (7, 1000, 200), (33, 520, 1544), (64, 257, 72), (48, 2048, 4100)]
+    for idx, (M, N, K) in enumerate(shapes):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16):
+            pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5 if dtype != W.PEAK_F16_F32 else 2.0,
+                   beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb, pad_c=idx % 2, case=idx)
+            for split in (0, 1, 3):
+                if split > max(1, (K + 63) // 64):
+                    continue
+                P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+                dc = R.DeviceCase(c)
+                dc.run(P.PEAK_VARIANT_AUTO)
+                name = P.peak_last_kernel()
+                assert "umma_gemm_kernel<1, 64," in name and ", 1> " in name, name
+                ref, _ = dc.oracle_full()
+                want = oracle.round_to(R.OT[c.out_type], ref)
+                got = dc.result()
+                got = got.view(np.uint32) if c.out_type == "f32" else got
+                assert np.array_equal(got, want), f"{c} split={split}"
+    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 0)
+    P.peak_set_tuning(P.PEAK_TUNE_SWAP_AB, 0)
+    c = mk(W.PEAK_BF16_BF16, ta, tb, 16, 1024, 512, dist="smallint", pad_a=(-(16 if ta else 512)) % 8)
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert ", 0> " in P.peak_last_kernel()
+
+
+def test_swapped_operands_real_values_and_fused_tail(reset_tuning):
+    """Real-valued inputs through the exchanged-operand kernel, with bias (one value per column of C, i.e. per
+    accumulator row), GELU and a residual; whole tiles and k-slices."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(31)
+    P.peak_set_tuning(P.PEAK_TUNE_SWAP_AB, 2)
+    for idx, (ta, tb, M, N, K, a, b) in enumerate([(1, 0, 16, 4096, 4096, 0.5, 2.0), (0, 1, 40, 1100, 520, 1.0, 0.0),
+                                                   (0, 0, 64, 512, 1000, -1.0, 1.0), (1, 1, 5, 300, 136, 2.0, 0.0)]):
+        pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+        c = W.GemmCase(f"swap{idx}", W.PEAK_BF16_BF16 if idx % 2 == 0 else W.PEAK_F16_F32, bool(ta), bool(tb), M, N, K, a, b,
+                       "uniform", pad_a=pa, pad_b=pb, pad_c=idx, case=idx)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_AUTO)
+        assert ", 1> " in P.peak_last_kernel()
+        R.check_full(dc, what=f"{c}")
+        bias = (rng.standard_normal(N) * 2).astype(np.float32)
+        res = make_residual(c, rng, idx)
+        for split in (0, 2):
+            P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+            dcf = run_fused(c, P.PEAK_VARIANT_AUTO, bias, P.PEAK_ACT_GELU, res)
+            assert ", 1> " in P.peak_last_kernel()
+            check_fused(dcf, bias, P.PEAK_ACT_GELU, f"swapped fused {c} split={split}", res)
+        P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 0)

@@ -178,6 +178,10 @@ def test_bench_traffic_is_read_from_the_profile_of_the_launched_kernel():
     import bench
     t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 512, __nv_bfloat16, 0, 0, 0, 0> grid=148 items=512 splits=1")
     assert t is not None and 0.3e9 < t < 3e9 and "profiles/" in src
+    t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 512, __nv_bfloat16, 0, 0, 0, 0, 0> grid=148")
+    assert t is not None                                   # a trailing flag added later, left at 0: same kernel
+    t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 512, __nv_bfloat16, 0, 0, 0, 0, 1> grid=148")
+    assert t is None
     t, src = bench.profile_traffic("bf16_8192_nn", "umma_gemm_kernel<2, 256, __nv_bfloat16, 0, 0, 0, 0> grid=148")
     assert t is None and "differs" in src
     t, src = bench.profile_traffic("no_such_workload", "x_kernel<1>")
