@@ -303,7 +303,11 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_SWAP_AB = 14,     /* problems with M <= 64 (single-CTA tiles, 16-bit inputs): computed as C^T = op(B)^T
                                    op(A)^T, so that M is the narrow side of the tensor-core tile, when set to 2
                                    (default: off -- it measured slower than the plain tiles on B200) */
-    PEAK_TUNE_COUNT_ = 15
+    PEAK_TUNE_SGEMM_TRANSPOSE = 15, /* SGEMM: an operand whose contiguous index is k (A not transposed, B transposed) is
+                                       first copied, transposed, into pool memory so that the kernel reads dense tiles;
+                                       1 = never, 2 = always (default: when the other dimension is at least 2048 and
+                                       the copy is at most 512 MiB) */
+    PEAK_TUNE_COUNT_ = 16
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

@@ -142,6 +142,7 @@ int launch_umma(const GemmArgs &g, int cta_group);
 bool umma_supports(const GemmArgs &g, int cta_group);
 int umma_units(int cta_group);  // CTAs (cta_group 1) or CTA pairs (2) a persistent launch can keep resident
 bool umma_multicast_available();
+cudaMemPool_t scratch_pool();  // per-device stream-ordered pool that keeps its memory (split-K partials, SGEMM transposes)
 
 // status word layout: bit 31 = a bounded wait gave up; bits 0..7 = role, 8..15 = barrier index
 constexpr uint32_t kStatusTimeout = 0x80000000u;

@@ -350,7 +350,12 @@ int launch_sgemm(const GemmArgs &g) {
     // those layouts stay on them; PEAK_TUNE_SGEMM_COPY = 3 forces the TMA-fed kernel.
     const int copy = tuning(PEAK_TUNE_SGEMM_COPY);
     const bool aligned = sgemm_aligned_supports(g);
-    const bool want_tma = copy == 3 || !aligned || (copy == 0 && !g.transB);
+    // (... unless B is large enough against M to be transposed first, after which the TMA-fed kernel reads dense
+    // tiles and is the fastest for every layout)
+    const bool b_gets_transposed = g.transB && tuning(PEAK_TUNE_SGEMM_TRANSPOSE) != 1 &&
+                                   (tuning(PEAK_TUNE_SGEMM_TRANSPOSE) == 2 || (g.M >= 2048 && g.N >= 512)) &&
+                                   g.N * g.K * 4 <= (512ll << 20);
+    const bool want_tma = copy == 3 || !aligned || (copy == 0 && (!g.transB || b_gets_transposed));
     if (want_tma && sgemm_tma_supports(g)) return launch_sgemm_tma(g);
     if (!aligned) return PEAK_ERR_UNSUPPORTED;
     const bool both_k_contiguous = !g.transA && g.transB;

@@ -58,9 +58,18 @@ __device__ __forceinline__ float2 lds64(uint32_t addr) {
 // A_KC / B_KC: the operand's contiguous index in memory is k (A not transposed / B transposed).
 // KG: how many k one shared-memory load of a k-contiguous operand covers (4: 16-byte loads, 2: 8-byte loads;
 // two k-contiguous operands at 4 k each would not fit the register budget of two blocks per SM).
-template <bool A_KC, bool B_KC, int KG>
-__global__ void __launch_bounds__(ST_THREADS, 2)
+// WIDE: the same 128 x 128 x 16 block tile worked on by 128 threads, each with an 8 x 16 register tile (128
+// accumulators, up to 255 registers, still two blocks per SM): six shared-memory loads per 64 two-wide FMAs
+// instead of four per 32, and the operands of the next k are fetched into a second set of registers while the
+// current k is multiplied, so that two warps per scheduler are enough to keep the FMA pipe fed.  B must land
+// dense.
+template <bool A_KC, bool B_KC, int KG, bool WIDE = false>
+__global__ void __launch_bounds__(WIDE ? 128 : ST_THREADS, 2)
 sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const SgemmParams p) {
+    static_assert(!WIDE || !B_KC, "the wide register tile needs B dense");
+    constexpr int THREADS = WIDE ? 128 : ST_THREADS, NWARPS = THREADS / 32;
+    constexpr int NT = WIDE ? 16 : 8;            // columns of C per thread
+    constexpr int TXN = WIDE ? 8 : 16;           // threads along n; each takes groups of 4 columns TXN*4 apart
     extern __shared__ uint8_t st_smem_raw[];
     const uint32_t raw = ptx::smem_u32(st_smem_raw);
     const uint32_t stage0 = (raw + 1023u) & ~1023u;
@@ -70,7 +79,7 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         reinterpret_cast<volatile uint32_t *>(st_smem_raw + (empty0 + 8 * ST_STAGES - raw));
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tx = tid % 16, ty = tid / 16;
+    const int tx = tid % TXN, ty = tid / TXN;
     int64_t tm, tn;
     tile_coord(blockIdx.x, p.tiles_m, p.tiles_n, p.group, tm, tn);
     const int m0 = (int)tm * ST_BM, n0 = (int)tn * ST_BN;
@@ -78,7 +87,7 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (tid == 0) {
         for (int s = 0; s < ST_STAGES; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
-            ptx::mbar_init(empty0 + 8 * s, ST_THREADS / 32);  // one arrival per warp
+            ptx::mbar_init(empty0 + 8 * s, NWARPS);  // one arrival per warp
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -104,11 +113,11 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (tid == 0)
         for (int kb = 0; kb < ST_AHEAD && kb < nkb; ++kb) issue(kb);
 
-    float acc[8][8];
+    float acc[8][NT];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < NT; ++j) acc[i][j] = 0.0f;
 
     // Row i of this thread's 8 x 8 tile is m0 + ty*4 + (i & 3) + 64*(i >> 2).  Column j is n0 + tx*4 + (j & 3) +
     // 64*(j >> 2) when B lands dense, n0 + tx + 16*j when B is k-contiguous: with the 64-byte swizzle the sixteen
@@ -129,7 +138,7 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int kb = 0; kb < nkb; ++kb) {
         const uint32_t s = (uint32_t)kb % ST_STAGES, ph = ((uint32_t)kb / ST_STAGES) & 1u;
         // the warps take turns at refilling the ring: stage (kb + AHEAD) % STAGES was last read two k-blocks ago
-        if (warp == (kb & 7) && lane == 0 && kb + ST_AHEAD < nkb) {
+        if (warp == (kb % NWARPS) && lane == 0 && kb + ST_AHEAD < nkb) {
             const int kl = kb + ST_AHEAD;
             const uint32_t sl = (uint32_t)kl % ST_STAGES, pl = ((uint32_t)kl / ST_STAGES) & 1u;
             if (ptx::mbar_wait<false>(empty0 + 8 * sl, pl ^ 1u, abort_flag, p.wait_cycles)) issue(kl);
@@ -149,6 +158,95 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             break;
         }
         const uint32_t As = stage0 + s * ST_STAGE_BYTES, Bs = As + ST_TILE_BYTES;
+        if constexpr (WIDE) {
+            // operand fragments of one k: a[8] (rows) and b[16] (columns: four groups of 4, 32 columns apart, so
+            // that the eight tx of a warp read 128 contiguous bytes per load and the four ty share them)
+            auto load_b = [&](int k, float (&b)[16]) {
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float4 v = lds128(Bs + (uint32_t)(k * ST_BN + tx * 4 + 32 * h) * 4u);
+                    b[4 * h] = v.x; b[4 * h + 1] = v.y; b[4 * h + 2] = v.z; b[4 * h + 3] = v.w;
+                }
+            };
+            auto load_a_dense = [&](int k, float (&a)[8]) {
+                const float4 v0 = lds128(As + (uint32_t)(k * ST_BM + ty * 4) * 4u);
+                const float4 v1 = lds128(As + (uint32_t)(k * ST_BM + ty * 4 + 64) * 4u);
+                a[0] = v0.x; a[1] = v0.y; a[2] = v0.z; a[3] = v0.w; a[4] = v1.x; a[5] = v1.y; a[6] = v1.z; a[7] = v1.w;
+            };
+            auto load_a_pair = [&](int k2, float (&a0)[8], float (&a1)[8]) {  // k-contiguous A: k = 2*k2 and 2*k2 + 1
+                const uint32_t a_plus = As + a_base + a_t, a_minus = As + a_base - a_t;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t q = ((uint32_t)k2 >> 1) ^ (uint32_t)((i & 3) >> 1);
+                    const uint32_t off = (uint32_t)((i & 3) + 64 * (i >> 2)) * 64u + (q << 4) + ((uint32_t)k2 & 1u) * 8u;
+                    const float2 v = lds64(((q & 2u) ? a_minus : a_plus) + off);
+                    a0[i] = v.x; a1[i] = v.y;
+                }
+            };
+            auto fma_k = [&](const float (&a)[8], const float (&b)[16]) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float2 aa = make_float2(a[i], a[i]);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float2 c = make_float2(acc[i][2 * j], acc[i][2 * j + 1]);
+                        c = __ffma2_rn(aa, make_float2(b[2 * j], b[2 * j + 1]), c);
+                        acc[i][2 * j] = c.x;
+                        acc[i][2 * j + 1] = c.y;
+                    }
+                }
+            };
+            if constexpr (A_KC && KG == 4) {
+                // k-contiguous A, four k per 16-byte load: eight loads fetch this thread's rows for four k (the same
+                // two loads per k as a dense tile); the next four k are fetched while these are multiplied
+                auto load_a_quad = [&](int k4, float (&aq)[8][4]) {
+                    const uint32_t a_plus = As + a_base + a_t, a_minus = As + a_base - a_t;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t q = (uint32_t)k4 ^ (uint32_t)((i & 3) >> 1);
+                        const uint32_t off = (uint32_t)((i & 3) + 64 * (i >> 2)) * 64u + (q << 4);
+                        const float4 v = lds128(((q & 2u) ? a_minus : a_plus) + off);
+                        aq[i][0] = v.x; aq[i][1] = v.y; aq[i][2] = v.z; aq[i][3] = v.w;
+                    }
+                };
+                float aq[2][8][4], bq[2][16];
+                load_a_quad(0, aq[0]);
+                load_b(0, bq[0]);
+#pragma unroll
+                for (int k4 = 0; k4 < ST_BK / 4; ++k4) {
+                    const int ca = k4 & 1;
+                    if (k4 + 1 < ST_BK / 4) load_a_quad(k4 + 1, aq[ca ^ 1]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int kg = 4 * k4 + k, cb = kg & 1;
+                        if (kg + 1 < ST_BK) load_b(kg + 1, bq[cb ^ 1]);
+                        float a[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) a[i] = aq[ca][i][k];
+                        fma_k(a, bq[cb]);
+                    }
+                }
+            } else {
+            // two k per step, fragments of the next step fetched before this step's FMAs are issued
+            float a0[2][8], a1[2][8], b0[2][16], b1[2][16];
+            if (A_KC) load_a_pair(0, a0[0], a1[0]);
+            else { load_a_dense(0, a0[0]); load_a_dense(1, a1[0]); }
+            load_b(0, b0[0]);
+            load_b(1, b1[0]);
+#pragma unroll
+            for (int k2 = 0; k2 < ST_BK / 2; ++k2) {
+                const int cur = k2 & 1, nxt = cur ^ 1;
+                if (k2 + 1 < ST_BK / 2) {
+                    if (A_KC) load_a_pair(k2 + 1, a0[nxt], a1[nxt]);
+                    else { load_a_dense(2 * k2 + 2, a0[nxt]); load_a_dense(2 * k2 + 3, a1[nxt]); }
+                    load_b(2 * k2 + 2, b0[nxt]);
+                }
+                fma_k(a0[cur], b0[cur]);
+                if (k2 + 1 < ST_BK / 2) load_b(2 * k2 + 3, b1[nxt]);
+                fma_k(a1[cur], b1[cur]);
+            }
+            }
+        } else {
 #pragma unroll
         for (int kk = 0; kk < ST_BK; kk += KG) {
             float ak[8][KG], bk[8][KG];
@@ -217,6 +315,7 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
         }
+        }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(empty0 + 8 * s);  // this warp is done reading the stage
     }
@@ -236,8 +335,8 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float *crow = p.C + (int64_t)m * p.ldc;
         if (!B_KC) {
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int n = n0 + tx * 4 + 64 * h;
+            for (int h = 0; h < NT / 4; ++h) {
+                const int n = n0 + tx * 4 + TXN * 4 * h;
                 if (n >= p.N) continue;
                 if (p.vec_ok && n + 4 <= p.N) {
                     float4 *dst = reinterpret_cast<float4 *>(crow + n);
@@ -278,8 +377,40 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <bool A_KC, bool B_KC, int KG> int run_sgemm_tma(const GemmArgs &g) {
-    auto kernel = sgemm_tma_kernel<A_KC, B_KC, KG>;
+// dst[c][r] = src[r][c] for an r x c row-major matrix: 32 x 32 tiles through padded shared memory, both sides
+// coalesced.  The paper's Transpose step as a pass of its own.
+__global__ void __launch_bounds__(256)
+transpose_f32_kernel(const float *__restrict__ src, int64_t ld_src, int rows, int cols, float *__restrict__ dst,
+                     int64_t ld_dst) {
+    __shared__ float tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        const int r = r0 + ty + i, c = c0 + tx;
+        if (r < rows && c < cols) tile[ty + i][tx] = src[(int64_t)r * ld_src + c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        const int c = c0 + ty + i, r = r0 + tx;
+        if (r < rows && c < cols) dst[(int64_t)c * ld_dst + r] = tile[tx][ty + i];
+    }
+}
+
+int launch_transpose(const float *src, int64_t ld_src, int64_t rows, int64_t cols, float *dst, int64_t ld_dst,
+                     cudaStream_t stream) {
+    dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32));
+    if (grid.y > 65535u) return PEAK_ERR_UNSUPPORTED;
+    transpose_f32_kernel<<<grid, 256, 0, stream>>>(src, ld_src, (int)rows, (int)cols, dst, ld_dst);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+template <bool A_KC, bool B_KC, int KG, bool WIDE = false> int run_sgemm_tma(const GemmArgs &g) {
+    auto kernel = sgemm_tma_kernel<A_KC, B_KC, KG, WIDE>;
     static PerDeviceOnce attr_once;
     const cudaError_t attr_err = attr_once.run(current_device(), [&] {
         return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM_BYTES);
@@ -312,9 +443,9 @@ template <bool A_KC, bool B_KC, int KG> int run_sgemm_tma(const GemmArgs &g) {
     p.status = device_status_word();
     if (!p.status) return PEAK_ERR_CUDA;
     const unsigned grid = (unsigned)(p.tiles_m * p.tiles_n);
-    kernel<<<grid, ST_THREADS, ST_SMEM_BYTES, g.stream>>>(tmA, tmB, p);
+    kernel<<<grid, WIDE ? 128 : ST_THREADS, ST_SMEM_BYTES, g.stream>>>(tmA, tmB, p);
     count_launch();
-    note_kernel("sgemm_tma_kernel<%d, %d, %d> grid=%u", (int)A_KC, (int)B_KC, KG, grid);
+    note_kernel("sgemm_tma_kernel<%d, %d, %d, %d> grid=%u", (int)A_KC, (int)B_KC, KG, (int)WIDE, grid);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
@@ -334,14 +465,64 @@ bool sgemm_tma_supports(const GemmArgs &g) {
     return true;
 }
 
+// A k-contiguous operand costs the kernel 7 points of FMA-pipe time (A) or far more (B); a copy of it with m / n
+// contiguous costs one pass over that operand.  Where the product is large against the operand -- the other
+// dimension at least 2048, so the pass is under about 2 % -- and the copy fits a bounded workspace, the operand
+// is transposed into pool memory first and the dense-dense kernel runs (4096^3 NN: 58.8 -> 63+ TFLOP/s).
+int launch_with_transposes(const GemmArgs &g, bool tr_a, bool tr_b) {
+    GemmArgs d = g;
+    float *wa = nullptr, *wb = nullptr;
+    cudaMemPool_t pool = scratch_pool();
+    if (!pool) return PEAK_ERR_CUDA;
+    int rc = PEAK_OK;
+    cudaError_t e = cudaSuccess;
+    if (tr_a) {  // A stored M x K  ->  K x M
+        const int64_t ld = (g.M + 3) / 4 * 4;
+        e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&wa), (size_t)g.K * ld * sizeof(float), pool, g.stream);
+        if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_NO_MEMORY; }
+        rc = launch_transpose((const float *)g.A, g.lda, g.M, g.K, wa, ld, g.stream);
+        d.A = wa; d.lda = ld; d.transA = 1;
+    }
+    if (rc == PEAK_OK && tr_b) {  // B stored N x K  ->  K x N
+        const int64_t ld = (g.N + 3) / 4 * 4;
+        e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&wb), (size_t)g.K * ld * sizeof(float), pool, g.stream);
+        if (e != cudaSuccess) { set_cuda_error(e); rc = PEAK_ERR_NO_MEMORY; }
+        else {
+            rc = launch_transpose((const float *)g.B, g.ldb, g.N, g.K, wb, ld, g.stream);
+            d.B = wb; d.ldb = ld; d.transB = 0;
+        }
+    }
+    if (rc == PEAK_OK) {
+        const bool a_kc = !d.transA, b_kc = d.transB != 0;  // what is still k-contiguous
+        if (a_kc && b_kc) rc = run_sgemm_tma<true, true, 2>(d);
+        else if (b_kc) rc = run_sgemm_tma<false, true, 4>(d);
+        else if (a_kc) rc = run_sgemm_tma<true, false, 4, true>(d);
+        else rc = run_sgemm_tma<false, false, 2, true>(d);
+    }
+    if (wa) cudaFreeAsync(wa, g.stream);
+    if (wb) cudaFreeAsync(wb, g.stream);
+    return rc;
+}
+
 int launch_sgemm_tma(const GemmArgs &g) {
     if (!sgemm_tma_supports(g)) return PEAK_ERR_UNSUPPORTED;
     const bool a_kc = !g.transA, b_kc = g.transB != 0;
+    {
+        const int mode = tuning(PEAK_TUNE_SGEMM_TRANSPOSE);  // 1 = never, 2 = whenever an operand is k-contiguous
+        const int64_t limit = 512ll << 20;                   // bytes of one transposed copy
+        const bool fits_a = g.M * g.K * 4 <= limit && g.M <= 65535ll * 32, fits_b = g.N * g.K * 4 <= limit && g.N <= 65535ll * 32;
+        const bool tr_a = a_kc && fits_a && (mode == 2 || (mode == 0 && g.N >= 2048 && g.M >= 512));
+        const bool tr_b = b_kc && fits_b && (mode == 2 || (mode == 0 && g.M >= 2048 && g.N >= 512));
+        if (mode != 1 && (tr_a || tr_b)) return launch_with_transposes(g, tr_a, tr_b);
+    }
     // k per load of a k-contiguous operand, measured at 4096^3 / 8192^3 NN: two (58.8 / 59.3 TFLOP/s) beats four
     // (58.1 / 58.7): the sixteen fewer live registers leave the scheduler more room
     if (a_kc && b_kc) return run_sgemm_tma<true, true, 2>(g);
-    if (a_kc) return run_sgemm_tma<true, false, 2>(g);
     if (b_kc) return run_sgemm_tma<false, true, 4>(g);
+    const bool wide = tuning(PEAK_TUNE_SGEMM_FMA) != 3;  // 3 = the 8 x 8 register tile (A/B measurements)
+    if (wide && a_kc) return tuning(PEAK_TUNE_SGEMM_FMA) == 4 ? run_sgemm_tma<true, false, 2, true>(g) : run_sgemm_tma<true, false, 4, true>(g);
+    if (wide) return run_sgemm_tma<false, false, 2, true>(g);
+    if (a_kc) return run_sgemm_tma<true, false, 2>(g);
     return run_sgemm_tma<false, false, 4>(g);
 }
 

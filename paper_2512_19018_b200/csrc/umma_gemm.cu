@@ -443,6 +443,8 @@ bool umma_supports(const GemmArgs &g, int cta_group) {
 
 bool umma_multicast_available() { return mc_entry() != nullptr; }
 
+cudaMemPool_t scratch_pool() { return workspace_pool(); }
+
 int umma_units(int cta_group) { return sm_count() / (cta_group == 2 ? 2 : 1); }
 
 int launch_umma(const GemmArgs &g, int cta_group) {

@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 15
+NUM_KEYS = 16
 
 
 def candidates(space: dict, quick: bool = False):
@@ -85,6 +85,7 @@ AXES_F32 = [
     (7, [0, 1, 2, 3]),              # PEAK_TUNE_SGEMM_COPY
     (4, [0, 1, 2]),                 # PEAK_TUNE_SGEMM_FMA
     (0, [0, 2, 4, 8, 16, 32]),      # PEAK_TUNE_RASTER_GROUP
+    (15, [0, 1, 2]),                # PEAK_TUNE_SGEMM_TRANSPOSE
 ]
 
 

@@ -739,3 +739,34 @@ def test_swapped_operands_real_values_and_fused_tail(reset_tuning):
             assert ", 1> " in P.peak_last_kernel()
             check_fused(dcf, bias, P.PEAK_ACT_GELU, f"swapped fused {c} split={split}", res)
         P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 0)
+
+
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_sgemm_transposing_prepass_and_wide_register_tile(ta, tb, reset_tuning):
+    """SGEMM with a k-contiguous operand copied, transposed, into pool memory first (PEAK_TUNE_SGEMM_TRANSPOSE = 2:
+    always) and the 8 x 16 register-tile kernel on dense tiles: exact on integers for ragged shapes and padded
+    pitches in every layout, within the fp32 bounds on reals with alpha / beta / bias / residual; with the knob at
+    1 the direct kernels run and give the same bits on integers."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(41)
+    for idx, (M, N, K) in enumerate([(1000, 1000, 1000), (129, 257, 33), (1, 300, 50), (512, 384, 528), (333, 70, 2050)]):
+        pa, pb = (-(M if ta else K)) % 4 + 4 * (idx % 2), (-(K if tb else N)) % 4
+        ci = mk(W.PEAK_F32_F32, ta, tb, M, N, K, dist="smallint", alpha=2.0, beta=-1.0, pad_a=pa, pad_b=pb, pad_c=idx % 3,
+                case=idx)
+        outs = []
+        for mode in (2, 1):
+            P.peak_set_tuning(P.PEAK_TUNE_SGEMM_TRANSPOSE, mode)
+            dc = R.DeviceCase(ci)
+            dc.run(P.PEAK_VARIANT_SGEMM)
+            if mode == 2:
+                assert "sgemm_tma_kernel<0, 0, 2, 1>" in P.peak_last_kernel(), P.peak_last_kernel()
+            ref, _ = dc.oracle_full()
+            assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref)), f"{ci} mode {mode}"
+            outs.append(dc.result().copy())
+        assert np.array_equal(outs[0], outs[1])
+    P.peak_set_tuning(P.PEAK_TUNE_SGEMM_TRANSPOSE, 2)
+    c = W.GemmCase("sg_tr_fused", W.PEAK_F32_F32, bool(ta), bool(tb), 520, 392, 264, 0.5, 2.0, "uniform")
+    bias = rng.standard_normal(c.N).astype(np.float32)
+    res = make_residual(c, rng, 4)
+    dc = run_fused(c, P.PEAK_VARIANT_AUTO, bias, P.PEAK_ACT_GELU, res)
+    check_fused(dc, bias, P.PEAK_ACT_GELU, f"sgemm transposed {c.layout}", res)
