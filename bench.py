@@ -55,7 +55,7 @@ OTHER_WORKLOADS = [
     "bf16_tfm_16384x4096x4096_nt", "bf16_tfm_16384x14336x4096_nt", "bf16_tfm_16384x4096x14336_nt",
     "bf16_5000x3000x2500_tn", "bf16_16x4096x4096_tn", "bf16_128x14336x4096_tn",
     "fp32_4096_nn", "fp32_8192_nn",
-    "e4m3_8192_nt",
+    "e4m3_8192_nt", "e4m3_8192_nn",
 ]
 
 
