@@ -770,3 +770,57 @@ def test_sgemm_transposing_prepass_and_wide_register_tile(ta, tb, reset_tuning):
     res = make_residual(c, rng, 4)
     dc = run_fused(c, P.PEAK_VARIANT_AUTO, bias, P.PEAK_ACT_GELU, res)
     check_fused(dc, bias, P.PEAK_ACT_GELU, f"sgemm transposed {c.layout}", res)
+
+
+def test_sgemm_tma_paths_in_a_cuda_graph_and_on_two_streams(reset_tuning):
+    """The TMA-fed SGEMM inside a captured graph -- a ragged problem, and one whose k-contiguous operands are first
+    transposed into pool memory (allocated and freed inside the capture) -- replayed twice; then the same two
+    problems from two host threads on two streams at once."""
+    import threading
+    P.peak_set_tuning(P.PEAK_TUNE_SGEMM_TRANSPOSE, 2)
+    cases = [mk(W.PEAK_F32_F32, 0, 1, 520, 392, 264, alpha=0.5, beta=2.0, case=1),      # both operands transposed first
+             mk(W.PEAK_F32_F32, 1, 0, 333, 260, 100, alpha=1.0, beta=0.0, pad_a=3, case=2)]
+    dcs = [R.DeviceCase(c) for c in cases]
+    for dc in dcs:
+        dc.run(stream=None)                                    # first-use set-up outside the capture
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for dc in dcs:
+                c = dc.case
+                P.peak_gemm(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta,
+                            dc.C, c.ldc, stream)
+    for rep in range(2):
+        for dc in dcs:
+            dc.Cfull.copy_(R.to_device(dc.Cfull_h, dc.case.out_type))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert P.peak_check()[0] == P.PEAK_OK
+        for dc in dcs:
+            R.check_full(dc, what=f"sgemm graph replay {rep} {dc.case.name}")
+    errors = []
+
+    def worker(idx):
+        try:
+            st = torch.cuda.Stream()
+            dc = dcs[idx]
+            c = dc.case
+            for rep in range(10):
+                dc.reset_c()
+                st.wait_stream(torch.cuda.current_stream())
+                P.peak_gemm(c.dtype, c.transA, c.transB, c.M, c.N, c.K, c.alpha, dc.A, c.lda, dc.B, c.ldb, c.beta, dc.C,
+                            c.ldc, st)
+                rc, detail = P.peak_check(st)
+                assert rc == P.PEAK_OK, hex(detail)
+            R.check_full(dc, what=f"sgemm thread {idx}")
+        except Exception as exc:
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[0]
