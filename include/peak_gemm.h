@@ -307,7 +307,9 @@ typedef enum peak_tuning_key {
                                        first copied, transposed, into pool memory so that the kernel reads dense tiles;
                                        1 = never, 2 = always (default: when the other dimension is at least 2048 and
                                        the copy is at most 512 MiB) */
-    PEAK_TUNE_COUNT_ = 16
+    PEAK_TUNE_SHORT_A = 16,     /* single-CTA tiles of problems with M < 128: 1 = always fetch all 128 rows of the A tile
+                                   (default: only the rows that exist, which saves copy-engine requests) */
+    PEAK_TUNE_COUNT_ = 17
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

@@ -104,6 +104,12 @@ struct UmmaParams {
     int64_t ldr;
     int r_vec;             // R base and pitch allow 16-byte vector loads
     int k_alternate;       // 1: every other item of a CTA walks its k-blocks downwards (L2 reuse across waves)
+    // Single-CTA tiles of a problem with fewer than 128 rows load only the rows of A that exist (rounded up to
+    // the copy's granularity): every box row is one request to the copy engine, whose request rate -- not bytes --
+    // bounds these kernels.  What the unloaded rows of the stage hold only reaches accumulator rows that are never
+    // stored.  a_boxes: MN-major A, how many 64-row (8-bit: 128-row) boxes are fetched; stage_tx: bytes per stage.
+    int a_boxes;
+    uint32_t stage_tx;
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;
@@ -567,7 +573,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && j == nk - 1)
                         continue;  // test hook: leave this stage empty so that the waits downstream run out
                     uint32_t bar = full0 + 8 * s;
-                    if (leader) ptx::mbar_arrive_expect_tx(bar, (uint32_t)(C_::STAGE_BYTES * CG));
+                    if (leader) ptx::mbar_arrive_expect_tx(bar, CG == 1 ? p.stage_tx : (uint32_t)(C_::STAGE_BYTES * CG));
                     if (CG == 2) bar = ptx::map_to_cta(bar, leader_crank);
                     const uint32_t a_dst = stage_base + s * C_::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
@@ -577,6 +583,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     } else {
 #pragma unroll
                         for (int h = 0; h < BM / MN_ELEMS; ++h) {
+                            if (CG == 1 && h >= p.a_boxes) break;
                             load_tile<CG, BATCHED>(a_dst + h * MN_ATOM, &tmA, m_cta + MN_ELEMS * h, k0, bz, bar);
                         }
                     }

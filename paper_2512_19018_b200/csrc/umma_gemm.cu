@@ -130,8 +130,13 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     // elements) by all k-rows of a k-block; an 8-bit B of that kind needs at least 128 columns per CTA.
     constexpr int MNE = IN8 ? 128 : 64;
     if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
+    // rows of A a single-CTA tile fetches: all 128, or, when the whole problem has fewer, only those that exist
+    // (K-major: rounded up to 8; MN-major: whole boxes of MNE rows)
+    const bool short_a = CG == 1 && g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
+    const int a_rows = short_a ? (int)((g.M + 7) / 8 * 8) : 128;
+    const int a_boxes = short_a ? (int)((g.M + MNE - 1) / MNE) : 128 / MNE;
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, MNE, BKE, nb, g.strideA)
-                   : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, 128, nb, g.strideA);
+                   : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, a_rows, nb, g.strideA);
     ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, MNE, BKE, nb, g.strideB)
                      : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS, nb, g.strideB));
     if (!ok) return nb > 1 ? PEAK_ERR_UNSUPPORTED : PEAK_ERR_CUDA;  // e.g. a batch stride TMA cannot express
@@ -160,6 +165,8 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.kb_per_split = (p.num_kb + plan.tail_splits - 1) / plan.tail_splits;
     p.total_items = plan.full_tiles + (tiles - plan.full_tiles) * plan.tail_splits;
     p.a_mn = a_mn; p.b_mn = b_mn;
+    p.a_boxes = a_boxes;
+    p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
     // operand format field: f16 kind: 0 = fp16, 1 = bf16; f8f6f4 kind: 0 = E4M3, 1 = E5M2
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |

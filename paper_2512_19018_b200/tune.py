@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 16
+NUM_KEYS = 17
 
 
 def candidates(space: dict, quick: bool = False):

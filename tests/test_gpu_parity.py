@@ -742,6 +742,45 @@ def test_swapped_operands_real_values_and_fused_tail(reset_tuning):
 
 
 @pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_short_a_loads_exact(ta, tb, reset_tuning):
+    """Problems with M < 128 on single-CTA tiles fetch only the rows of A that exist (rounded up to 8; whole
+    64-row boxes when A is stored m-contiguous), so the rest of the A stage keeps whatever an earlier tile left
+    there -- NaN patterns included -- and only accumulator rows that are never stored see it.  Exact on integers
+    for M from 1 to 127 after a problem that filled every stage with NaNs, with and without a k-split and for
+    8-bit inputs; PEAK_TUNE_SHORT_A = 1 (whole boxes) gives the same bits."""
+    nan_case = mk(W.PEAK_BF16_BF16, ta, tb, 128, 148 * 256, 512, dist="smallint", case=77)
+    dn = R.DeviceCase(nan_case)                  # one tile on every SM, shared memory left full of NaN patterns
+    dn.A.view(torch.int16).fill_(0x7FC0)
+    dn.B.view(torch.int16).fill_(0x7FC0)
+    for idx, (M, N, K) in enumerate([(1, 4096, 1024), (8, 136, 72), (9, 1000, 520), (16, 4096, 4096), (63, 264, 200),
+                                     (65, 520, 136), (100, 2048, 1032), (127, 384, 4100)]):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_E4M3_BF16):
+            unit = 16 if dtype == W.PEAK_E4M3_BF16 else 8
+            pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0][idx % 2], pad_a=pa, pad_b=pb,
+                   case=idx)
+            results = []
+            for mode in (0, 1):
+                for split in (0, 1, 4):
+                    if split > max(1, (K + 63) // 64):
+                        continue
+                    P.peak_set_tuning(P.PEAK_TUNE_SHORT_A, 1)
+                    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 1)
+                    dn.run(P.PEAK_VARIANT_UMMA_1CTA)
+                    P.peak_set_tuning(P.PEAK_TUNE_SHORT_A, mode)
+                    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+                    dc = R.DeviceCase(c)
+                    dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+                    ref, _ = dc.oracle_full()
+                    want = oracle.round_to(R.OT[c.out_type], ref)
+                    got = dc.result()
+                    got = got.view(np.uint32) if c.out_type == "f32" else got
+                    assert np.array_equal(got, want), f"{c} short_a={mode} split={split}"
+                    results.append(got.copy())
+            assert all(np.array_equal(results[0], r) for r in results[1:])
+
+
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
 def test_sgemm_transposing_prepass_and_wide_register_tile(ta, tb, reset_tuning):
     """SGEMM with a k-contiguous operand copied, transposed, into pool memory first (PEAK_TUNE_SGEMM_TRANSPOSE = 2:
     always) and the 8 x 16 register-tile kernel on dense tiles: exact on integers for ragged shapes and padded
