@@ -309,7 +309,10 @@ typedef enum peak_tuning_key {
                                        the copy is at most 512 MiB) */
     PEAK_TUNE_SHORT_A = 16,     /* single-CTA tiles of problems with M < 128: 1 = always fetch all 128 rows of the A tile
                                    (default: only the rows that exist, which saves copy-engine requests) */
-    PEAK_TUNE_COUNT_ = 17
+    PEAK_TUNE_CLUSTER_K = 17,   /* a single matrix on single-CTA tiles whose every tile is split 2 or 4 ways: 1 = partial tiles
+                                   through the workspace and a reduction kernel (default: the slices run on the CTAs of
+                                   a cluster and are added through distributed shared memory, one launch) */
+    PEAK_TUNE_COUNT_ = 18
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

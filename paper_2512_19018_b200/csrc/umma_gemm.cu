@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "umma_device.cuh"
+#include "umma_clusterk.cuh"
 #include "umma_host.cuh"
 #include "mc_plugin.h"
 
@@ -52,6 +53,9 @@ int64_t tiles_of(const GemmArgs &g, int cg, int bn) {
     return ((g.M + BM * cg - 1) / (BM * cg)) * ((g.N + bn - 1) / bn) * g.nbatch();
 }
 
+// Clusters of KC single-CTA tiles of width bn that can be resident at once on the current device (umma_clusterk.cuh).
+int clusterk_max_clusters(int bn, int kc);
+
 // Tile width and k-splitting from a small cost model (cycles): an item costs its k-blocks times the slower
 // of the tensor pipe (2*BN cycles per k-block per SM) and the operand stream (bytes per k-block over an
 // about 40 bytes/cycle/SM of L2->shared bandwidth), plus a fixed per-item overhead; items are spread over
@@ -64,6 +68,23 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     double best_cost = 1e300;
     const int force_bn = tuning(PEAK_TUNE_TILE_N), force_split = tuning(PEAK_TUNE_SPLIT_K);
     const int tail_mode = tuning(PEAK_TUNE_TAIL_SPLIT);  // 2 = split the last wave whenever possible
+    // Single matrices whose 128 x 128 tiles fill between an eighth and all of the SMs: k-slices on the CTAs of a
+    // cluster cost one launch and no workspace, so the rule is simply the most CTAs that still run at once --
+    // measured (NT, us; best other plan in brackets): 128x7168x4096 two slices 18.6 (20.4), 256x4096x4096 two slices
+    // 17.8 (20.2), 128x4096x8192 four slices 20.0 (21.8), 64x4096x4096 four slices 12.6 (14.8), 128x14336x4096
+    // whole tiles 29.3 (30.9).  Each slice keeps at least eight k-blocks.
+    if (cg == 1 && g.nbatch() == 1 && !force_bn && !force_split && tail_mode != 2 && tuning(PEAK_TUNE_CLUSTER_K) != 1) {
+        const int64_t t128 = tiles_of(g, 1, 128);
+        if (t128 <= units && t128 * 8 > units) {
+            for (int s : {4, 2}) {
+                const int64_t kbps = (num_kb + s - 1) / s;
+                if (t128 * s > units || kbps < 8 || kbps * (s - 1) >= num_kb) continue;
+                if (t128 > clusterk_max_clusters(128, s)) continue;
+                return Plan{128, 0, s};
+            }
+            return Plan{128, (int)t128, 1};
+        }
+    }
     for (int bn : {512, 256, 128}) {
         if (force_bn ? bn != force_bn : bn == 512) continue;  // 512-wide tiles only on request (see launch_umma)
         if (bn == 512 && cg != 2) continue;
@@ -374,6 +395,148 @@ int run_umma_static_ws(const GemmArgs &g, int splits, float *ws) {
     return launch_typed<1, 128>(g, plan, sm_count(), ws);
 }
 
+// ---- k-slices on the CTAs of a cluster, added through distributed shared memory (umma_clusterk.cuh) -------
+// One launch instead of tile kernel + reduction kernel, no workspace.  Single matrices, single-CTA tiles,
+// every tile split KC = 2 or 4 ways.
+template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const GemmArgs &g, const Plan &plan) {
+    using C_ = Cfg<1, BN>;
+    constexpr int BKE = IN8 ? 2 * BK : BK;
+    constexpr int MNE = IN8 ? 128 : 64;
+    auto kernel = umma_clusterk_kernel<BN, TOut, KC, IN8>;
+    static PerDeviceOnce attr_once;
+    const cudaError_t attr_err = attr_once.run(current_device(), [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) { set_cuda_error(attr_err); return PEAK_ERR_CUDA; }
+    const Elem ein = in_elem(g.dtype), eout = out_elem(g.dtype);
+    const int a_mn = g.transA ? 1 : 0, b_mn = g.transB ? 0 : 1;
+    if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
+    const bool short_a = g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
+    const int a_rows = short_a ? (int)((g.M + 7) / 8 * 8) : 128;
+    const int a_boxes = short_a ? (int)((g.M + MNE - 1) / MNE) : 128 / MNE;
+    CUtensorMap tmA, tmB, tmC;
+    bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, MNE, BKE) : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, a_rows);
+    ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, MNE, BKE)
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS));
+    if (!ok) return PEAK_ERR_CUDA;
+    UmmaParams p = {};
+    p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
+    p.num_kb = (int)((g.K + BKE - 1) / BKE);
+    p.tiles_m = (int)((g.M + BM - 1) / BM);
+    p.tiles_n = (int)((g.N + BN - 1) / BN);
+    p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 16;
+    p.tiles_per_batch = p.tiles_m * p.tiles_n;
+    p.full_tiles = 0;
+    p.tail_splits = KC;
+    p.kb_per_split = (p.num_kb + KC - 1) / KC;
+    p.total_items = p.tiles_per_batch * KC;
+    p.a_mn = a_mn; p.b_mn = b_mn;
+    p.a_boxes = a_boxes;
+    p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
+    const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    p.alpha = g.alpha; p.beta = g.beta;
+    p.C = g.C; p.ldc = g.ldc;
+    p.bias = g.bias; p.act = g.act;
+    const int ob = elem_bytes(eout);
+    p.R = g.R; p.ldr = g.ldr;
+    p.r_vec = (g.R && reinterpret_cast<uintptr_t>(g.R) % 16 == 0 && (g.ldr * ob) % 16 == 0) ? 1 : 0;
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(g.C) % 16) == 0 && (g.ldc * ob) % 16 == 0) ? 1 : 0;
+    const int epi = tuning(PEAK_TUNE_EPILOGUE);
+    p.tma_store = (p.vec_ok && (g.N * ob) % 16 == 0 && epi != 1) ? 1 : 0;
+    p.c_prefetch = (p.tma_store && g.beta != 0.0f && epi != 3) ? 1 : 0;
+    tmC = tmA;
+    if (p.tma_store && !make_map(&tmC, eout, g.C, g.N, g.M, g.ldc, 128 / ob, 32)) return PEAK_ERR_CUDA;
+    p.status = device_status_word();
+    if (!p.status) return PEAK_ERR_CUDA;
+    const int wait_ms = tuning(PEAK_TUNE_WAIT_MS);
+    p.wait_cycles = wait_ms > 0 ? (long long)wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
+    p.inject_stall = tuning(PEAK_TUNE_INJECT_STALL) == 1 ? 1 : 0;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.total_items);
+    cfg.blockDim = dim3(ClusterKCfg<BN, KC>::THREADS);
+    cfg.dynamicSmemBytes = C_::SMEM_BYTES;
+    cfg.stream = g.stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = KC; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+    count_launch();
+    note_kernel("umma_clusterk_kernel<%d, %s, %d, %d> grid=%d clusters=%d", BN,
+                sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"), KC, (int)IN8,
+                p.total_items, p.tiles_per_batch);
+    if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+// PEAK_TUNE_CLUSTER_K: 1 = never (workspace + reduction kernel), otherwise whenever the plan splits every tile of
+// a single matrix 2 or 4 ways on single-CTA tiles.
+bool clusterk_applies(const GemmArgs &g, int cta_group, const Plan &plan) {
+    if (tuning(PEAK_TUNE_CLUSTER_K) == 1) return false;
+    if (cta_group != 1 || g.nbatch() > 1 || plan.full_tiles != 0) return false;
+    if (plan.bn != 128 && plan.bn != 256) return false;
+    if (is_fp8(in_elem(g.dtype)) && !g.transB && plan.bn < 128) return false;
+    return plan.tail_splits == 2 || plan.tail_splits == 4;
+}
+
+template <int BN, int KC> int launch_clusterk_typed(const GemmArgs &g, const Plan &plan) {
+    const bool in8 = is_fp8(in_elem(g.dtype));
+    switch (out_elem(g.dtype)) {
+        case Elem::F32:
+            return in8 ? launch_clusterk<BN, float, KC, true>(g, plan) : launch_clusterk<BN, float, KC, false>(g, plan);
+        case Elem::F16: return launch_clusterk<BN, __half, KC, false>(g, plan);
+        case Elem::BF16:
+            return in8 ? launch_clusterk<BN, __nv_bfloat16, KC, true>(g, plan)
+                       : launch_clusterk<BN, __nv_bfloat16, KC, false>(g, plan);
+        default: break;
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
+template <int BN, int KC> int max_clusters_of() {
+    static int cached[kMaxDevices] = {};
+    static std::mutex m;
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return 0;
+    std::lock_guard<std::mutex> lock(m);
+    if (cached[dev] == 0) {
+        using C_ = Cfg<1, BN>;
+        auto kernel = umma_clusterk_kernel<BN, __nv_bfloat16, KC, false>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(KC * 64);
+        cfg.blockDim = dim3(ClusterKCfg<BN, KC>::THREADS);
+        cfg.dynamicSmemBytes = C_::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = KC; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        cached[dev] = n > 0 ? n : -1;
+    }
+    return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+int clusterk_max_clusters(int bn, int kc) {
+    if (bn == 128) return kc == 2 ? max_clusters_of<128, 2>() : max_clusters_of<128, 4>();
+    return kc == 2 ? max_clusters_of<256, 2>() : max_clusters_of<256, 4>();
+}
+
+int run_clusterk(const GemmArgs &g, const Plan &plan) {
+    if (plan.bn == 128)
+        return plan.tail_splits == 2 ? launch_clusterk_typed<128, 2>(g, plan) : launch_clusterk_typed<128, 4>(g, plan);
+    return plan.tail_splits == 2 ? launch_clusterk_typed<256, 2>(g, plan) : launch_clusterk_typed<256, 4>(g, plan);
+}
+
 // ---- exchanged operands for very skinny problems (M <= 64) -----------------------------------------------
 // C^T = op(B)^T op(A)^T: N takes the role of the MMA's M (128-row tiles over N) and M that of its N (one 64-wide
 // tile), so the small operand costs 8 KiB of shared memory and a few hundred bytes of traffic per k-block
@@ -515,6 +678,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         }
     }
     if (wide) plan = Plan{512, (int)tiles_of(g, 2, 512), 1};
+    if (clusterk_applies(g, cta_group, plan)) return run_clusterk(g, plan);
     if (cta_group == 2) {
         if (plan.bn == 512) return run_umma<2, 512>(g, plan, units);
         return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);

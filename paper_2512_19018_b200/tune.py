@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 17
+NUM_KEYS = 18
 
 
 def candidates(space: dict, quick: bool = False):
@@ -79,6 +79,7 @@ AXES_TENSOR = [
     (3, [0, 1, 2]),                 # PEAK_TUNE_EPILOGUE
     (13, [0, 1, 2]),                # PEAK_TUNE_K_ORDER
     (14, [0, 1, 2]),                # PEAK_TUNE_SWAP_AB
+    (17, [0, 1]),                   # PEAK_TUNE_CLUSTER_K
 ]
 AXES_F32 = [
     ("variant", ["auto"]),

@@ -682,6 +682,110 @@ def test_alternating_k_order_is_exact_and_repeatable(variant, reset_tuning):
         assert np.array_equal(dc.result(), first)
 
 
+# ------------------------------------------------------------------ k-slices on the CTAs of a cluster
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_cluster_k_slices_exact(ta, tb, reset_tuning):
+    """Every tile split 2 or 4 ways on single-CTA tiles runs as one launch: the slices on the CTAs of a cluster,
+    added through distributed shared memory in slice order.  Exact on integers for ragged M, N, K (several tile
+    rows, last slice shorter, slices narrower than a store chunk), every output type, 8-bit inputs, alpha / beta,
+    TMA and direct stores; the workspace path (PEAK_TUNE_CLUSTER_K = 1) gives the same bits."""
+    shapes = [(16, 4096, 1024), (1, 128, 512), (100, 1000, 2056), (128, 264, 1100), (300, 520, 1544), (130, 77, 4100)]
+    for idx, (M, N, K) in enumerate(shapes):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16, W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32):
+            in8 = dtype in (W.PEAK_E4M3_BF16, W.PEAK_E5M2_F32)
+            unit = 16 if in8 else 8
+            pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5 if dtype != W.PEAK_F16_F32 else 2.0,
+                   beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb, pad_c=[0, 8, 3][idx % 3], case=idx)
+            kblocks = (K + (127 if in8 else 63)) // (128 if in8 else 64)
+            for bn in (128, 256):
+                for split in (2, 4):
+                    per = (kblocks + split - 1) // split
+                    if per * (split - 1) >= kblocks:
+                        continue                                  # a slice would be empty: the library refuses
+                    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, bn)
+                    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+                    outs = []
+                    for mode in (0, 1):
+                        P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, mode)
+                        dc = R.DeviceCase(c)
+                        dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+                        name = P.peak_last_kernel()
+                        assert ("umma_clusterk_kernel<%d," % bn in name) == (mode == 0), name
+                        ref, _ = dc.oracle_full()
+                        want = oracle.round_to(R.OT[c.out_type], ref)
+                        got = dc.result()
+                        got = got.view(np.uint32) if c.out_type == "f32" else got
+                        assert np.array_equal(got, want), f"{c} bn={bn} split={split} cluster_k={mode}"
+                        outs.append(got.copy())
+                    assert np.array_equal(outs[0], outs[1])
+
+
+def test_cluster_k_real_values_fused_tail_and_selection(reset_tuning):
+    """Real-valued inputs through the cluster-split kernel with bias, GELU and a residual, run twice (bitwise
+    repeatable); and the dispatcher's own choice: a skinny problem whose 128-wide tiles fill a quarter of the SMs
+    runs four slices per tile in one launch."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(41)
+    for idx, (ta, tb, M, N, K, a, b) in enumerate([(1, 0, 16, 4096, 4096, 0.5, 2.0), (0, 1, 128, 1100, 2056, 1.0, 0.0),
+                                                   (0, 0, 200, 512, 1000, -1.0, 1.0), (1, 1, 5, 300, 1096, 2.0, 0.0)]):
+        pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+        c = W.GemmCase(f"ck{idx}", W.PEAK_BF16_BF16 if idx % 2 == 0 else W.PEAK_F16_F32, bool(ta), bool(tb), M, N, K, a, b,
+                       "uniform", pad_a=pa, pad_b=pb, pad_c=idx, case=idx)
+        for bn, split in ((128, 4), (256, 2)):
+            P.peak_set_tuning(P.PEAK_TUNE_TILE_N, bn)
+            P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+            dc = R.DeviceCase(c)
+            dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+            assert "umma_clusterk_kernel" in P.peak_last_kernel()
+            R.check_full(dc, what=f"{c} bn={bn} split={split}")
+            first = dc.result().copy()
+            dc.reset_c()
+            dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+            assert np.array_equal(first, dc.result())
+            bias = (rng.standard_normal(N) * 2).astype(np.float32)
+            res = make_residual(c, rng, idx)
+            dcf = run_fused(c, P.PEAK_VARIANT_UMMA_1CTA, bias, P.PEAK_ACT_GELU, res)
+            assert "umma_clusterk_kernel" in P.peak_last_kernel()
+            check_fused(dcf, bias, P.PEAK_ACT_GELU, f"cluster-k fused {c} bn={bn} split={split}", res)
+    for k in range(P.PEAK_TUNE_COUNT):
+        P.peak_set_tuning(k, 0)
+    c = W.config4_ragged(1)
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "umma_clusterk_kernel<128, __nv_bfloat16, 4, 0>" in P.peak_last_kernel(), P.peak_last_kernel()
+    R.check_full(dc, what=c.name)
+    P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, 1)
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "umma_gemm_kernel<1," in P.peak_last_kernel()
+    R.check_full(dc, what=c.name)
+
+
+def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
+    """The stalled-stage hook in the cluster-split kernel: the CTA whose stage never fills gives up after its
+    budget, still reaches both cluster barriers (its peers wait there, not on a flag), the status word reports the
+    timeout once and the context computes correctly afterwards."""
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 128, 512, 2048)
+    dc = R.DeviceCase(c)
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 128)
+    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 4)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 20)
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 1)
+    P.peak_gemm_variant(P.PEAK_VARIANT_UMMA_1CTA, c.dtype, c.transA, c.transB, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb,
+                        0.0, dc.C, c.ldc)
+    assert "umma_clusterk_kernel" in P.peak_last_kernel()
+    rc, detail = P.peak_check()
+    assert rc == P.PEAK_ERR_TIMEOUT and (detail & 0x80000000)
+    assert P.peak_check()[0] == P.PEAK_OK
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 0)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 0)
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+    assert "umma_clusterk_kernel" in P.peak_last_kernel()
+    R.check_full(dc)
+
+
 # ------------------------------------------------------------------ exchanged operands (M <= 64)
 @pytest.mark.parametrize("ta,tb", LAYOUTS)
 def test_swapped_operands_exact_and_selected(ta, tb, reset_tuning):
