@@ -312,7 +312,10 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_CLUSTER_K = 17,   /* a single matrix on single-CTA tiles whose every tile is split 2 or 4 ways: 1 = partial tiles
                                    through the workspace and a reduction kernel (default: the slices run on the CTAs of
                                    a cluster and are added through distributed shared memory, one launch) */
-    PEAK_TUNE_COUNT_ = 18
+    PEAK_TUNE_SHARE = 18,       /* single-GPU plug-in, 16-bit inputs: single-CTA tiles in clusters of CM x CN tiles that share
+                                   their A / B tiles by multicast copies: 1 = never, 100 * w + 10 * CM + CN (w = 1: 128-wide
+                                   tiles, 2: 256-wide) = that cluster shape whenever the plug-in is present */
+    PEAK_TUNE_COUNT_ = 19
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

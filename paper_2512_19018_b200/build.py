@@ -16,8 +16,10 @@ LIB = os.path.join(HERE, "libpeak_gemm.so")
 MC_SOURCE = os.path.join(CSRC, "umma_gemm_mc.cu")
 MC_LIB = os.path.join(HERE, "libpeak_gemm_mc.so")
 SOURCES = ["api.cu", "fallback_gemm.cu", "sgemm.cu", "sgemm_tma.cu", "tuned_table.cu", "umma_gemm.cu"]
-HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "ptx.cuh", "umma_device.cuh", "umma_host.cuh", "mc_plugin.h")] + [
+HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "ptx.cuh", "umma_device.cuh", "umma_clusterk.cuh", "umma_host.cuh",
+                                           "mc_plugin.h")] + [
     os.path.join(os.path.dirname(HERE), "include", "peak_gemm.h")]
+MC_HEADERS = [os.path.join(CSRC, "umma_share_mc.cuh")]  # plug-in only (multicast copies)
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 
@@ -59,7 +61,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-ldl"]
         subprocess.run(cmd, check=True)
         os.replace(tmp, LIB)
-    if os.path.exists(MC_SOURCE) and (force or _stale(MC_LIB, [MC_SOURCE] + HEADERS)):
+    if os.path.exists(MC_SOURCE) and (force or _stale(MC_LIB, [MC_SOURCE] + HEADERS + MC_HEADERS)):
         tmp = MC_LIB + f".tmp{os.getpid()}"
         cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-shared", MC_SOURCE, "-o", tmp]
         r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)

@@ -1,5 +1,6 @@
 // Interface between the main library and its optional single-GPU accelerator plug-in
-// (libpeak_gemm_mc.so): the tensor-core GEMM run by clusters of four CTAs that share B tiles.
+// (libpeak_gemm_mc.so): the tensor-core GEMM run by clusters of four CTAs that share B tiles, and single-CTA tiles
+// in clusters that share A and / or B tiles (problems with few tiles).
 // Plain C structs and one entry point, so that the two shared objects need nothing else from each other.
 //
 // Contract: the plug-in is for single-GPU processes.  Its tensor maps must cover memory of the GPU it runs on
@@ -35,6 +36,8 @@ struct peak_mc_request {
     const void *R;          // fused epilogue: residual matrix (output type, device) or NULL
     int64_t ldr;
     int k_order;            // PEAK_TUNE_K_ORDER value
+    int share_cm, share_cn; // both 0: CTA-pair tiles as described above; otherwise single-CTA 128 x tile_n tiles (tile_n
+                            // 128 or 256) in clusters of share_cm x share_cn tiles that share their A / B tiles
     int cuda_error;         // out: cudaError_t of a failing CUDA call
 };
 

@@ -1,19 +1,26 @@
-// Split-K inside one launch (the paper's Split-K transformation, section 4.1, for problems with too few tiles
-// to fill the GPU): the KC k-slices of an output tile run on the KC CTAs of a thread-block cluster, each with
-// its own fp32 accumulator in tensor memory, and are added through distributed shared memory instead of through
-// a workspace and a second kernel.
+// One-tile-per-CTA tensor-core kernel for problems whose tiles all run at once (single-CTA 128 x BN tiles, single
+// matrices), with split-K inside the launch (the paper's Split-K transformation, section 4.1, for problems with
+// too few tiles to fill the GPU): the KC k-slices of an output tile run on the KC CTAs of a thread-block cluster,
+// each with its own fp32 accumulators in tensor memory, and are added through distributed shared memory instead
+// of through a workspace and a second kernel.  KC = 1 is the same kernel without a cluster: whole tiles.
 //
-//   main loop   as in umma_gemm_kernel with single-CTA tiles: warp 0 feeds a ring of 128-byte-swizzled stages by
-//               TMA, one thread of warp 1 issues tcgen05.mma over this CTA's k-blocks;
-//   exchange    the tile's BN columns are divided into KC column slices, one per CTA.  When every CTA of the
-//               cluster has finished its main loop (cluster barrier 1: the stage ring is free everywhere), each
-//               epilogue thread copies, for every other CTA d, its row of slice d from tensor memory into a
-//               receive area in CTA d's ring (st.shared::cluster, swizzled like the staging buffers so that the
-//               32 lanes of a warp hit different banks);
-//   reduction   after cluster barrier 2 each CTA adds the KC partials of its own slice in slice order 0..KC-1
-//               (its own from tensor memory at its position in that order), writes the sums back to tensor
-//               memory and runs the ordinary tile epilogue (alpha/beta, bias, activation, residual, TMA or
-//               direct stores) over its slice.
+//   main loop   a ring of 128-byte-swizzled stages fed by TMA and consumed by tcgen05.mma, with the issuing work
+//               spread over more threads than in umma_gemm_kernel: two producer warps take the k-blocks in turn
+//               and issue the copies of a stage from several lanes in one instruction; with 128-wide tiles two
+//               MMA issuers take the k-blocks in turn as well, each accumulating into its own half of tensor
+//               memory.  (A 128 x 128 x 64 k-block is 256 tensor cycles, while one thread needs about 540 cycles
+//               per k-block for barrier wait, fence, descriptors, four MMAs and commit: measured, the main loop
+//               of 512x4096x4096 went from 540 to 413 cycles per k-block, where the operand stream takes over.)
+//   exchange    (KC > 1) the tile's BN columns are divided into KC column slices, one per CTA.  When every CTA of
+//               the cluster has finished its main loop (cluster barrier 1: the stage ring is free everywhere),
+//               each epilogue thread copies, for every other CTA d, its row of slice d (both accumulators added)
+//               into a receive area in CTA d's ring (st.shared::cluster, swizzled like the staging buffers so
+//               that the 32 lanes of a warp hit different banks);
+//   reduction   (KC > 1) after cluster barrier 2 each CTA adds the KC partials of its own slice in slice order
+//               0..KC-1 (its own at its position in that order) and writes the sums back to tensor memory;
+//   epilogue    the ordinary tile epilogue (alpha/beta, bias, activation, residual, TMA or direct stores) over the
+//               slice -- or, for KC = 1, over the whole tile by two groups of four warps that read and add both
+//               accumulators.
 // The order of the additions is fixed by the launch, so results are run-to-run identical.  Every mbarrier wait
 // is bounded; the two cluster barriers are reached by every thread whether or not a wait gave up, so a CTA
 // whose wait ran out cannot leave its peers waiting.
@@ -28,15 +35,24 @@ template <int BN, int KC> struct ClusterKCfg {
     static constexpr int SW = BN / KC;            // columns each CTA finalises
     static constexpr int CHUNKS = SW / 32;        // 32-column chunks per slice
     static constexpr int RECV_BYTES = KC * CHUNKS * BM * 128;  // [source CTA][chunk][row][128 bytes]
-    static constexpr int TMEM_COLS = 256;         // BN accumulator columns (+ slack for a 64-wide chunk read)
-    static constexpr int THREADS = 192;
+    // Two MMA issuers, each with an accumulator of its own, take the k-blocks in turn (128-wide tiles: both
+    // accumulators fit 256 columns of tensor memory; 256-wide tiles keep one issuer).
+    static constexpr bool DUAL = BN == 128;
+    static constexpr int TMEM_COLS = 256;         // accumulator columns (+ slack for a 64-wide chunk read)
+    // warps: 0 producer, 1 MMA issuer, then GROUPS groups of four epilogue warps, second producer, second issuer.  Whole
+    // tiles (KC = 1) are drained by two groups, half of the columns each; a column slice of a split tile by one.
+    static constexpr int GROUPS = KC == 1 ? 2 : 1;
+    static constexpr int PRODUCER2 = 2 + 4 * GROUPS;
+    static constexpr int ISSUER2 = PRODUCER2 + 1;
+    static constexpr int THREADS = 32 * (ISSUER2 + 1);
+    static_assert(KC == 1 || KC == 2 || KC == 4, "cluster sizes");
     static_assert(SW % 32 == 0 && SW >= 32, "a slice is a whole number of 32-column chunks");
     static_assert(RECV_BYTES <= C_::STAGES * C_::STAGE_BYTES, "the receive area lives in the stage ring");
-    static_assert(BN + 32 <= TMEM_COLS || SW >= 64, "a 16-bit chunk read may look 32 columns past the slice");
+    static_assert((DUAL ? 2 : 1) * BN <= TMEM_COLS, "accumulators fit the allocation");
 };
 
 template <int BN, typename TOut, int KC, bool IN8>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__((ClusterKCfg<BN, KC>::THREADS), 1)
 umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
     using C_ = Cfg<1, BN>;
@@ -61,7 +77,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     constexpr int MN_ATOM = IN8 ? 2 * ATOM_BYTES : ATOM_BYTES;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t me = ptx::cluster_ctarank();  // k-slice of this CTA, and the column slice it finalises
+    const uint32_t me = KC > 1 ? ptx::cluster_ctarank() : 0u;  // k-slice of this CTA, and the column slice it finalises
     const int tile = blockIdx.x / KC;
 
     if (threadIdx.x == 0) {
@@ -69,7 +85,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::mbar_init(full0 + 8 * s, 1);
             ptx::mbar_init(empty0 + 8 * s, 1);
         }
-        ptx::mbar_init(accfull, 1);
+        ptx::mbar_init(accfull, K_::DUAL ? 2 : 1);
         for (int b = 0; b < 8; ++b) ptx::mbar_init(cbar0 + 8 * b, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -99,53 +115,62 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);  // the host guarantees kb0 < kb1
     bool ok = true;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                if (!ptx::mbar_wait<false>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles)) {
-                    report_timeout(p, abort_flag, 1, s);
-                    break;
-                }
-                if (p.inject_stall && blockIdx.x == 0 && kb == kb1 - 1)
-                    continue;  // test hook: leave this stage empty so that the waits downstream run out
-                const uint32_t bar = full0 + 8 * s;
-                ptx::mbar_arrive_expect_tx(bar, p.stage_tx);
-                const uint32_t a_dst = stage_base + s * C_::STAGE_BYTES;
-                const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                const int k0 = kb * (IN8 ? 2 * BK : BK);
-                if (!p.a_mn) {
-                    ptx::tma_load_2d(a_dst, &tmA, k0, m0, bar);
-                } else {
-#pragma unroll
-                    for (int h = 0; h < BM / MN_ELEMS; ++h) {
-                        if (h >= p.a_boxes) break;
-                        ptx::tma_load_2d(a_dst + h * MN_ATOM, &tmA, m0 + MN_ELEMS * h, k0, bar);
-                    }
-                }
-                if (!p.b_mn) {
-#pragma unroll
-                    for (int h = 0; h < C_::HROWS / C_::B_BOX_ROWS; ++h)
-                        ptx::tma_load_2d(b_dst + h * C_::B_BOX_ROWS * 128, &tmB, k0, n0 + C_::B_BOX_ROWS * h, bar);
-                } else {
-#pragma unroll
-                    for (int h = 0; h < C_::HROWS / MN_ELEMS; ++h)
-                        ptx::tma_load_2d(b_dst + h * MN_ATOM, &tmB, n0 + MN_ELEMS * h, k0, bar);
-                }
+    if (warp == 0 || warp == K_::PRODUCER2) {
+        // ------------------------------------------------------------------ producers
+        // Two warps take the k-blocks in turn, and inside a warp every copy of a stage is issued by a lane of its
+        // own in one instruction: a copy instruction occupies its thread for a few hundred cycles, and with a
+        // 128 x BN tile a k-block is only 2 * BN tensor cycles long, so one thread issuing everything is what
+        // bounds the main loop (measured on a copy-only kernel: 1100 cycles per k-block with one thread, 420 with
+        // two warps of two lanes).
+        const int pw = warp == 0 ? 0 : 1;
+        // this lane's copy within a stage: A boxes first, then B boxes
+        const int a_ops = p.a_mn ? p.a_boxes : 1;
+        const int b_ops = p.b_mn ? C_::HROWS / MN_ELEMS : C_::HROWS / C_::B_BOX_ROWS;
+        const bool mine = lane < a_ops + b_ops;
+        const bool is_a = lane < a_ops;
+        const int h = is_a ? lane : lane - a_ops;
+        const CUtensorMap *tmap = is_a ? &tmA : &tmB;
+        const bool mn = is_a ? p.a_mn != 0 : p.b_mn != 0;
+        const int mn0 = (is_a ? m0 : n0) + h * (mn ? MN_ELEMS : (is_a ? 0 : C_::B_BOX_ROWS));
+        const uint32_t off = (is_a ? 0u : (uint32_t)A_STAGE_BYTES) +
+                             (uint32_t)h * (mn ? (uint32_t)MN_ATOM : (uint32_t)(C_::B_BOX_ROWS * 128));
+        uint32_t it = (uint32_t)pw;
+        for (int kb = kb0 + pw; kb < kb1; kb += 2, it += 2) {
+            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+            const uint32_t bar = full0 + 8 * s;
+            bool go = true;
+            if (lane == 0) {
+                go = ptx::mbar_wait<false>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles);
+                if (!go) report_timeout(p, abort_flag, 1, s);
+                else if (!(p.inject_stall && blockIdx.x == 0 && kb == kb1 - 1)) ptx::mbar_arrive_expect_tx(bar, p.stage_tx);
             }
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (!go) break;
+            if (p.inject_stall && blockIdx.x == 0 && kb == kb1 - 1)
+                continue;  // test hook: leave this stage empty so that the waits downstream run out
+            if (mine) {
+                const int k0 = kb * (IN8 ? 2 * BK : BK);
+                const uint32_t dst = stage_base + s * C_::STAGE_BYTES + off;
+                ptx::tma_load_2d(dst, tmap, mn ? mn0 : k0, mn ? k0 : mn0, bar);  // one instruction for all lanes
+            }
+            __syncwarp();
         }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+    } else if (warp == 1 || warp == K_::ISSUER2) {
+        // ------------------------------------------------------------------ MMA issuers
+        // With 128-wide tiles the four MMAs of a k-block keep the tensor pipe busy for about 380 cycles while the
+        // issuing thread needs about 540 per k-block (barrier wait, fence, descriptors, commit), so two threads
+        // take the k-blocks in turn, each accumulating into its own half of tensor memory; the halves are added
+        // when the accumulators are read.
+        constexpr int NI = K_::DUAL ? 2 : 1;
+        const int iw = warp == 1 ? 0 : 1;
+        if (lane == 0 && iw < NI) {
             const uint32_t a_lbo = p.a_mn ? (uint32_t)MN_ATOM : 16u, b_lbo = p.b_mn ? (uint32_t)MN_ATOM : 16u;
             constexpr uint32_t MN_KSTEP = IN8 ? 4096u : 2048u;
             const uint32_t a_kstep = p.a_mn ? MN_KSTEP : 32u, b_kstep = p.b_mn ? MN_KSTEP : 32u;
-            uint32_t it = 0;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(iw * BN);
+            uint32_t it = (uint32_t)iw;
             bool mma_ok = true;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            for (int kb = kb0 + iw; kb < kb1; kb += NI, it += NI) {
                 const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                 if (!ptx::mbar_wait<false>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
                     report_timeout(p, abort_flag, 4, s);
@@ -159,16 +184,16 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 for (int k = 0; k < BK / UMMA_K; ++k) {
                     const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
                     const uint64_t bd = smem_desc(b_base + k * b_kstep, b_lbo, 1024u);
-                    if (IN8) ptx::umma_f8<1>(tmem_base, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
-                    else ptx::umma_f16<1>(tmem_base, ad, bd, p.idesc, (uint32_t)((kb > kb0) | (k != 0)));
+                    if (IN8) ptx::umma_f8<1>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
+                    else ptx::umma_f16<1>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
                 }
                 ptx::umma_commit_1cta(empty0 + 8 * s);
             }
-            if (mma_ok) ptx::umma_commit_1cta(accfull);
+            if (mma_ok) ptx::umma_commit_1cta(accfull);  // (an issuer without k-blocks arrives at once)
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue warps: wait for the accumulator
+        // ------------------------------------------------------------------ epilogue warps (2..5): wait for the accumulator
         const bool got = ptx::mbar_wait<false>(accfull, 0u, abort_flag, p.wait_cycles);
         ok = __all_sync(0xffffffffu, got);
         if (!ok && lane == 0) report_timeout(p, abort_flag, 5, 0);
@@ -176,13 +201,28 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
 
     // cluster barrier 1: every CTA's main loop is over (or has given up), so every stage ring may be overwritten
-    ptx::cluster_sync();
+    if (KC > 1) ptx::cluster_sync();
 
     const int q = warp & 3;                       // TMEM lane quadrant of an epilogue warp
     const int row0 = m0 + q * 32;                 // first row of this warp
-    const bool live = warp >= 2 && ok && row0 < p.M;
+    const bool live = warp >= 2 && warp < K_::PRODUCER2 && ok && row0 < p.M;
     const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
     const int trow = q * 32 + lane;               // row inside the tile
+    // this CTA's partial sums of 32 columns: the first issuer's accumulator plus, when the second issuer had
+    // k-blocks of its own, the second's
+    const bool two_acc = K_::DUAL && kb1 - kb0 >= 2;
+    auto load_partial = [&](int col, uint32_t (&r)[32]) {
+        ptx::tmem_ld_32x32(t_row + (uint32_t)col, r);
+        if (two_acc) {
+            uint32_t r2[32];
+            ptx::tmem_ld_32x32(t_row + (uint32_t)(BN + col), r2);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+        } else {
+            ptx::tmem_ld_wait();
+        }
+    };
     if (live) {
         // ------------------------------------------------------------------ exchange
 #pragma unroll 1
@@ -191,8 +231,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll 1
             for (int c = 0; c < K_::CHUNKS; ++c) {
                 uint32_t r[32];
-                ptx::tmem_ld_32x32(t_row + d * SW + c * 32, r);
-                ptx::tmem_ld_wait();
+                load_partial((int)d * SW + c * 32, r);
                 if (m0 + trow < p.M) {
                     const uint32_t local = stage_base + (uint32_t)(((int)me * K_::CHUNKS + c) * BM + trow) * 128u;
                     const uint32_t remote = ptx::map_to_cta(local, d);
@@ -206,16 +245,15 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
 
     // cluster barrier 2: all partials have arrived (release / acquire at cluster scope)
-    ptx::cluster_sync();
+    if (KC > 1) ptx::cluster_sync();
 
     if (live) {
         // ------------------------------------------------------------------ reduction of this CTA's slice
 #pragma unroll 1
-        for (int c = 0; c < K_::CHUNKS; ++c) {
+        for (int c = 0; c < K_::CHUNKS && KC > 1; ++c) {
             uint32_t own[32];
             const uint32_t t_addr = t_row + me * SW + c * 32;
-            ptx::tmem_ld_32x32(t_addr, own);
-            ptx::tmem_ld_wait();
+            load_partial((int)me * SW + c * 32, own);
             float acc[32];
 #pragma unroll 1
             for (uint32_t src = 0; src < (uint32_t)KC; ++src) {
@@ -252,23 +290,30 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::tmem_st_wait();
         // ------------------------------------------------------------------ tile epilogue over the slice
         constexpr int CC = 128 / (int)sizeof(TOut);        // columns per staged chunk
-        constexpr int W = SW < CC ? CC : SW;               // a slice narrower than a chunk takes the direct stores
-        const bool tma = p.tma_store != 0 && SW >= CC;
-        const int c_first = n0 + (int)me * SW;
-        const int c_limit = min(p.N, c_first + SW);
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
-        CFetch cf{cbar0 + 16u * (uint32_t)(warp - 2), 0u, tma && p.c_prefetch != 0, false};
+        constexpr int GW = SW / K_::GROUPS;                // columns this warp's group drains
+        constexpr int W = GW < CC ? CC : GW;               // a slice narrower than a chunk takes the direct stores
+        const int grp = (warp - 2) >> 2;
+        const bool tma = p.tma_store != 0 && GW >= CC;
+        const int c_first = n0 + (int)me * SW + grp * GW;
+        const int c_limit = min(p.N, c_first + GW);
+        // staging: two buffers per warp with one group, one per warp with two
+        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (K_::GROUPS == 1 ? 2u : 1u) * EPI_BUF_BYTES;
+        CFetch cf{K_::GROUPS == 1 ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
+                  tma && p.c_prefetch != 0, K_::GROUPS == 2};
         if (c_first < p.N) {
             if (cf.on && lane == 0) {
                 cfetch_issue<TOut, false>(cf, my_stage, 0, &tmC, c_first, row0, 0);
-                if (c_first + CC < c_limit) cfetch_issue<TOut, false>(cf, my_stage, 1, &tmC, c_first, row0, 0);
+                if (!cf.single && c_first + CC < c_limit) cfetch_issue<TOut, false>(cf, my_stage, 1, &tmC, c_first, row0, 0);
             }
             __syncwarp();
-            if (!epilogue_tile<TOut, W, false>(t_row + me * SW, my_stage, lane, reinterpret_cast<TOut *>(p.C), p.ldc,
-                                               row0 + lane, row0, p.M, c_first, c_limit, &tmC, c_first, row0, 0, tma,
-                                               p.vec_ok != 0, p.alpha, p.beta, p.bias, p.act,
-                                               reinterpret_cast<const TOut *>(p.R), p.ldr, p.r_vec != 0, cf, abort_flag,
-                                               p.wait_cycles)) {
+            const uint32_t t_first = t_row + me * SW + (uint32_t)(grp * GW);
+            // a whole tile (KC = 1) is read from both issuers' accumulators; a slice's sums were written back above
+            const uint32_t t_second = (KC == 1 && two_acc) ? t_first + BN : 0u;
+            if (!epilogue_tile<TOut, W, false, KC == 1>(t_first, my_stage, lane, reinterpret_cast<TOut *>(p.C), p.ldc,
+                                                        row0 + lane, row0, p.M, c_first, c_limit, &tmC, c_first, row0, 0, tma,
+                                                        p.vec_ok != 0, p.alpha, p.beta, p.bias, p.act,
+                                                        reinterpret_cast<const TOut *>(p.R), p.ldr, p.r_vec != 0, cf,
+                                                        abort_flag, p.wait_cycles, t_second)) {
                 if (lane == 0) report_timeout(p, abort_flag, 6, 0);
             }
         }

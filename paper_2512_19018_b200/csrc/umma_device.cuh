@@ -291,13 +291,16 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
 // store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
 // column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
 // (z0 is used when MAP3D says that `tm` is three-dimensional).
-template <typename T, int BN, bool MAP3D = false>
+// ACC2: the tile's sums are split over two accumulators (t_addr and, when nonzero, t_addr2: two MMA issuers that
+// took the k-blocks in turn); they are added as they are read.
+template <typename T, int BN, bool MAP3D = false, bool ACC2 = false>
 __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
                                               bool vec, float alpha, float beta, const float *bias, int act,
                                               const T *rbase, int64_t ldr, bool rvec, CFetch &cf,
-                                              volatile uint32_t *abort_flag, long long wait_cycles) {
+                                              volatile uint32_t *abort_flag, long long wait_cycles,
+                                              uint32_t t_addr2 = 0u) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
@@ -309,6 +312,18 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
 #pragma unroll
         for (int h = 0; h < CHUNK_COLS / 32; ++h) ptx::tmem_ld_32x32(t_addr + c * CHUNK_COLS + h * 32, r[h]);
         ptx::tmem_ld_wait();
+        if constexpr (ACC2) {
+            if (t_addr2 != 0u) {
+#pragma unroll
+                for (int h = 0; h < CHUNK_COLS / 32; ++h) {
+                    uint32_t r2[32];
+                    ptx::tmem_ld_32x32(t_addr2 + c * CHUNK_COLS + h * 32, r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[h][i] = __float_as_uint(__uint_as_float(r[h][i]) + __uint_as_float(r2[i]));
+                }
+            }
+        }
         if (cf.on) {
             // chunks 0 and 1 were requested before the accumulator was waited for; chunk c + 1 (c >= 1) goes
             // into the buffer chunk c - 1 left by a store, which has had this chunk's tensor-memory load to

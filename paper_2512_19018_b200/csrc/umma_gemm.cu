@@ -479,9 +479,11 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
 // a single matrix 2 or 4 ways on single-CTA tiles.
 bool clusterk_applies(const GemmArgs &g, int cta_group, const Plan &plan) {
     if (tuning(PEAK_TUNE_CLUSTER_K) == 1) return false;
-    if (cta_group != 1 || g.nbatch() > 1 || plan.full_tiles != 0) return false;
+    if (cta_group != 1 || g.nbatch() > 1) return false;
     if (plan.bn != 128 && plan.bn != 256) return false;
-    if (is_fp8(in_elem(g.dtype)) && !g.transB && plan.bn < 128) return false;
+    // whole tiles that all run at once: the same kernel without a cluster (one tile per CTA, two MMA issuers)
+    if (plan.tail_splits == 1) return plan.bn == 128 && plan.full_tiles <= sm_count();
+    if (plan.full_tiles != 0) return false;
     return plan.tail_splits == 2 || plan.tail_splits == 4;
 }
 
@@ -532,6 +534,7 @@ int clusterk_max_clusters(int bn, int kc) {
 }
 
 int run_clusterk(const GemmArgs &g, const Plan &plan) {
+    if (plan.tail_splits == 1) return launch_clusterk_typed<128, 1>(g, plan);
     if (plan.bn == 128)
         return plan.tail_splits == 2 ? launch_clusterk_typed<128, 2>(g, plan) : launch_clusterk_typed<128, 4>(g, plan);
     return plan.tail_splits == 2 ? launch_clusterk_typed<256, 2>(g, plan) : launch_clusterk_typed<256, 4>(g, plan);
@@ -565,6 +568,21 @@ bool swap_applies(const GemmArgs &g) {
     const int mode = tuning(PEAK_TUNE_SWAP_AB);
     if (mode != 2 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype)) || g.M > 64 || g.N < 128) return false;
     return true;
+}
+
+// Shared-operand clusters of single-CTA tiles (plug-in).  PEAK_TUNE_SHARE: 1 = never; 100 * w + 10 * CM + CN with
+// w = 1 (128-wide tiles) or 2 (256-wide) forces a cluster shape; 0 = the built-in rule.
+bool share_applies(const GemmArgs &g, int &bn, int &cm, int &cn) {
+    const int mode = tuning(PEAK_TUNE_SHARE);
+    if (mode == 1 || tuning(PEAK_TUNE_MULTICAST) == 1 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype)) || !mc_entry())
+        return false;
+    if (mode >= 100) {
+        bn = mode / 100 == 2 ? 256 : 128;
+        cm = mode / 10 % 10;
+        cn = mode % 10;
+        return true;
+    }
+    return false;
 }
 
 int launch_swapped(const GemmArgs &g) {
@@ -620,6 +638,28 @@ int umma_units(int cta_group) { return sm_count() / (cta_group == 2 ? 2 : 1); }
 int launch_umma(const GemmArgs &g, int cta_group) {
     if (!umma_supports(g, cta_group)) return PEAK_ERR_UNSUPPORTED;
     if (cta_group == 1 && swap_applies(g)) return launch_swapped(g);
+    {
+        // Single-CTA tiles in clusters that share operand tiles by multicast (single-GPU plug-in).
+        int bn = 0, cm = 0, cn = 0;
+        if (share_applies(g, bn, cm, cn)) {
+            peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
+                              g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
+                              tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),
+                              tuning(PEAK_TUNE_INJECT_STALL), tuning(PEAK_TUNE_BALANCED_GRID), g.bias, g.act,
+                              tuning(PEAK_TUNE_EPILOGUE_WARPS), bn, g.R, g.ldr, tuning(PEAK_TUNE_K_ORDER), cm, cn, 0};
+            if (!r.status) return PEAK_ERR_CUDA;
+            const int rc = mc_entry()(&r);
+            if (rc == PEAK_OK) {
+                count_launch();
+                const Elem eo = out_elem(g.dtype);
+                note_kernel("umma_share_kernel<%d, %s, %d, %d> (cluster-multicast plug-in)", bn,
+                            eo == Elem::F32 ? "float" : (eo == Elem::F16 ? "__half" : "__nv_bfloat16"), cm, cn);
+                return rc;
+            }
+            if (rc == PEAK_ERR_CUDA) { set_cuda_error((cudaError_t)r.cuda_error); return rc; }
+            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+        }
+    }
     const int units = sm_count() / cta_group;
     Plan plan = choose_plan(g, cta_group, units);
     const bool in8 = is_fp8(in_elem(g.dtype));

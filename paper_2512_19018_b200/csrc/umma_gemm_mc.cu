@@ -22,6 +22,7 @@ template <int MC> struct McOps;
 }  // namespace peak
 
 #include "umma_device.cuh"
+#include "umma_share_mc.cuh"
 #include "umma_host.cuh"
 #include "mc_plugin.h"
 
@@ -148,6 +149,105 @@ template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(
     return PEAK_OK;
 }
 
+// Single-CTA tiles in clusters of CM x CN tiles with shared operand tiles (umma_share_mc.cuh).  16-bit inputs.
+template <int BN, typename TOut, int CM, int CN> int launch_share(peak_mc_request *r) {
+    using C_ = Cfg<1, BN>;
+    using S_ = ShareCfg<BN, CM, CN>;
+    auto kernel = umma_share_kernel<BN, TOut, CM, CN>;
+    const int dev = current_device();
+    static PerDeviceOnce attr_once;
+    const cudaError_t attr_err = attr_once.run(dev, [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+    });
+    if (attr_err != cudaSuccess) { r->cuda_error = (int)attr_err; return PEAK_ERR_CUDA; }
+    const Elem ein = in_elem(r->dtype), eout = out_elem(r->dtype);
+    const int a_mn = r->transA ? 1 : 0, b_mn = r->transB ? 0 : 1;
+    CUtensorMap tmA, tmB, tmC;
+    // one box per operand part: K-major `part` matrix rows of one k-block; MN-major 64 elements of M / N by up to
+    // 64 k-rows
+    constexpr int A_BOX_K = S_::A_PART < 64 ? S_::A_PART : 64, B_BOX_K = S_::B_PART < 64 ? S_::B_PART : 64;
+    bool ok = a_mn ? make_map(&tmA, ein, r->A, r->M, r->K, r->lda, 64, A_BOX_K)
+                   : make_map(&tmA, ein, r->A, r->K, r->M, r->lda, BK, S_::A_PART);
+    ok = ok && (b_mn ? make_map(&tmB, ein, r->B, r->N, r->K, r->ldb, 64, B_BOX_K)
+                     : make_map(&tmB, ein, r->B, r->K, r->N, r->ldb, BK, S_::B_PART));
+    if (!ok) return PEAK_ERR_CUDA;
+
+    UmmaParams p = {};
+    p.M = (int)r->M; p.N = (int)r->N; p.K = (int)r->K;
+    p.num_kb = (int)((r->K + BK - 1) / BK);
+    p.tiles_m = (int)((r->M + CM * BM - 1) / (CM * BM));   // super-tiles
+    p.tiles_n = (int)((r->N + CN * BN - 1) / (CN * BN));
+    p.group = r->raster_group > 0 ? r->raster_group : 16;
+    const int super_tiles = p.tiles_m * p.tiles_n;
+    p.tiles_per_batch = super_tiles;
+    p.full_tiles = super_tiles; p.tail_splits = 1; p.kb_per_split = p.num_kb; p.total_items = super_tiles;
+    p.a_mn = a_mn; p.b_mn = b_mn;
+    const uint32_t fmt = (ein == Elem::BF16) ? 1u : 0u;
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    p.alpha = r->alpha; p.beta = r->beta;
+    p.C = r->C; p.ldc = r->ldc;
+    p.bias = r->bias; p.act = r->activation;
+    const int ob = elem_bytes(eout);
+    p.R = r->R; p.ldr = r->ldr;
+    p.r_vec = (r->R && reinterpret_cast<uintptr_t>(r->R) % 16 == 0 && (r->ldr * ob) % 16 == 0) ? 1 : 0;
+    p.vec_ok = ((reinterpret_cast<uintptr_t>(r->C) % 16) == 0 && (r->ldc * ob) % 16 == 0) ? 1 : 0;
+    p.tma_store = (p.vec_ok && (r->N * ob) % 16 == 0 && r->epilogue != 1) ? 1 : 0;
+    tmC = tmA;
+    p.c_prefetch = (p.tma_store && r->beta != 0.0f && r->epilogue != 3) ? 1 : 0;
+    if (p.tma_store && !make_map(&tmC, eout, r->C, r->N, r->M, r->ldc, 128 / ob, 32)) return PEAK_ERR_CUDA;
+    p.a_boxes = BM / 64; p.stage_tx = (uint32_t)C_::STAGE_BYTES;
+    p.status = r->status;
+    p.wait_cycles = r->wait_ms > 0 ? (long long)r->wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
+    p.inject_stall = r->inject_stall == 1 ? 1 : 0;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(super_tiles * S_::CL));
+    cfg.blockDim = dim3(S_::THREADS);
+    cfg.dynamicSmemBytes = C_::SMEM_BYTES;
+    cfg.stream = r->stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S_::CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = r->dependent_launch == 1 ? 1 : 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+    if (e != cudaSuccess) { r->cuda_error = (int)e; return PEAK_ERR_CUDA; }
+    return PEAK_OK;
+}
+
+template <int BN, int CM, int CN> int launch_share_typed(peak_mc_request *r) {
+    switch (out_elem(r->dtype)) {
+        case Elem::F32: return launch_share<BN, float, CM, CN>(r);
+        case Elem::F16: return launch_share<BN, __half, CM, CN>(r);
+        case Elem::BF16: return launch_share<BN, __nv_bfloat16, CM, CN>(r);
+        default: break;
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
+int run_share(peak_mc_request *r) {
+    if (is_fp8(in_elem(r->dtype))) return PEAK_ERR_UNSUPPORTED;
+    const int key = r->tile_n * 100 + r->share_cm * 10 + r->share_cn;
+    switch (key) {
+        case 12812: return launch_share_typed<128, 1, 2>(r);
+        case 12814: return launch_share_typed<128, 1, 4>(r);
+        case 12821: return launch_share_typed<128, 2, 1>(r);
+        case 12822: return launch_share_typed<128, 2, 2>(r);
+        case 12824: return launch_share_typed<128, 2, 4>(r);
+        case 12841: return launch_share_typed<128, 4, 1>(r);
+        case 12842: return launch_share_typed<128, 4, 2>(r);
+        case 25612: return launch_share_typed<256, 1, 2>(r);
+        case 25614: return launch_share_typed<256, 1, 4>(r);
+        case 25621: return launch_share_typed<256, 2, 1>(r);
+        case 25622: return launch_share_typed<256, 2, 2>(r);
+        default: break;
+    }
+    return PEAK_ERR_UNSUPPORTED;
+}
+
 }  // namespace
 }  // namespace peak
 
@@ -168,6 +268,7 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
             !local_device_memory(b0) || !local_device_memory(b0 + ((b_rows - 1) * r->ldb + b_cols) * ib - 1))
             return PEAK_ERR_UNSUPPORTED;
     }
+    if (r->share_cm > 0 || r->share_cn > 0) return run_share(r);
     // two groups of epilogue warps when the launch is at most two waves of 512 x 256 super-tiles long (the
     // last tile's epilogue is then a visible part of the run time)
     const int64_t super_tiles = ((r->M + 511) / 512) * ((r->N + 255) / 256);

@@ -762,6 +762,49 @@ def test_cluster_k_real_values_fused_tail_and_selection(reset_tuning):
     R.check_full(dc, what=c.name)
 
 
+def test_one_tile_per_cta_kernel_two_issuers_exact(reset_tuning):
+    """Whole 128-wide tiles that all run at once take the one-tile-per-CTA kernel without a cluster: two MMA
+    issuers accumulate the even and the odd k-blocks separately and the epilogue adds them.  Exact on integers in
+    every layout for one k-block (second accumulator never written), odd and even counts, ragged edges, every
+    output type, beta != 0 with TMA and direct stores; real values within the bounds, bitwise repeatable; the
+    persistent kernel (PEAK_TUNE_CLUSTER_K = 1) gives the same bits on integers."""
+    shapes = [(128, 1024, 64), (100, 1000, 136), (300, 520, 1544), (128, 4100, 520), (512, 1280, 4096), (7, 130, 200)]
+    for ta, tb in LAYOUTS:
+        for idx, (M, N, K) in enumerate(shapes):
+            for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16, W.PEAK_E4M3_BF16):
+                unit = 16 if dtype == W.PEAK_E4M3_BF16 else 8
+                pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
+                c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa,
+                       pad_b=pb, pad_c=[0, 8, 3][idx % 3], case=idx)
+                P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 128)
+                P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 1)
+                outs = []
+                for mode in (0, 1):
+                    P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, mode)
+                    dc = R.DeviceCase(c)
+                    dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+                    name = P.peak_last_kernel()
+                    assert ("umma_clusterk_kernel<128," in name and ", 1, " in name) == (mode == 0), name
+                    ref, _ = dc.oracle_full()
+                    want = oracle.round_to(R.OT[c.out_type], ref)
+                    got = dc.result()
+                    got = got.view(np.uint32) if c.out_type == "f32" else got
+                    assert np.array_equal(got, want), f"{c} cluster_k={mode}"
+                    outs.append(got.copy())
+                assert np.array_equal(outs[0], outs[1])
+    for k in range(P.PEAK_TUNE_COUNT):
+        P.peak_set_tuning(k, 0)
+    c = mk(W.PEAK_BF16_BF16, 1, 0, 128, 14336, 1024, alpha=0.5, beta=2.0)
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "umma_clusterk_kernel<128, __nv_bfloat16, 1, 0>" in P.peak_last_kernel(), P.peak_last_kernel()
+    R.check_full(dc, what=f"{c}")
+    first = dc.result().copy()
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert np.array_equal(first, dc.result())
+
+
 def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
     """The stalled-stage hook in the cluster-split kernel: the CTA whose stage never fills gives up after its
     budget, still reaches both cluster barriers (its peers wait there, not on a flag), the status word reports the
@@ -783,6 +826,58 @@ def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
     dc.reset_c()
     dc.run(P.PEAK_VARIANT_UMMA_1CTA)
     assert "umma_clusterk_kernel" in P.peak_last_kernel()
+    R.check_full(dc)
+
+
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_shared_operand_clusters_plugin_exact(ta, tb, reset_tuning):
+    """The plug-in's single-CTA tiles in clusters of CM x CN tiles that share A / B tiles by multicast copies
+    (PEAK_TUNE_SHARE = 100 w + 10 CM + CN): every cluster shape, exact on integers for ragged shapes (clusters
+    that reach beyond the matrix), alpha / beta, 16-bit and fp32 output, and the same bits as the main library's
+    own kernels."""
+    if not P.peak_multicast_available():
+        pytest.skip("libpeak_gemm_mc.so is not present (multi-GPU runs leave it out)")
+    for idx, (M, N, K) in enumerate([(128, 1024, 512), (100, 1000, 264), (512, 512, 64), (300, 900, 1096)]):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32):
+            pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[1.0, 0.0][idx % 2], pad_a=pa, pad_b=pb,
+                   pad_c=[0, 8][idx % 2], case=idx)
+            want = None
+            for mode in (1, 112, 114, 121, 122, 124, 141, 142, 212, 214, 221, 222):
+                P.peak_set_tuning(P.PEAK_TUNE_SHARE, mode)
+                dc = R.DeviceCase(c)
+                dc.run(P.PEAK_VARIANT_AUTO)
+                assert ("umma_share_kernel" in P.peak_last_kernel()) == (mode != 1), P.peak_last_kernel()
+                got = dc.result()
+                got = got.view(np.uint32) if c.out_type == "f32" else got
+                if want is None:
+                    ref, _ = dc.oracle_full()
+                    want = oracle.round_to(R.OT[c.out_type], ref)
+                assert np.array_equal(got, want), f"{c} share={mode}"
+
+
+def test_shared_operand_clusters_bounded_wait(reset_tuning):
+    """The stalled-stage hook in the shared-operand kernel: one CTA never sends its parts of the last stage, so
+    its own and its peers' waits run out; every CTA still reaches the closing cluster barrier, the timeout is
+    reported once and the context computes correctly afterwards."""
+    if not P.peak_multicast_available():
+        pytest.skip("libpeak_gemm_mc.so is not present (multi-GPU runs leave it out)")
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 256, 512, 1024)
+    dc = R.DeviceCase(c)
+    P.peak_set_tuning(P.PEAK_TUNE_SHARE, 122)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 20)
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 1)
+    P.peak_gemm_variant(P.PEAK_VARIANT_AUTO, c.dtype, c.transA, c.transB, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb,
+                        0.0, dc.C, c.ldc)
+    assert "umma_share_kernel" in P.peak_last_kernel()
+    rc, detail = P.peak_check()
+    assert rc == P.PEAK_ERR_TIMEOUT and (detail & 0x80000000)
+    assert P.peak_check()[0] == P.PEAK_OK
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 0)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 0)
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "umma_share_kernel" in P.peak_last_kernel()
     R.check_full(dc)
 
 
