@@ -311,7 +311,10 @@ typedef enum peak_tuning_key {
                                    (default: only the rows that exist, which saves copy-engine requests) */
     PEAK_TUNE_CLUSTER_K = 17,   /* a single matrix on single-CTA tiles whose every tile is split 2 or 4 ways: 1 = partial tiles
                                    through the workspace and a reduction kernel (default: the slices run on the CTAs of
-                                   a cluster and are added through distributed shared memory, one launch) */
+                                   a cluster and are added through distributed shared memory, one launch; one-wave problems
+                                   of whole 128-wide tiles run the same one-tile-per-CTA kernel); 2 = as default, but
+                                   the slices always travel by bulk copies (default: plain remote stores for tiles of
+                                   at most 32 rows) */
     PEAK_TUNE_SHARE = 18,       /* single-GPU plug-in, 16-bit inputs: single-CTA tiles in clusters of CM x CN tiles that share
                                    their A / B tiles by multicast copies: 1 = never, 100 * w + 10 * CM + CN (w = 1: 128-wide
                                    tiles, 2: 256-wide) = that cluster shape whenever the plug-in is present */

@@ -12,18 +12,20 @@
 //               per k-block for barrier wait, fence, descriptors, four MMAs and commit: measured, the main loop
 //               of 512x4096x4096 went from 540 to 413 cycles per k-block, where the operand stream takes over.)
 //   exchange    (KC > 1) the tile's BN columns are divided into KC column slices, one per CTA.  When every CTA of
-//               the cluster has finished its main loop (cluster barrier 1: the stage ring is free everywhere),
-//               each epilogue thread copies, for every other CTA d, its row of slice d (both accumulators added)
-//               into a receive area in CTA d's ring (st.shared::cluster, swizzled like the staging buffers so
-//               that the 32 lanes of a warp hit different banks);
-//   reduction   (KC > 1) after cluster barrier 2 each CTA adds the KC partials of its own slice in slice order
+//               the cluster has finished its main loop (a cluster barrier: the stage ring is free everywhere), each
+//               epilogue warp stages its 32 rows of every other CTA's slice (both accumulators added) in its own
+//               ring, swizzled against bank conflicts, and sends them with one 4 KiB bulk copy per 32-column chunk
+//               into a receive area in that CTA's ring; the receiver's mbarrier counts the bytes.  Tiles of at most
+//               32 rows skip the staging: plain remote stores into the peers' idle staging buffers and one cluster
+//               barrier;
+//   reduction   (KC > 1) when all bytes are in, each CTA adds the KC partials of its own slice in slice order
 //               0..KC-1 (its own at its position in that order) and writes the sums back to tensor memory;
 //   epilogue    the ordinary tile epilogue (alpha/beta, bias, activation, residual, TMA or direct stores) over the
 //               slice -- or, for KC = 1, over the whole tile by two groups of four warps that read and add both
 //               accumulators.
 // The order of the additions is fixed by the launch, so results are run-to-run identical.  Every mbarrier wait
-// is bounded; the two cluster barriers are reached by every thread whether or not a wait gave up, so a CTA
-// whose wait ran out cannot leave its peers waiting.
+// is bounded; the cluster barriers (after the main loop and before exit) are reached by every thread whether or
+// not a wait gave up, so a CTA whose wait ran out cannot leave its peers waiting.
 #pragma once
 #include "umma_device.cuh"
 
@@ -34,7 +36,9 @@ template <int BN, int KC> struct ClusterKCfg {
     using C_ = Cfg<1, BN>;
     static constexpr int SW = BN / KC;            // columns each CTA finalises
     static constexpr int CHUNKS = SW / 32;        // 32-column chunks per slice
-    static constexpr int RECV_BYTES = KC * CHUNKS * BM * 128;  // [source CTA][chunk][row][128 bytes]
+    // receive area [peer 0..KC-2][chunk][row][128 bytes] and, behind it, a send area of the same shape, both in the ring
+    static constexpr int AREA_BYTES = (KC - 1) * CHUNKS * BM * 128;
+    static constexpr int RECV_BYTES = 2 * AREA_BYTES;
     // Two MMA issuers, each with an accumulator of its own, take the k-blocks in turn (128-wide tiles: both
     // accumulators fit 256 columns of tensor memory; 256-wide tiles keep one issuer).
     static constexpr bool DUAL = BN == 128;
@@ -71,6 +75,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const uint32_t full0 = ptx::smem_u32(bars);
     const uint32_t empty0 = full0 + 8 * STAGES;
     const uint32_t accfull = empty0 + 8 * STAGES;
+    const uint32_t recvbar = accfull + 8;  // the peers' partial sums of this CTA's slice have arrived
+    const uint32_t ackbar = accfull + 16;  // the peers have received what this CTA sent them (bulk copies)
     const uint32_t cbar0 = accfull + 32;
 
     constexpr int MN_ELEMS = IN8 ? 128 : 64;
@@ -79,6 +85,20 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int lane = threadIdx.x & 31;
     const uint32_t me = KC > 1 ? ptx::cluster_ctarank() : 0u;  // k-slice of this CTA, and the column slice it finalises
     const int tile = blockIdx.x / KC;
+    int64_t tm, tn;
+    tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
+    const int m0 = (int)tm * BM, n0 = (int)tn * BN;
+    const int kb0 = (int)me * p.kb_per_split;
+    const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);  // the host guarantees kb0 < kb1
+    // How the k-slices travel (KC > 1).  A tile with at most 32 rows: the one warp that owns them writes its few
+    // values straight into the peers' staging buffers (unused there: only one epilogue warp works), followed by
+    // one cluster barrier (measured at 16x4096x4096: 11.8 us, against 12.5 with a remote mbarrier arrival in place
+    // of the barrier and 12.9 with bulk copies).  Taller tiles: bulk copies into the peers' rings, which must be
+    // free first (cluster barrier after the main loop); the receiver's mbarrier counts the bytes and the senders
+    // are told when their staging may go away (256x4096x4096: 17.0 us with per-thread remote stores between two
+    // cluster barriers, 16.4 this way).
+    const int live_warps = min(4, (p.M - m0 + 31) / 32);
+    const bool direct = KC > 1 && live_warps == 1 && !p.bulk_exchange;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -86,6 +106,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::mbar_init(empty0 + 8 * s, 1);
         }
         ptx::mbar_init(accfull, K_::DUAL ? 2 : 1);
+        ptx::mbar_init(recvbar, 1);
+        ptx::mbar_init(ackbar, KC > 1 ? KC - 1 : 1);
         for (int b = 0; b < 8; ++b) ptx::mbar_init(cbar0 + 8 * b, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -102,18 +124,20 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    // this CTA's barriers exist: tell the peers (they wait for it only when the main loop is over)
+    if (KC > 1) ptx::cluster_arrive();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's shared and tensor memory and may overlap the previous kernel
     ptx::grid_dependency_wait();
     ptx::grid_launch_dependents();
 
-    int64_t tm, tn;
-    tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-    const int m0 = (int)tm * BM, n0 = (int)tn * BN;
-    const int kb0 = (int)me * p.kb_per_split;
-    const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);  // the host guarantees kb0 < kb1
     bool ok = true;
+    if (KC > 1 && !direct && threadIdx.x == 0) {
+        // what the peers will send: from each of them, for every 32-row block of the tile that exists, one 4 KiB
+        // piece per 32-column chunk of this CTA's slice
+        ptx::mbar_arrive_expect_tx(recvbar, (uint32_t)((KC - 1) * K_::CHUNKS * live_warps * 4096));
+    }
 
     if (warp == 0 || warp == K_::PRODUCER2) {
         // ------------------------------------------------------------------ producers
@@ -200,8 +224,10 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::tc_fence_after_sync();
     }
 
-    // cluster barrier 1: every CTA's main loop is over (or has given up), so every stage ring may be overwritten
-    if (KC > 1) ptx::cluster_sync();
+    if (KC > 1) {
+        ptx::cluster_wait();              // the peers' barriers exist (they arrived long ago)
+        if (!direct) ptx::cluster_sync(); // every CTA's main loop is over (or has given up): every ring may be overwritten
+    }
 
     const int q = warp & 3;                       // TMEM lane quadrant of an epilogue warp
     const int row0 = m0 + q * 32;                 // first row of this warp
@@ -223,31 +249,77 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::tmem_ld_wait();
         }
     };
-    if (live) {
+    bool exchange_ok = true;
+    if (live && KC > 1) {
         // ------------------------------------------------------------------ exchange
+        if (direct) {
+            // slot i of the receive area: 4 KiB pieces in the staging buffers the idle epilogue warps do not use
+            // (the one working warp, quadrant 0, owns bytes 16..24 KiB of the 32 KiB)
+#pragma unroll 1
+            for (int dd = 1; dd < KC; ++dd) {
+                const uint32_t d = (me + (uint32_t)dd) % KC;
+                const int ord_there = KC - 1 - dd;
+#pragma unroll 1
+                for (int c = 0; c < K_::CHUNKS; ++c) {
+                    uint32_t r[32];
+                    load_partial((int)d * SW + c * 32, r);
+                    if (m0 + trow < p.M) {
+                        const int slot = ord_there * K_::CHUNKS + c;
+                        const uint32_t local = epi_base + (uint32_t)((slot < 4 ? slot : slot + 2) * 4096 + lane * 128);
+                        const uint32_t remote = ptx::map_to_cta(local, d);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            ptx::st_cluster_v4(remote + (uint32_t)((j ^ (lane & 7)) * 16), r[4 * j], r[4 * j + 1], r[4 * j + 2],
+                                               r[4 * j + 3]);
+                    }
+                }
+            }
+        } else {
+        // Each warp stages its 32 rows of a peer's slice in this CTA's own ring (free since its accumulators are
+        // complete) and sends them with one bulk copy per 32-column chunk; the peer's barrier counts the bytes.
 #pragma unroll 1
         for (int dd = 1; dd < KC; ++dd) {
             const uint32_t d = (me + (uint32_t)dd) % KC;  // start with the neighbour: the CTAs write to different peers
+            const int ord_there = KC - 1 - dd;            // this CTA's place among d's peers: (me - d - 1) mod KC
 #pragma unroll 1
             for (int c = 0; c < K_::CHUNKS; ++c) {
                 uint32_t r[32];
                 load_partial((int)d * SW + c * 32, r);
-                if (m0 + trow < p.M) {
-                    const uint32_t local = stage_base + (uint32_t)(((int)me * K_::CHUNKS + c) * BM + trow) * 128u;
-                    const uint32_t remote = ptx::map_to_cta(local, d);
+                const uint32_t row = stage_base + (uint32_t)K_::AREA_BYTES +
+                                     (uint32_t)((((dd - 1) * K_::CHUNKS + c) * BM + trow) * 128);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        ptx::st_cluster_v4(remote + (uint32_t)((j ^ (trow & 7)) * 16), r[4 * j], r[4 * j + 1], r[4 * j + 2],
-                                           r[4 * j + 3]);
+                for (int j = 0; j < 8; ++j)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (uint32_t)((j ^ (trow & 7)) * 16)),
+                                 "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3])
+                                 : "memory");
+            }
+            ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the bulk copy
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t bar_there = ptx::map_to_cta(recvbar, d);
+#pragma unroll 1
+                for (int c = 0; c < K_::CHUNKS; ++c) {
+                    const uint32_t src = stage_base + (uint32_t)K_::AREA_BYTES +
+                                         (uint32_t)((((dd - 1) * K_::CHUNKS + c) * BM + q * 32) * 128);
+                    const uint32_t dst = stage_base + (uint32_t)(((ord_there * K_::CHUNKS + c) * BM + q * 32) * 128);
+                    ptx::bulk_copy_to_cluster(ptx::map_to_cta(dst, d), src, 4096u, bar_there);
                 }
             }
         }
+        }
+        // the peers' partial sums of this CTA's slice: all bytes in (bounded wait)
+        const bool arrived = direct || ptx::mbar_wait<true>(recvbar, 0u, abort_flag, p.wait_cycles);
+        if (!__all_sync(0xffffffffu, arrived)) {
+            if (lane == 0) report_timeout(p, abort_flag, 7, 0);
+            exchange_ok = false;
+        } else if (!direct && q == 0 && lane == 0) {
+            // everything the peers sent has been written here, so their send areas are no longer read: tell them
+            for (int dd = 1; dd < KC; ++dd) ptx::mbar_arrive_cluster(ptx::map_to_cta(ackbar, (me + (uint32_t)dd) % KC));
+        }
     }
 
-    // cluster barrier 2: all partials have arrived (release / acquire at cluster scope)
-    if (KC > 1) ptx::cluster_sync();
-
-    if (live) {
+    if (direct) ptx::cluster_sync();  // the few values of a short tile have been stored everywhere (release / acquire)
+    if (live && exchange_ok) {
         // ------------------------------------------------------------------ reduction of this CTA's slice
 #pragma unroll 1
         for (int c = 0; c < K_::CHUNKS && KC > 1; ++c) {
@@ -262,7 +334,10 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(own[i]);
                 } else {
-                    const uint32_t rowaddr = stage_base + (uint32_t)(((int)src * K_::CHUNKS + c) * BM + trow) * 128u;
+                    const int ord = ((int)src - (int)me - 1 + KC) % KC;  // src's place among this CTA's peers
+                    const int slot = ord * K_::CHUNKS + c;
+                    const uint32_t rowaddr = direct ? epi_base + (uint32_t)((slot < 4 ? slot : slot + 2) * 4096 + lane * 128)
+                                                    : stage_base + (uint32_t)((ord * K_::CHUNKS + c) * BM + trow) * 128u;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         uint32_t w0, w1, w2, w3;
@@ -322,6 +397,11 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
 
     // ---------------------------------------------------------------------- teardown
+    if (KC > 1 && !direct && warp >= 2 && warp < K_::PRODUCER2 && (warp & 3) == 0 && lane == 0) {
+        // this CTA's send area must outlive the bulk copies that read it: every peer has acknowledged receipt
+        if (ok && exchange_ok && !ptx::mbar_wait<true>(ackbar, 0u, abort_flag, p.wait_cycles)) report_timeout(p, abort_flag, 8, 0);
+    }
+    __syncwarp();
     if (*abort_flag != 0) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);

@@ -110,6 +110,7 @@ struct UmmaParams {
     // stored.  a_boxes: MN-major A, how many 64-row (8-bit: 128-row) boxes are fetched; stage_tx: bytes per stage.
     int a_boxes;
     uint32_t stage_tx;
+    int bulk_exchange;     // one-tile-per-CTA kernel: 1 = k-slices always travel by bulk copies (also for tiles of <= 32 rows)
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
     uint32_t *status;

@@ -181,6 +181,7 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.tiles_per_batch = p.tiles_m * p.tiles_n;
     p.stride_c = g.strideC;
     const int tiles = p.tiles_per_batch * (int)nb;
+    p.bulk_exchange = 0;
     p.full_tiles = plan.full_tiles;
     p.tail_splits = plan.tail_splits;
     p.kb_per_split = (p.num_kb + plan.tail_splits - 1) / plan.tail_splits;
@@ -433,6 +434,7 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
     p.a_mn = a_mn; p.b_mn = b_mn;
     p.a_boxes = a_boxes;
     p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
+    p.bulk_exchange = tuning(PEAK_TUNE_CLUSTER_K) == 2 ? 1 : 0;
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);

@@ -107,6 +107,7 @@ template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(
     if (p.tma_store && !make_map(&tmC, eout, r->C, r->N, r->M, r->ldc, 128 / ob, 32)) return PEAK_ERR_CUDA;
     p.k_alternate = r->k_order == 2 ? 1 : 0;
     p.a_boxes = BM / 64; p.stage_tx = (uint32_t)C_::STAGE_BYTES;  // (pairs take their own byte count)
+    p.bulk_exchange = 0;
     p.status = r->status;
     p.wait_cycles = r->wait_ms > 0 ? (long long)r->wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
     p.inject_stall = r->inject_stall == 1 ? 1 : 0;
