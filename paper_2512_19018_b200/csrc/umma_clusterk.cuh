@@ -139,6 +139,21 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::mbar_arrive_expect_tx(recvbar, (uint32_t)((KC - 1) * K_::CHUNKS * live_warps * 4096));
     }
 
+    // epilogue parameters of this warp (meaningful for warps 2 .. PRODUCER2 - 1)
+    constexpr int CC = 128 / (int)sizeof(TOut);        // columns per staged chunk
+    constexpr int GW = SW / K_::GROUPS;                // columns this warp's group drains
+    constexpr int W = GW < CC ? CC : GW;               // a slice narrower than a chunk takes the direct stores
+    const int q = warp & 3;                            // TMEM lane quadrant of an epilogue warp
+    const int row0 = m0 + q * 32;                      // first row of this warp
+    const int grp = (warp - 2) >> 2;
+    const bool tma = p.tma_store != 0 && GW >= CC;
+    const int c_first = n0 + (int)me * SW + grp * GW;
+    const int c_limit = min(p.N, c_first + GW);
+    // staging: two buffers per warp with one group, one per warp with two
+    const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (K_::GROUPS == 1 ? 2u : 1u) * EPI_BUF_BYTES;
+    CFetch cf{K_::GROUPS == 1 ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
+              tma && p.c_prefetch != 0, K_::GROUPS == 2};
+
     if (warp == 0 || warp == K_::PRODUCER2) {
         // ------------------------------------------------------------------ producers
         // Two warps take the k-blocks in turn, and inside a warp every copy of a stage is issued by a lane of its
@@ -217,7 +232,13 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue warps (2..5): wait for the accumulator
+        // ------------------------------------------------------------------ epilogue warps: old C of the first chunk(s)
+        // is requested while the main loop runs (beta != 0 with TMA stores); then wait for the accumulator
+        if (cf.on && row0 < p.M && c_first < p.N && lane == 0) {
+            cfetch_issue<TOut, false>(cf, my_stage, 0, &tmC, c_first, row0, 0);
+            if (!cf.single && c_first + CC < c_limit) cfetch_issue<TOut, false>(cf, my_stage, 1, &tmC, c_first, row0, 0);
+        }
+        __syncwarp();
         const bool got = ptx::mbar_wait<false>(accfull, 0u, abort_flag, p.wait_cycles);
         ok = __all_sync(0xffffffffu, got);
         if (!ok && lane == 0) report_timeout(p, abort_flag, 5, 0);
@@ -229,8 +250,6 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (!direct) ptx::cluster_sync(); // every CTA's main loop is over (or has given up): every ring may be overwritten
     }
 
-    const int q = warp & 3;                       // TMEM lane quadrant of an epilogue warp
-    const int row0 = m0 + q * 32;                 // first row of this warp
     const bool live = warp >= 2 && warp < K_::PRODUCER2 && ok && row0 < p.M;
     const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
     const int trow = q * 32 + lane;               // row inside the tile
@@ -364,23 +383,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         ptx::tmem_st_wait();
         // ------------------------------------------------------------------ tile epilogue over the slice
-        constexpr int CC = 128 / (int)sizeof(TOut);        // columns per staged chunk
-        constexpr int GW = SW / K_::GROUPS;                // columns this warp's group drains
-        constexpr int W = GW < CC ? CC : GW;               // a slice narrower than a chunk takes the direct stores
-        const int grp = (warp - 2) >> 2;
-        const bool tma = p.tma_store != 0 && GW >= CC;
-        const int c_first = n0 + (int)me * SW + grp * GW;
-        const int c_limit = min(p.N, c_first + GW);
-        // staging: two buffers per warp with one group, one per warp with two
-        const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (K_::GROUPS == 1 ? 2u : 1u) * EPI_BUF_BYTES;
-        CFetch cf{K_::GROUPS == 1 ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
-                  tma && p.c_prefetch != 0, K_::GROUPS == 2};
         if (c_first < p.N) {
-            if (cf.on && lane == 0) {
-                cfetch_issue<TOut, false>(cf, my_stage, 0, &tmC, c_first, row0, 0);
-                if (!cf.single && c_first + CC < c_limit) cfetch_issue<TOut, false>(cf, my_stage, 1, &tmC, c_first, row0, 0);
-            }
-            __syncwarp();
             const uint32_t t_first = t_row + me * SW + (uint32_t)(grp * GW);
             // a whole tile (KC = 1) is read from both issuers' accumulators; a slice's sums were written back above
             const uint32_t t_second = (KC == 1 && two_acc) ? t_first + BN : 0u;
