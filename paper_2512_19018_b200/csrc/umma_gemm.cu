@@ -469,6 +469,12 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
     cfg.attrs = attr;
     cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+    if (e == cudaErrorInvalidClusterSize || e == cudaErrorLaunchOutOfResources || e == cudaErrorInvalidConfiguration) {
+        // a device (or partition) that cannot place this cluster shape: nothing was launched, the caller takes the
+        // workspace path
+        (void)cudaGetLastError();
+        return PEAK_ERR_UNSUPPORTED;
+    }
     count_launch();
     note_kernel("umma_clusterk_kernel<%d, %s, %d, %d> grid=%d clusters=%d", BN,
                 sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"), KC, (int)IN8,
@@ -720,7 +726,10 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         }
     }
     if (wide) plan = Plan{512, (int)tiles_of(g, 2, 512), 1};
-    if (clusterk_applies(g, cta_group, plan)) return run_clusterk(g, plan);
+    if (clusterk_applies(g, cta_group, plan)) {
+        const int rc = run_clusterk(g, plan);
+        if (rc != PEAK_ERR_UNSUPPORTED) return rc;  // otherwise: the persistent kernel, with a workspace for k-slices
+    }
     if (cta_group == 2) {
         if (plan.bn == 512) return run_umma<2, 512>(g, plan, units);
         return plan.bn == 256 ? run_umma<2, 256>(g, plan, units) : run_umma<2, 128>(g, plan, units);
