@@ -634,14 +634,24 @@ def test_old_c_by_tma_with_a_group_that_has_no_columns(dtype, knobs, reset_tunin
 
 def test_cuda_graph_with_k_split_and_several_calls():
     """A captured sequence: a k-split problem (pooled workspace allocated and freed inside the capture, reduce
-    kernel launched as a programmatic dependent), a beta != 0 problem and a wide-tile problem, replayed twice."""
+    kernel launched as a programmatic dependent), a beta != 0 problem, a wide-tile problem and the three forms of
+    the one-tile-per-CTA kernel (cluster launches), replayed twice."""
     cases = [mk(W.PEAK_BF16_BF16, 1, 0, 16, 1024, 2048, alpha=0.5, beta=2.0, case=1),        # split-K
              mk(W.PEAK_F16_F32, 0, 1, 520, 776, 264, alpha=1.0, beta=1.0, case=2),
-             mk(W.PEAK_BF16_BF16, 0, 0, 512, 1024, 4096, case=3)]
+             mk(W.PEAK_BF16_BF16, 0, 0, 512, 1024, 4096, case=3),
+             # the one-tile-per-CTA kernel: four k-slices on a cluster, two k-slices, whole tiles
+             mk(W.PEAK_BF16_BF16, 1, 0, 16, 4096, 4096, alpha=0.5, beta=2.0, case=4),
+             mk(W.PEAK_BF16_F32, 0, 1, 128, 4096, 1024, alpha=1.0, beta=1.0, case=5),
+             mk(W.PEAK_F16_F16, 0, 0, 256, 2560, 512, alpha=2.0, beta=0.0, case=6)]
     dcs = [R.DeviceCase(c) for c in cases]
     stream = torch.cuda.Stream()
+    names = []
     for dc in dcs:
         dc.run(stream=None)                                    # first-use set-up outside the capture
+        names.append(P.peak_last_kernel())
+    assert "umma_clusterk_kernel<128, __nv_bfloat16, 4, 0>" in names[3], names[3]
+    assert "umma_clusterk_kernel<128, float, 2, 0>" in names[4], names[4]
+    assert "umma_clusterk_kernel<128, __half, 1, 0>" in names[5], names[5]
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(stream):
