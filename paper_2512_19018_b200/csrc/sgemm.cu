@@ -355,7 +355,12 @@ int launch_sgemm(const GemmArgs &g) {
     const bool b_gets_transposed = g.transB && tuning(PEAK_TUNE_SGEMM_TRANSPOSE) != 1 &&
                                    (tuning(PEAK_TUNE_SGEMM_TRANSPOSE) == 2 || (g.M >= 2048 && g.N >= 512)) &&
                                    g.N * g.K * 4 <= (512ll << 20);
-    const bool want_tma = copy == 3 || !aligned || (copy == 0 && (!g.transB || b_gets_transposed));
+    // (... or the grid is too small for whole tiles: the TMA-fed path cuts such problems along k, after transposing B)
+    const int64_t tiles = ((g.M + 127) / 128) * ((g.N + 127) / 128);
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const bool small_grid = tiles < 2 * (int64_t)sms && tuning(PEAK_TUNE_SGEMM_TRANSPOSE) != 1;
+    const bool want_tma = copy == 3 || !aligned || (copy == 0 && (!g.transB || b_gets_transposed || small_grid));
     if (want_tma && sgemm_tma_supports(g)) return launch_sgemm_tma(g);
     if (!aligned) return PEAK_ERR_UNSUPPORTED;
     const bool both_k_contiguous = !g.transA && g.transB;

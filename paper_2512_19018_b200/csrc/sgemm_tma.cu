@@ -14,6 +14,8 @@
 //     to two k-blocks instead of waiting for the slowest warp at every step.  Every wait is bounded.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "umma_host.cuh"
@@ -40,6 +42,11 @@ struct SgemmParams {
     const float *R;  // residual added after the activation, or nullptr
     int64_t ldr;
     int vec_ok;  // C (and R) base and pitch allow 16-byte accesses
+    // k-slices (gridDim.y > 1): block (x, y) multiplies k-blocks [y * kb_per_split, ...) of tile x and stores the
+    // raw sums to ws[y][M][ldw]; sgemm_splitk_reduce_kernel adds the slices in order and applies the epilogue
+    int kb_per_split;
+    float *ws;
+    int64_t ldw;
     long long wait_cycles;
     uint32_t *status;
 };
@@ -96,12 +103,15 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::prefetch_tensormap(&tmB);
     }
     __syncthreads();
+    ptx::grid_launch_dependents();  // a reduction kernel that follows may be scheduled; it waits for this grid to end
 
-    auto issue = [&](int kb) {  // one thread: both tiles of k-block kb into stage kb % STAGES
+    const bool sliced = gridDim.y > 1;
+    const int koff = sliced ? (int)blockIdx.y * p.kb_per_split : 0;  // first k-block of this block's slice
+    auto issue = [&](int kb) {  // one thread: both tiles of k-block kb (of the slice) into stage kb % STAGES
         const uint32_t s = (uint32_t)kb % ST_STAGES;
         const uint32_t bar = full0 + 8 * s;
         const uint32_t a_dst = stage0 + s * ST_STAGE_BYTES, b_dst = a_dst + ST_TILE_BYTES;
-        const int k0 = kb * ST_BK;
+        const int k0 = (koff + kb) * ST_BK;
         ptx::mbar_arrive_expect_tx(bar, (uint32_t)ST_STAGE_BYTES);
         if (A_KC) ptx::tma_load_2d(a_dst, &tmA, k0, m0, bar);
         else ptx::tma_load_2d(a_dst, &tmA, m0, k0, bar);
@@ -109,7 +119,7 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         else ptx::tma_load_2d(b_dst, &tmB, n0, k0, bar);
     };
 
-    const int nkb = p.nkb;
+    const int nkb = sliced ? min(p.kb_per_split, p.nkb - koff) : p.nkb;
     if (tid == 0)
         for (int kb = 0; kb < ST_AHEAD && kb < nkb; ++kb) issue(kb);
 
@@ -327,28 +337,35 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 
     // ---- epilogue: alpha / beta (+ bias, activation) in fp32, predicated at the edges -------------------------
-    const float alpha = p.alpha, beta = p.beta;
+    // a k-slice stores its raw sums to the workspace: alpha = 1, beta = 0, nothing fused
+    const float alpha = sliced ? 1.0f : p.alpha, beta = sliced ? 0.0f : p.beta;
+    float *const c_base = sliced ? p.ws + (int64_t)blockIdx.y * p.M * p.ldw : p.C;
+    const int64_t c_ld = sliced ? p.ldw : p.ldc;
+    const float *const bias = sliced ? nullptr : bias;
+    const int act = sliced ? 0 : act;
+    const float *const res = sliced ? nullptr : p.R;
+    const bool vec_ok = sliced ? true : p.vec_ok != 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int m = m0 + ty * 4 + (i & 3) + 64 * (i >> 2);
         if (m >= p.M) continue;
-        float *crow = p.C + (int64_t)m * p.ldc;
+        float *crow = c_base + (int64_t)m * c_ld;
         if (!B_KC) {
 #pragma unroll
             for (int h = 0; h < NT / 4; ++h) {
                 const int n = n0 + tx * 4 + TXN * 4 * h;
                 if (n >= p.N) continue;
-                if (p.vec_ok && n + 4 <= p.N) {
+                if (vec_ok && n + 4 <= p.N) {
                     float4 *dst = reinterpret_cast<float4 *>(crow + n);
                     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (beta != 0.0f) o = *dst;
                     float4 r;
-                    r.x = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x), p.bias, n + 0, p.act);
-                    r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), p.bias, n + 1, p.act);
-                    r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), p.bias, n + 2, p.act);
-                    r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), p.bias, n + 3, p.act);
-                    if (p.R) {
-                        const float4 q = *reinterpret_cast<const float4 *>(p.R + (int64_t)m * p.ldr + n);
+                    r.x = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 0], beta, o.x), bias, n + 0, act);
+                    r.y = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 1], beta, o.y), bias, n + 1, act);
+                    r.z = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 2], beta, o.z), bias, n + 2, act);
+                    r.w = finish_f32(epilogue_f32(alpha, acc[i][4 * h + 3], beta, o.w), bias, n + 3, act);
+                    if (res) {
+                        const float4 q = *reinterpret_cast<const float4 *>(res + (int64_t)m * p.ldr + n);
                         r.x += q.x; r.y += q.y; r.z += q.z; r.w += q.w;
                     }
                     *dst = r;
@@ -357,8 +374,8 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     for (int q = 0; q < 4; ++q) {
                         if (n + q < p.N) {
                             const float o = (beta != 0.0f) ? crow[n + q] : 0.0f;
-                            crow[n + q] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][4 * h + q], beta, o), p.bias, n + q, p.act),
-                                                       p.R, (int64_t)m * p.ldr + n + q);
+                            crow[n + q] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][4 * h + q], beta, o), bias, n + q, act),
+                                                       res, (int64_t)m * p.ldr + n + q);
                         }
                     }
                 }
@@ -369,8 +386,51 @@ sgemm_tma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n = n0 + tx + 16 * j;
                 if (n < p.N) {
                     const float o = (beta != 0.0f) ? crow[n] : 0.0f;
-                    crow[n] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][j], beta, o), p.bias, n, p.act), p.R,
+                    crow[n] = add_residual(finish_f32(epilogue_f32(alpha, acc[i][j], beta, o), bias, n, act), res,
                                            (int64_t)m * p.ldr + n);
+                }
+            }
+        }
+    }
+}
+
+// Adds the k-slices of a sliced launch in slice order and applies the epilogue: C = alpha * (ws[0] + ws[1] + ...) +
+// beta * C (+ bias, activation, residual), four columns per thread.
+__global__ void __launch_bounds__(256)
+sgemm_splitk_reduce_kernel(const float *__restrict__ ws, int splits, int M, int N, int64_t ldw, float alpha, float beta,
+                           float *__restrict__ C, int64_t ldc, const float *__restrict__ bias, int act,
+                           const float *__restrict__ R, int64_t ldr, int vec_ok) {
+    const int n4 = (N + 3) / 4;
+    const int64_t total = (int64_t)M * n4;
+    const int64_t slice = (int64_t)M * ldw;
+    // launched as a programmatic dependent of the slice kernel: the slices may be read once that kernel has completed
+    ptx::grid_dependency_wait();
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int m = (int)(e / n4), n = (int)(e - (int64_t)m * n4) * 4;
+        const float *src = ws + (int64_t)m * ldw + n;
+        float4 a = *reinterpret_cast<const float4 *>(src);
+        for (int sl = 1; sl < splits; ++sl) {
+            const float4 v = *reinterpret_cast<const float4 *>(src + sl * slice);
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        const float av[4] = {a.x, a.y, a.z, a.w};
+        float *crow = C + (int64_t)m * ldc;
+        if (vec_ok && n + 4 <= N) {
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (beta != 0.0f) o = *reinterpret_cast<const float4 *>(crow + n);
+            const float ov[4] = {o.x, o.y, o.z, o.w};
+            float r[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                r[q] = add_residual(finish_f32(epilogue_f32(alpha, av[q], beta, ov[q]), bias, n + q, act), R, (int64_t)m * ldr + n + q);
+            *reinterpret_cast<float4 *>(crow + n) = make_float4(r[0], r[1], r[2], r[3]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (n + q < N) {
+                    const float o = (beta != 0.0f) ? crow[n + q] : 0.0f;
+                    crow[n + q] = add_residual(finish_f32(epilogue_f32(alpha, av[q], beta, o), bias, n + q, act), R,
+                                               (int64_t)m * ldr + n + q);
                 }
             }
         }
@@ -443,10 +503,56 @@ template <bool A_KC, bool B_KC, int KG, bool WIDE = false> int run_sgemm_tma(con
     p.status = device_status_word();
     if (!p.status) return PEAK_ERR_CUDA;
     const unsigned grid = (unsigned)(p.tiles_m * p.tiles_n);
-    kernel<<<grid, WIDE ? 128 : ST_THREADS, ST_SMEM_BYTES, g.stream>>>(tmA, tmB, p);
+    // k-slices for small grids.  The kernel needs two blocks per SM to keep the FMA pipe fed (four warps of a lone
+    // block reach about 40 % of it), so a problem with fewer tiles than that is cut along k until it has them, down
+    // to four k-blocks per slice and never beyond one full wave of two blocks per SM (measured, us, NN: 256^3 47 ->
+    // 15.6, 512^3 69 -> 18.4, 1024^3 113 -> 55.6, 1536^3 159 -> 142, 128x4096x4096 381 -> 92.6; cuBLAS 8.2 / 13.2 /
+    // 45.1 / 121 / 104.7).  PEAK_TUNE_SPLIT_K forces the number of slices (1 = none).
+    int splits = 1;
+    {
+        const int want_blocks = 2 * umma::sm_count();
+        const int forced = tuning(PEAK_TUNE_SPLIT_K);
+        if (forced > 0) splits = forced;
+        else if ((int)grid < want_blocks) splits = std::max(1, want_blocks / (int)grid);  // one full wave of two blocks per SM
+        splits = std::min(splits, std::max(1, p.nkb / 4));
+        splits = std::min(splits, 64);
+        while (splits > 1 && (size_t)splits * (size_t)g.M * (size_t)((g.N + 3) / 4 * 4) * 4 > (256ull << 20)) --splits;
+        p.kb_per_split = (p.nkb + splits - 1) / splits;
+        splits = (p.nkb + p.kb_per_split - 1) / p.kb_per_split;  // no empty slice
+    }
+    p.ws = nullptr; p.ldw = (g.N + 3) / 4 * 4;
+    if (splits > 1) {
+        cudaMemPool_t pool = scratch_pool();
+        if (!pool) return PEAK_ERR_CUDA;
+        cudaError_t me = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&p.ws), (size_t)splits * g.M * p.ldw * sizeof(float),
+                                                 pool, g.stream);
+        if (me != cudaSuccess) { set_cuda_error(me); return PEAK_ERR_NO_MEMORY; }
+    }
+    kernel<<<dim3(grid, (unsigned)splits), WIDE ? 128 : ST_THREADS, ST_SMEM_BYTES, g.stream>>>(tmA, tmB, p);
     count_launch();
-    note_kernel("sgemm_tma_kernel<%d, %d, %d, %d> grid=%u", (int)A_KC, (int)B_KC, KG, (int)WIDE, grid);
+    note_kernel("sgemm_tma_kernel<%d, %d, %d, %d> grid=%u slices=%d", (int)A_KC, (int)B_KC, KG, (int)WIDE, grid, splits);
     cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && splits > 1) {
+        const int64_t work = (int64_t)g.M * ((g.N + 3) / 4);
+        const unsigned rgrid = (unsigned)std::min<int64_t>((work + 255) / 256, 4 * (int64_t)umma::sm_count());
+        cudaLaunchConfig_t rcfg = {};
+        rcfg.gridDim = dim3(rgrid);
+        rcfg.blockDim = dim3(256);
+        rcfg.stream = g.stream;
+        cudaLaunchAttribute rattr[1];
+        rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        rattr[0].val.programmaticStreamSerializationAllowed = 1;
+        rcfg.attrs = rattr;
+        rcfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 0 : 1;
+        const float *ws_c = p.ws;
+        e = cudaLaunchKernelEx(&rcfg, sgemm_splitk_reduce_kernel, ws_c, splits, p.M, p.N, p.ldw, g.alpha, g.beta, (float *)g.C,
+                               g.ldc, g.bias, g.act, (const float *)g.R, g.ldr, p.vec_ok);
+        count_launch();
+    }
+    if (p.ws) {
+        const cudaError_t fe = cudaFreeAsync(p.ws, g.stream);
+        if (e == cudaSuccess) e = fe;
+    }
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
@@ -512,7 +618,10 @@ int launch_sgemm_tma(const GemmArgs &g) {
         const int64_t limit = 512ll << 20;                   // bytes of one transposed copy
         const bool fits_a = g.M * g.K * 4 <= limit && g.M <= 65535ll * 32, fits_b = g.N * g.K * 4 <= limit && g.N <= 65535ll * 32;
         const bool tr_a = a_kc && fits_a && (mode == 2 || (mode == 0 && g.N >= 2048 && g.M >= 512));
-        const bool tr_b = b_kc && fits_b && (mode == 2 || (mode == 0 && g.M >= 2048 && g.N >= 512));
+        // (a B with k contiguous is also transposed first when the grid is small: the problem is then cut along k by
+        // the dense kernel, which beats the k-contiguous kernel's 60 % of the FMA rate by more than the extra pass costs)
+        const bool small_grid = ((g.M + ST_BM - 1) / ST_BM) * ((g.N + ST_BN - 1) / ST_BN) < 2 * (int64_t)umma::sm_count();
+        const bool tr_b = b_kc && fits_b && (mode == 2 || (mode == 0 && ((g.M >= 2048 && g.N >= 512) || small_grid)));
         if (mode != 1 && (tr_a || tr_b)) return launch_with_transposes(g, tr_a, tr_b);
     }
     // k per load of a k-contiguous operand, measured at 4096^3 / 8192^3 NN: two (58.8 / 59.3 TFLOP/s) beats four

@@ -1020,6 +1020,52 @@ def test_sgemm_transposing_prepass_and_wide_register_tile(ta, tb, reset_tuning):
     check_fused(dc, bias, P.PEAK_ACT_GELU, f"sgemm transposed {c.layout}", res)
 
 
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_sgemm_k_slices_exact_and_selected(ta, tb, reset_tuning):
+    """SGEMM problems with fewer tiles than two blocks per SM are cut along k: every block stores the raw sums of
+    its slice, a second kernel (a programmatic dependent) adds the slices in order and applies alpha / beta, bias,
+    activation and residual.  Exact on integers in every layout for ragged shapes, forced slice counts (the last
+    slice shorter), padded pitches; chosen by the dispatcher for small grids and not for large ones; bitwise
+    repeatable on reals."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(43)
+    for idx, (M, N, K) in enumerate([(256, 256, 256), (129, 257, 1000), (1, 300, 530), (512, 384, 528), (100, 70, 4100)]):
+        pa, pb = (-(M if ta else K)) % 4 + 4 * (idx % 2), (-(K if tb else N)) % 4
+        ci = mk(W.PEAK_F32_F32, ta, tb, M, N, K, dist="smallint", alpha=2.0, beta=-1.0, pad_a=pa, pad_b=pb, pad_c=idx % 3,
+                case=idx)
+        outs = []
+        for split in (0, 1, 2, 3, 7):
+            P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
+            dc = R.DeviceCase(ci)
+            dc.run(P.PEAK_VARIANT_SGEMM)
+            name = P.peak_last_kernel()
+            slices = int(name.split("slices=")[1])
+            if split == 0:
+                assert slices > 1, name                      # a handful of tiles: the dispatcher cuts along k
+            elif split == 1:
+                assert slices == 1, name
+            else:
+                assert 1 < slices <= split, name
+            ref, _ = dc.oracle_full()
+            assert np.array_equal(dc.result().view(np.uint32), oracle.round_to(oracle.F32, ref)), f"{ci} split {split}"
+            outs.append(dc.result().copy())
+        assert all(np.array_equal(outs[0], o) for o in outs[1:])
+    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 0)
+    c = W.GemmCase("sg_slices_fused", W.PEAK_F32_F32, bool(ta), bool(tb), 520, 392, 1064, 0.5, 2.0, "uniform")
+    bias = rng.standard_normal(c.N).astype(np.float32)
+    res = make_residual(c, rng, 4)
+    dc = run_fused(c, P.PEAK_VARIANT_AUTO, bias, P.PEAK_ACT_GELU, res)
+    assert "slices=" in P.peak_last_kernel() and not P.peak_last_kernel().endswith("slices=1"), P.peak_last_kernel()
+    check_fused(dc, bias, P.PEAK_ACT_GELU, f"sgemm k-slices fused {c.layout}", res)
+    first = dc.result().copy()
+    dc2 = run_fused(c, P.PEAK_VARIANT_AUTO, bias, P.PEAK_ACT_GELU, res)
+    assert np.array_equal(first, dc2.result())
+    big = mk(W.PEAK_F32_F32, ta, tb, 2304, 2304, 64, dist="smallint")     # 324 tiles: whole tiles
+    dc = R.DeviceCase(big)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert P.peak_last_kernel().endswith("slices=1"), P.peak_last_kernel()
+
+
 def test_sgemm_tma_paths_in_a_cuda_graph_and_on_two_streams(reset_tuning):
     """The TMA-fed SGEMM inside a captured graph -- a ragged problem, and one whose k-contiguous operands are first
     transposed into pool memory (allocated and freed inside the capture) -- replayed twice; then the same two
