@@ -44,5 +44,8 @@ struct peak_mc_request {
 // Returns a peak_status_t.  PEAK_ERR_UNSUPPORTED: the caller should run its own kernel instead.
 typedef int (*peak_mc_gemm_fn)(peak_mc_request *req);
 int peak_mc_gemm(peak_mc_request *req);
+// Four-CTA clusters of the pair kernel (tile_n 256 or 512) the current device holds at once; 0 = unknown.
+typedef int (*peak_mc_max_clusters_fn)(int tile_n);
+int peak_mc_max_clusters(int tile_n);
 
 }  // extern "C"

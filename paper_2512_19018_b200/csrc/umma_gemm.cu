@@ -23,6 +23,7 @@ namespace {
 using namespace umma;
 
 // ---- optional single-GPU plug-in (cluster-multicast B loads), loaded from beside this library ------------
+peak_mc_max_clusters_fn g_mc_max_clusters = nullptr;
 peak_mc_gemm_fn mc_entry() {
     static peak_mc_gemm_fn fn = nullptr;
     static std::once_flag once;
@@ -35,8 +36,12 @@ peak_mc_gemm_fn mc_entry() {
         void *h = dlopen(path.c_str(), RTLD_NOW | RTLD_LOCAL);
         if (!h) return;
         fn = reinterpret_cast<peak_mc_gemm_fn>(dlsym(h, "peak_mc_gemm"));
+        g_mc_max_clusters = reinterpret_cast<peak_mc_max_clusters_fn>(dlsym(h, "peak_mc_max_clusters"));
     });
     return fn;
+}
+int mc_max_clusters(int tile_n) {
+    return (mc_entry() && g_mc_max_clusters) ? g_mc_max_clusters(tile_n) : 0;
 }
 
 constexpr double kL2BytesPerClk = 40.0;        // L2 -> shared-memory bytes per cycle one SM sustains (measured ~39)
@@ -688,7 +693,8 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         const int64_t min_kb = !light_tail ? 128 : (in8 ? 96 : 48);
         auto fill = [&](int64_t tiles) { return (double)tiles / (double)(((tiles + units - 1) / units) * units); };
         const int64_t t512 = tiles_of(g, 2, 512), t256 = tiles_of(g, 2, 256);
-        wide = num_kb >= min_kb && t512 >= units && fill(t512) >= fill(t256) - 0.02;
+        // (3072^3: 72 wide tiles on 74 pairs, one wave: 40.0 us against 41.3 for two waves of 256-wide tiles)
+        wide = num_kb >= min_kb && t512 * 10 >= (int64_t)units * 9 && fill(t512) >= fill(t256) - 0.02;
     }
     // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
     // Measured (sustained, random inputs, interleaved): fp16 4096^3 -> fp32 1162 against 1132 (512-wide) and
@@ -706,7 +712,13 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         const int mc_tile_n = ((whole512 || wide_first) && !in8) ? 512 : 256;
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + mc_tile_n - 1) / mc_tile_n);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;
-        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11)) {
+        // A cluster works on two pair tiles at once, but fewer clusters fit the device than half its pairs (33 of 37
+        // here): the plug-in only runs when its super-tiles need no more waves than the pair tiles would on all pairs
+        // (3072^3: 72 super-tiles = 3 waves against 2 -- 56.7 us through the plug-in, 40.0 without).
+        const int maxc = mc_max_clusters(mc_tile_n);
+        const int64_t pair_tiles = tiles_of(g, 2, mc_tile_n);
+        const bool waves_ok = maxc <= 0 || (super_tiles + maxc - 1) / maxc <= (pair_tiles + units - 1) / units;
+        if (mc_mode == 2 || (super_tiles >= 32 && flops <= 2e11 && waves_ok)) {
             peak_mc_request r{g.dtype, g.transA, g.transB, g.M, g.N, g.K, g.alpha, g.beta, g.A, g.B, g.C, g.lda, g.ldb,
                               g.ldc, g.stream, device_status_word(), tuning(PEAK_TUNE_RASTER_GROUP),
                               tuning(PEAK_TUNE_EPILOGUE), tuning(PEAK_TUNE_WAIT_MS), tuning(PEAK_TUNE_DEPENDENT_LAUNCH),

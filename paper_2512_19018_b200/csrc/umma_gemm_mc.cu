@@ -301,4 +301,42 @@ extern "C" int peak_mc_gemm(peak_mc_request *r) {
     return PEAK_ERR_INVALID_VALUE;
 }
 
-extern "C" int peak_mc_max_clusters(void) { return 0; }
+// How many four-CTA clusters of the pair kernel the current device holds at once (tile_n 256 or 512; 8-bit inputs use
+// the same shared-memory footprint as 16-bit ones at 256): the caller compares waves of super-tiles on that many
+// clusters with waves of pair tiles on all pairs.  0 = unknown.
+extern "C" int peak_mc_max_clusters(int tile_n) {
+    using namespace peak;
+    using namespace peak::umma;
+    static int cached[kMaxDevices][2] = {};
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices) return 0;
+    const int slot = tile_n == 512 ? 1 : 0;
+    if (cached[dev][slot] != 0) return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(4 * 37);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 4; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (slot == 1) {
+        using C_ = Cfg<2, 512>;
+        auto kernel = umma_gemm_kernel<2, 512, __nv_bfloat16, 1, false, false, false>;
+        cfg.blockDim = dim3(C_::threads(false));
+        cfg.dynamicSmemBytes = C_::SMEM_BYTES;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+    } else {
+        using C_ = Cfg<2, 256>;
+        auto kernel = umma_gemm_kernel<2, 256, __nv_bfloat16, 1, false, false, false>;
+        cfg.blockDim = dim3(C_::threads(false));
+        cfg.dynamicSmemBytes = C_::SMEM_BYTES;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+    }
+    if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    cached[dev][slot] = n > 0 ? n : -1;
+    return n > 0 ? n : 0;
+}
