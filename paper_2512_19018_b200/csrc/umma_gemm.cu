@@ -695,6 +695,11 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         const int64_t t512 = tiles_of(g, 2, 512), t256 = tiles_of(g, 2, 256);
         // (3072^3: 72 wide tiles on 74 pairs, one wave: 40.0 us against 41.3 for two waves of 256-wide tiles)
         wide = num_kb >= min_kb && t512 * 10 >= (int64_t)units * 9 && fill(t512) >= fill(t256) - 0.02;
+        // ... and from 32 k-blocks on where the wide tiles make one wave of what would be two waves of 256-wide ones
+        // (sustained, 16-bit output, beta = 0: 3000^3 1109 against 962 TFLOP/s; ties at 2304^3 and 2560^3)
+        if (!wide && light_tail && !in8 && elem_bytes(out_elem(g.dtype)) == 2 && num_kb >= 32 && t512 <= units &&
+            t256 > units && t512 * 10 >= (int64_t)units * 6)
+            wide = true;
     }
     // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
     // Measured (sustained, random inputs, interleaved): fp16 4096^3 -> fp32 1162 against 1132 (512-wide) and
