@@ -318,7 +318,10 @@ typedef enum peak_tuning_key {
     PEAK_TUNE_SHARE = 18,       /* single-GPU plug-in, 16-bit inputs: single-CTA tiles in clusters of CM x CN tiles that share
                                    their A / B tiles by multicast copies: 1 = never, 100 * w + 10 * CM + CN (w = 1: 128-wide
                                    tiles, 2: 256-wide) = that cluster shape whenever the plug-in is present */
-    PEAK_TUNE_COUNT_ = 19
+    PEAK_TUNE_NARROW = 19,      /* CTA-pair tiles of 192 / 384 columns on the 256- / 512-wide kernels (B transposed, whole tiles),
+                                   chosen where they fill one wave instead of starting a nearly empty second one: 1 = never.
+                                   PEAK_TUNE_TILE_N = 192 / 384 forces them */
+    PEAK_TUNE_COUNT_ = 20
 } peak_tuning_key_t;
 int peak_set_tuning(int key, int value);
 

@@ -246,9 +246,9 @@ def peak_tile_coord(tile, tiles_m, tiles_n, group):
 PEAK_TUNE_RASTER_GROUP, PEAK_TUNE_TILE_N, PEAK_TUNE_SPLIT_K, PEAK_TUNE_EPILOGUE, PEAK_TUNE_SGEMM_FMA, \
     PEAK_TUNE_TAIL_SPLIT, PEAK_TUNE_DEPENDENT_LAUNCH, PEAK_TUNE_SGEMM_COPY, PEAK_TUNE_WAIT_MS, \
     PEAK_TUNE_INJECT_STALL, PEAK_TUNE_MULTICAST, PEAK_TUNE_BALANCED_GRID, PEAK_TUNE_EPILOGUE_WARPS, \
-    PEAK_TUNE_K_ORDER, PEAK_TUNE_SWAP_AB, PEAK_TUNE_SGEMM_TRANSPOSE, PEAK_TUNE_SHORT_A, PEAK_TUNE_CLUSTER_K, PEAK_TUNE_SHARE = \
-    0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18
-PEAK_TUNE_COUNT = 19
+    PEAK_TUNE_K_ORDER, PEAK_TUNE_SWAP_AB, PEAK_TUNE_SGEMM_TRANSPOSE, PEAK_TUNE_SHORT_A, PEAK_TUNE_CLUSTER_K, PEAK_TUNE_SHARE, PEAK_TUNE_NARROW = \
+    0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19
+PEAK_TUNE_COUNT = 20
 
 
 def peak_set_tuning(key: int, value: int) -> int:

@@ -37,7 +37,7 @@ bool knob_allowed(int key) {
     switch (key) {
         case PEAK_TUNE_RASTER_GROUP: case PEAK_TUNE_TILE_N: case PEAK_TUNE_SPLIT_K: case PEAK_TUNE_EPILOGUE:
         case PEAK_TUNE_SGEMM_FMA: case PEAK_TUNE_TAIL_SPLIT: case PEAK_TUNE_SGEMM_COPY: case PEAK_TUNE_MULTICAST:
-        case PEAK_TUNE_BALANCED_GRID: case PEAK_TUNE_EPILOGUE_WARPS: case PEAK_TUNE_K_ORDER: case PEAK_TUNE_SWAP_AB: case PEAK_TUNE_SGEMM_TRANSPOSE: case PEAK_TUNE_SHORT_A: case PEAK_TUNE_CLUSTER_K: case PEAK_TUNE_SHARE:
+        case PEAK_TUNE_BALANCED_GRID: case PEAK_TUNE_EPILOGUE_WARPS: case PEAK_TUNE_K_ORDER: case PEAK_TUNE_SWAP_AB: case PEAK_TUNE_SGEMM_TRANSPOSE: case PEAK_TUNE_SHORT_A: case PEAK_TUNE_CLUSTER_K: case PEAK_TUNE_SHARE: case PEAK_TUNE_NARROW:
             return true;
     }
     return false;

@@ -110,6 +110,12 @@ struct UmmaParams {
     // stored.  a_boxes: MN-major A, how many 64-row (8-bit: 128-row) boxes are fetched; stage_tx: bytes per stage.
     int a_boxes;
     uint32_t stage_tx;
+    // Narrower tiles on the same kernel (CTA pairs, B with k contiguous, whole tiles): the tile is bn_eff <= BN columns
+    // wide -- slot_eff = bn_eff / HALVES per accumulator slot, a multiple of the 128-byte store chunk -- so that a
+    // problem's tiles can fill one wave where the next power of two would leave most of a second wave empty.  Shared
+    // and tensor memory keep the layout of the full width; each CTA fetches hrows_eff = slot_eff / 2 rows of B per
+    // half, and the MMA's N comes from the instruction descriptor.  bn_eff = BN everywhere else.
+    int bn_eff, slot_eff, hrows_eff;
     int bulk_exchange;     // one-tile-per-CTA kernel: 1 = k-slices always travel by bulk copies (also for tiles of <= 32 rows)
     long long wait_cycles; // budget of every mbarrier wait
     int inject_stall;      // test hook: CTA (pair) 0 never fills the stage of its last k-block
@@ -577,7 +583,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 int64_t tm, tn;
                 tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
-                const int n_cta = (int)tn * BN + (int)rank * C_::HROWS;  // first B row of this CTA (half 0)
+                const int n_cta = (int)tn * p.bn_eff + (int)rank * p.hrows_eff;  // first B row of this CTA (half 0)
                 for (int j = 0, nk = w.kb1 - w.kb0; j < nk; ++j, ++it) {
                     const int kb = rev ? w.kb1 - 1 - j : w.kb0 + j;
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
@@ -589,7 +595,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (p.inject_stall && unit == 0 && leader && item + num_units >= total_items && j == nk - 1)
                         continue;  // test hook: leave this stage empty so that the waits downstream run out
                     uint32_t bar = full0 + 8 * s;
-                    if (leader) ptx::mbar_arrive_expect_tx(bar, CG == 1 ? p.stage_tx : (uint32_t)(C_::STAGE_BYTES * CG));
+                    if (leader) ptx::mbar_arrive_expect_tx(bar, p.stage_tx);
                     if (CG == 2) bar = ptx::map_to_cta(bar, leader_crank);
                     const uint32_t a_dst = stage_base + s * C_::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
@@ -609,7 +615,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint16_t mask = (uint16_t)((1u << crank) | (1u << (crank ^ 2u)));
 #pragma unroll
                         for (int hf = 0; hf < C_::HALVES; ++hf) {
-                            const int n_q = n_cta + hf * C_::SLOT_N + 64 * (int)pair;
+                            const int n_q = n_cta + hf * p.slot_eff + 64 * (int)pair;
                             McOps<MC>::load_b_quarter(b_dst + hf * C_::HROWS * 128 + pair * ATOM_BYTES, &tmB,
                                                       p.b_mn ? n_q : k0, p.b_mn ? k0 : n_q, bz, bar, mask);
                         }
@@ -619,7 +625,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                             for (int h = 0; h < C_::HROWS / C_::B_BOX_ROWS; ++h) {
                                 const uint32_t d = b_dst + (hf * C_::HROWS + h * C_::B_BOX_ROWS) * 128;
-                                const int n = n_cta + hf * C_::SLOT_N + C_::B_BOX_ROWS * h;
+                                const int n = n_cta + hf * p.slot_eff + C_::B_BOX_ROWS * h;
                                 load_tile<CG, BATCHED>(d, &tmB, k0, n, bz, bar);
                             }
                         }
@@ -629,7 +635,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                             for (int h = 0; h < C_::HROWS / MN_ELEMS; ++h) {  // (8-bit: HROWS >= 128, host-checked)
                                 const uint32_t d = b_dst + hf * C_::HROWS * 128 + h * MN_ATOM;
-                                const int n = n_cta + hf * C_::SLOT_N + MN_ELEMS * h;
+                                const int n = n_cta + hf * p.slot_eff + MN_ELEMS * h;
                                 load_tile<CG, BATCHED>(d, &tmB, n, k0, bz, bar);
                             }
                         }
@@ -771,7 +777,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int64_t tm, tn;
             tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
-            const int n0 = (int)tn * BN;
+            const int n0 = (int)tn * p.bn_eff;
             const bool live = row0 < p.M;  // none of this warp's 32 rows exists otherwise: nothing to drain
             {
                 const int hf = (C_::HALVES == 2) ? grp : 0;
@@ -780,13 +786,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (cf.on && live && w.ws_block < 0) {
                     // old C of the first two chunks is requested while the main loop still runs
                     constexpr int CC = 128 / (int)sizeof(TOut);
-                    const int c0 = n0 + ((C_::HALVES == 2) ? hf * C_::SLOT_N : (SPLIT_COLS ? grp * W : 0));
+                    const int c0 = n0 + ((C_::HALVES == 2) ? hf * p.slot_eff : (SPLIT_COLS ? grp * W : 0));
+                    const int c_end = min(p.N, n0 + ((C_::HALVES == 2) ? (hf + 1) * p.slot_eff : p.bn_eff));  // end of this warp's columns
                     // (a group whose columns start beyond N has no chunk in this tile: nothing to request, or the
                     // barrier would be armed for a wait that never comes)
-                    if (lane == 0 && c0 < p.N) {
+                    if (lane == 0 && c0 < c_end) {
                         ptx::tma_store_wait_read<0>();  // the previous tile's stores have read the buffer(s)
                         cfetch_issue<TOut, BATCHED>(cf, my_stage, 0, &tmC, c0, row0, bz);
-                        if (!cf.single && c0 + CC < p.N && CC < W) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, c0, row0, bz);
+                        if (!cf.single && c0 + CC < c_end && CC < W) cfetch_issue<TOut, BATCHED>(cf, my_stage, 1, &tmC, c0, row0, bz);
                     }
                     if (cf.single) {
                         // the later chunks are fetched one by one between stores: have them wait in L2
@@ -796,7 +803,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                   (BATCHED ? (int64_t)bz * p.stride_c : 0) + (int64_t)r * p.ldc + c0;
 #pragma unroll
                             for (int c = CC; c < W; c += CC)
-                                if (c0 + c < p.N) ptx::prefetch_l2(row_ptr + c);
+                                if (c0 + c < c_end) ptx::prefetch_l2(row_ptr + c);
                         }
                     }
                     __syncwarp();
@@ -809,10 +816,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const int co = SPLIT_COLS ? grp * W : hf * C_::SLOT_N;  // first tile column of this warp
+                const int co = SPLIT_COLS ? grp * W : hf * C_::SLOT_N;  // first accumulator column of this warp's slot
+                const int cn = SPLIT_COLS ? grp * W : hf * p.slot_eff;  // ... and the tile column it belongs to
                 const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + b * C_::SLOT_N +
                                         (SPLIT_COLS ? (uint32_t)(grp * W) : 0u);
-                const int nh = n0 + co;
+                const int nh = n0 + cn;
+                const int n_end = min(p.N, n0 + ((C_::HALVES == 2) ? (hf + 1) * p.slot_eff : p.bn_eff));
                 if (!live) {
                     // rows beyond M: the partial-tile reduction and C never look at them
                 } else if (SWAP && w.ws_block < 0) {
@@ -825,7 +834,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;
                     if (!epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc, row0 + lane, row0, p.M,
-                                                         nh, p.N, &tmC, nh, row0, bz, p.tma_store != 0, vec, p.alpha,
+                                                         nh, n_end, &tmC, nh, row0, bz, p.tma_store != 0, vec, p.alpha,
                                                          p.beta, p.bias, p.act, reinterpret_cast<const TOut *>(p.R),
                                                          p.ldr, p.r_vec != 0, cf, abort_flag, p.wait_cycles)) {
                         if (lane == 0) report_timeout(p, abort_flag, 6, b);

@@ -48,9 +48,10 @@ constexpr double kL2BytesPerClk = 40.0;        // L2 -> shared-memory bytes per 
 constexpr double kSplitFixedCycles = 20000.0;  // workspace allocation + second launch of a split (~12 us)
 
 struct Plan {
-    int bn;           // tile width: 256 or 128
+    int bn;           // tile width the kernel is instantiated for: 512, 256 or 128
     int full_tiles;   // tiles computed whole
     int tail_splits;  // k-slices of each remaining tile (1 when nothing is split)
+    int bn_eff = 0;   // columns of a tile actually computed (0 = bn): 192 on the 256-wide kernel, 384 on the 512-wide one
 };
 
 // Tiles of the whole call (all matrices of a strided batch).
@@ -158,20 +159,25 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
     // rows of A a single-CTA tile fetches: all 128, or, when the whole problem has fewer, only those that exist
     // (K-major: rounded up to 8; MN-major: whole boxes of MNE rows)
+    const int bn_eff = plan.bn_eff > 0 ? plan.bn_eff : BN;
+    const int slot_eff = bn_eff / C_::HALVES, hrows_eff = slot_eff / CG;
+    if (bn_eff != BN && (CG != 2 || b_mn || nb > 1 || plan.tail_splits != 1 || SWAP || slot_eff % 64 || bn_eff > BN))
+        return PEAK_ERR_UNSUPPORTED;  // narrower tiles: CTA pairs, B with k contiguous, whole tiles of a single matrix
     const bool short_a = CG == 1 && g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
     const int a_rows = short_a ? (int)((g.M + 7) / 8 * 8) : 128;
     const int a_boxes = short_a ? (int)((g.M + MNE - 1) / MNE) : 128 / MNE;
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, MNE, BKE, nb, g.strideA)
                    : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, a_rows, nb, g.strideA);
     ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, MNE, BKE, nb, g.strideB)
-                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS, nb, g.strideB));
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, bn_eff != BN ? hrows_eff : C_::B_BOX_ROWS, nb, g.strideB));
     if (!ok) return nb > 1 ? PEAK_ERR_UNSUPPORTED : PEAK_ERR_CUDA;  // e.g. a batch stride TMA cannot express
 
     UmmaParams p;
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.num_kb = (int)((g.K + BKE - 1) / BKE);
     p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
-    p.tiles_n = (int)((g.N + BN - 1) / BN);
+    p.tiles_n = (int)((g.N + bn_eff - 1) / bn_eff);
+    p.bn_eff = bn_eff; p.slot_eff = slot_eff; p.hrows_eff = hrows_eff;
     // tile-rows per raster group (measured: 16 rows of 256 x 512 tiles are 1 % faster than 8 at 8192^3)
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : ((CG == 1 || BN == 512) ? 16 : 8);
     if (tuning(PEAK_TUNE_RASTER_GROUP) == 0 && nb == 1 && p.tiles_m * (int64_t)p.tiles_n > 2 * units_max) {
@@ -193,11 +199,13 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     p.total_items = plan.full_tiles + (tiles - plan.full_tiles) * plan.tail_splits;
     p.a_mn = a_mn; p.b_mn = b_mn;
     p.a_boxes = a_boxes;
-    p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
+    // bytes a stage's barrier counts: a single CTA's A rows and B tile, or both CTAs' parts of a pair
+    p.stage_tx = CG == 1 ? (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128))
+                         : (uint32_t)(CG * (A_STAGE_BYTES + C_::HALVES * hrows_eff * 128));
     // operand format field: f16 kind: 0 = fp16, 1 = bf16; f8f6f4 kind: 0 = E4M3, 1 = E5M2
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-              ((uint32_t)(C_::SLOT_N >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
+              ((uint32_t)(slot_eff >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.ldc = g.ldc;
     p.bias = g.bias; p.act = g.act;
@@ -258,9 +266,10 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
     cfg.numAttrs = tuning(PEAK_TUNE_DEPENDENT_LAUNCH) == 1 ? 1 : 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, tmW, ws, p);
     count_launch();
-    note_kernel("umma_gemm_kernel<%d, %d, %s, 0, %d, %d, %d, %d> grid=%d items=%d splits=%d", CG, BN,
+    note_kernel("umma_gemm_kernel<%d, %d, %s, 0, %d, %d, %d, %d> grid=%d items=%d splits=%d%s", CG, BN,
                 sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"),
-                (int)BATCHED, (int)IN8, (int)G2, (int)SWAP, units * CG, p.total_items, plan.tail_splits);
+                (int)BATCHED, (int)IN8, (int)G2, (int)SWAP, units * CG, p.total_items, plan.tail_splits,
+                bn_eff == BN ? "" : (bn_eff == 192 ? " width=192" : " width=384"));
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     if (plan.full_tiles == tiles) return PEAK_OK;
 
@@ -326,6 +335,7 @@ template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, 
 
 // Bytes of fp32 partial tiles a plan needs (0 when nothing is split).
 size_t workspace_bytes(const GemmArgs &g, int cg, const Plan &plan) {
+    if (plan.tail_splits <= 1) return 0;
     const int64_t split_tiles = tiles_of(g, cg, plan.bn) - plan.full_tiles;
     return (size_t)split_tiles * plan.tail_splits * (size_t)(BM * cg) * plan.bn * sizeof(float);
 }
@@ -440,6 +450,7 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
     p.a_boxes = a_boxes;
     p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
     p.bulk_exchange = tuning(PEAK_TUNE_CLUSTER_K) == 2 ? 1 : 0;
+    p.bn_eff = BN; p.slot_eff = BN; p.hrows_eff = BN;
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -706,6 +717,38 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // 1108 (256-wide); +12 % at 5000x3000x2500; but with 16-bit output, where the exposed epilogue of the wide
     // tile is half as long, the wide tile wins (bf16 4096^3: 1231 against 1244-1249), and from 2.7e11 flop on
     // the plug-in loses 3-6 % (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
+    // Narrower tiles on the 256- / 512-wide pair kernels (192 / 384 columns; B with k contiguous, whole tiles): taken
+    // when a cycle estimate -- waves x k-blocks x the slower of the tensor pipe (2 cycles per column) and the operand
+    // stream (56 bytes per clock per SM), plus the exposed epilogue of a two-half tile -- says they beat the plan
+    // above by 15 %, which happens when they fill a single wave much better (measured, us, bf16 NT: 2304^3 32.1 -> 28.2,
+    // 2560^3 34.6 -> 30.4 with 384-wide tiles; cuBLAS 21.0 / 26.7; at an estimated 10 % the gains were 0-4 %).
+    // PEAK_TUNE_TILE_N = 192 / 384 forces them, PEAK_TUNE_NARROW = 1 switches the rule off.
+    if (cta_group == 2 && g.transB && g.nbatch() == 1 && plan.tail_splits == 1) {
+        const int forced = tuning(PEAK_TUNE_TILE_N);
+        const int bke = in8 ? 2 * BK : BK;
+        const int64_t num_kb = (g.K + bke - 1) / bke;
+        const int64_t rows = (g.M + 255) / 256;
+        auto estimate = [&](int w) {
+            const int64_t tiles = rows * ((g.N + w - 1) / w);
+            const int64_t waves = (tiles + units - 1) / units;
+            const double per_kb = fmax(2.0 * w, (16384.0 + 64.0 * w) / 56.0);
+            const double tail = w > 256 ? (g.beta != 0.0f ? 14000.0 : (elem_bytes(out_elem(g.dtype)) == 4 ? 11000.0 : 8000.0)) : 3000.0;
+            return (double)waves * ((double)num_kb * per_kb + (w > 256 ? tail : 0.0)) + (w > 256 ? 0.0 : tail);
+        };
+        int narrow = 0;
+        if (forced == 192 || forced == 384) narrow = forced;
+        else if (forced == 0 && tuning(PEAK_TUNE_NARROW) != 1 && g.M > 128) {
+            const double now = estimate(wide ? 512 : plan.bn);
+            const double e192 = estimate(192), e384 = estimate(384);
+            if (plan.bn >= 256 && e192 < 0.85 * now && e192 <= e384) narrow = 192;
+            else if (plan.bn >= 256 && e384 < 0.85 * now) narrow = 384;
+        }
+        if (narrow) {
+            Plan pn{narrow == 192 ? 256 : 512, (int)(rows * ((g.N + narrow - 1) / narrow)), 1, narrow};
+            const int rc = narrow == 192 ? run_umma<2, 256>(g, pn, units) : run_umma<2, 512>(g, pn, units);
+            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+        }
+    }
     const int mc_mode = tuning(PEAK_TUNE_MULTICAST);  // 1 = never, 2 = whenever possible
     // With a 16-bit output the wide tile is preferred, and the plug-in then shares its 512-wide B tile between
     // the two pairs of a cluster (512 x 512 super-tiles): bf16 4096^3 1222 -> 1248 in the bench protocol; at

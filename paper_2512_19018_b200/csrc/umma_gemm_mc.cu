@@ -106,8 +106,9 @@ template <typename TOut, bool G2, int BN = 256, bool IN8 = false> int launch_mc(
     p.c_prefetch = (p.tma_store && r->beta != 0.0f && r->epilogue != 3) ? 1 : 0;
     if (p.tma_store && !make_map(&tmC, eout, r->C, r->N, r->M, r->ldc, 128 / ob, 32)) return PEAK_ERR_CUDA;
     p.k_alternate = r->k_order == 2 ? 1 : 0;
-    p.a_boxes = BM / 64; p.stage_tx = (uint32_t)C_::STAGE_BYTES;  // (pairs take their own byte count)
+    p.a_boxes = BM / 64; p.stage_tx = (uint32_t)(C_::STAGE_BYTES * CG);  // both CTAs' parts arrive at the leader's barrier
     p.bulk_exchange = 0;
+    p.bn_eff = BN; p.slot_eff = C_::SLOT_N; p.hrows_eff = C_::HROWS;
     p.status = r->status;
     p.wait_cycles = r->wait_ms > 0 ? (long long)r->wait_ms * 2000000LL : ptx::kWaitBudgetCycles;
     p.inject_stall = r->inject_stall == 1 ? 1 : 0;

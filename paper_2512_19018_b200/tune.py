@@ -40,7 +40,7 @@ SPACE_F32 = {
     7: [1, 2],                   # PEAK_TUNE_SGEMM_COPY
     0: [0, 4, 16],
 }
-NUM_KEYS = 19
+NUM_KEYS = 20
 
 
 def candidates(space: dict, quick: bool = False):

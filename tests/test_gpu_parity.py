@@ -891,6 +891,59 @@ def test_shared_operand_clusters_bounded_wait(reset_tuning):
     R.check_full(dc)
 
 
+@pytest.mark.parametrize("ta,tb", [(0, 1), (1, 1)])
+def test_narrower_pair_tiles_exact_and_selected(ta, tb, reset_tuning):
+    """CTA-pair tiles of 192 / 384 columns on the 256- / 512-wide kernels (B with k contiguous): exact on integers
+    for ragged shapes, alpha / beta (old C by TMA and by per-thread loads), fp32 and 16-bit outputs, 8-bit inputs, one
+    and two groups of epilogue warps, the fused tail; the same bits as the full-width tiles; chosen by the dispatcher
+    where one wave of 384-wide tiles replaces a poorly filled wave of 512-wide ones."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(47)
+    for idx, (M, N, K) in enumerate([(512, 768, 256), (700, 1000, 264), (1024, 1920, 520), (300, 400, 72), (260, 2304, 136)]):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_E4M3_BF16):
+            unit = 16 if dtype == W.PEAK_E4M3_BF16 else 8
+            pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb,
+                   pad_c=[0, 8, 3][idx % 3], case=idx)
+            want = None
+            for width in (0, 192, 384):
+                for epi, warps in ((0, 0), (3, 1), (1, 2)):
+                    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, width)
+                    P.peak_set_tuning(P.PEAK_TUNE_EPILOGUE, epi)
+                    P.peak_set_tuning(P.PEAK_TUNE_EPILOGUE_WARPS, warps)
+                    P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, 1)
+                    dc = R.DeviceCase(c)
+                    dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+                    assert (f"width={width}" in P.peak_last_kernel()) == (width != 0), P.peak_last_kernel()
+                    got = dc.result()
+                    got = got.view(np.uint32) if c.out_type == "f32" else got
+                    if want is None:
+                        ref, _ = dc.oracle_full()
+                        want = oracle.round_to(R.OT[c.out_type], ref)
+                    assert np.array_equal(got, want), f"{c} width={width} epilogue={epi} warps={warps}"
+    for k in range(P.PEAK_TUNE_COUNT):
+        P.peak_set_tuning(k, 0)
+    c = W.GemmCase("narrow_fused", W.PEAK_BF16_BF16, bool(ta), bool(tb), 520, 1100, 264, 0.5, 2.0, "uniform", pad_a=(-(520 if ta else 264)) % 8,
+                   pad_b=0)
+    bias = rng.standard_normal(c.N).astype(np.float32)
+    res = make_residual(c, rng, 2)
+    for width in (192, 384):
+        P.peak_set_tuning(P.PEAK_TUNE_TILE_N, width)
+        dc = run_fused(c, P.PEAK_VARIANT_UMMA_2CTA, bias, P.PEAK_ACT_GELU, res)
+        assert f"width={width}" in P.peak_last_kernel()
+        check_fused(dc, bias, P.PEAK_ACT_GELU, f"narrow tiles fused {c.layout} width={width}", res)
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 0)
+    big = mk(W.PEAK_BF16_BF16, ta, tb, 2560, 2560, 2560, pad_a=0, pad_b=0)
+    dc = R.DeviceCase(big)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "width=384" in P.peak_last_kernel(), P.peak_last_kernel()
+    R.check_sampled(dc, tile_m=256, tile_n=384, what="2560^3 on 384-wide tiles")
+    P.peak_set_tuning(P.PEAK_TUNE_NARROW, 1)
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "width=" not in P.peak_last_kernel()
+
+
 # ------------------------------------------------------------------ exchanged operands (M <= 64)
 @pytest.mark.parametrize("ta,tb", LAYOUTS)
 def test_swapped_operands_exact_and_selected(ta, tb, reset_tuning):

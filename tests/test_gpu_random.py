@@ -41,7 +41,7 @@ def test_random_cases_against_the_oracle(seed):
             dist = str(rng.choice(["uniform", "smallint", "uniform"]))
             c = W.GemmCase(f"r{seed}_{n}", dt, bool(ta), bool(tb), M, N, K, alpha, beta, dist, pad_a=pa, pad_b=pb,
                            pad_c=pc, case=1000 * seed + n)
-            knobs = {P.PEAK_TUNE_TILE_N: int(rng.choice([0, 0, 128, 256, 512])),
+            knobs = {P.PEAK_TUNE_TILE_N: int(rng.choice([0, 0, 128, 256, 512, 192, 384])),
                      P.PEAK_TUNE_EPILOGUE: int(rng.choice([0, 0, 1, 2, 3])),
                      P.PEAK_TUNE_EPILOGUE_WARPS: int(rng.choice([0, 1, 2])),
                      P.PEAK_TUNE_SPLIT_K: int(rng.choice([0, 0, 0, 1, 2, 3])),
