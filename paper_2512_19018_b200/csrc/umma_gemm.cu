@@ -82,9 +82,13 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
     if (cg == 1 && g.nbatch() == 1 && !force_bn && !force_split && tail_mode != 2 && tuning(PEAK_TUNE_CLUSTER_K) != 1) {
         const int64_t t128 = tiles_of(g, 1, 128);
         if (t128 <= units && t128 * 8 > units) {
+            // a split must shorten the main loop (about 0.22 us per k-block) by more than the exchange costs: about
+            // 1 us for tiles of at most 32 rows, 4-5 us otherwise (fp16 1024^3 -> fp32, 16 k-blocks: whole tiles 7.7 us,
+            // two slices 8.6; bf16 1024x1024x2048, 32 k-blocks: 9.8 against 10.3; 256x4096x4096, 64: 20.7 against 16.3)
+            const int64_t need_saved = g.M <= 32 ? 6 : 24;
             for (int s : {4, 2}) {
                 const int64_t kbps = (num_kb + s - 1) / s;
-                if (t128 * s > units || kbps < 8 || kbps * (s - 1) >= num_kb) continue;
+                if (t128 * s > units || kbps < 8 || kbps * (s - 1) >= num_kb || num_kb - kbps < need_saved) continue;
                 if (t128 > clusterk_max_clusters(128, s)) continue;
                 return Plan{128, 0, s};
             }

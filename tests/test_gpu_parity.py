@@ -641,7 +641,7 @@ def test_cuda_graph_with_k_split_and_several_calls():
              mk(W.PEAK_BF16_BF16, 0, 0, 512, 1024, 4096, case=3),
              # the one-tile-per-CTA kernel: four k-slices on a cluster, two k-slices, whole tiles
              mk(W.PEAK_BF16_BF16, 1, 0, 16, 4096, 4096, alpha=0.5, beta=2.0, case=4),
-             mk(W.PEAK_BF16_F32, 0, 1, 128, 4096, 1024, alpha=1.0, beta=1.0, case=5),
+             mk(W.PEAK_BF16_F32, 0, 1, 128, 6400, 3200, alpha=1.0, beta=1.0, case=5),
              mk(W.PEAK_F16_F16, 0, 0, 256, 2560, 512, alpha=2.0, beta=0.0, case=6)]
     dcs = [R.DeviceCase(c) for c in cases]
     stream = torch.cuda.Stream()
