@@ -32,8 +32,8 @@
 namespace peak {
 namespace umma {
 
-template <int BN, int KC> struct ClusterKCfg {
-    using C_ = Cfg<1, BN>;
+template <int BN, int KC, int CG = 1> struct ClusterKCfg {
+    using C_ = Cfg<CG, BN>;
     static constexpr int SW = BN / KC;            // columns each CTA finalises
     static constexpr int CHUNKS = SW / 32;        // 32-column chunks per slice
     // receive area [peer 0..KC-2][chunk][row][128 bytes] and, behind it, a send area of the same shape, both in the ring
@@ -52,17 +52,21 @@ template <int BN, int KC> struct ClusterKCfg {
     static constexpr int ISSUER2 = PRODUCER2 + 1;
     static constexpr int THREADS = 32 * (ISSUER2 + 1);
     static_assert(KC == 1 || KC == 2 || KC == 4, "cluster sizes");
+    static_assert(CG == 1 || (CG == 2 && KC == 1 && BN == 128), "CTA pairs: whole 256 x 128 tiles");
     static_assert(SW % 32 == 0 && SW >= 32, "a slice is a whole number of 32-column chunks");
     static_assert(RECV_BYTES <= C_::STAGES * C_::STAGE_BYTES, "the receive area lives in the stage ring");
     static_assert((DUAL ? 2 : 1) * BN <= TMEM_COLS, "accumulators fit the allocation");
 };
 
-template <int BN, typename TOut, int KC, bool IN8>
-__global__ void __launch_bounds__((ClusterKCfg<BN, KC>::THREADS), 1)
+// CG = 2: the tile is 256 x 128, computed by a CTA pair (cta_group::2 MMAs issued by the pair's leader; each CTA
+// stages its 128 rows of A and its 64-row half of the B tile, a quarter less per SM than two 128 x 128 tiles, which
+// is what bounds one-wave problems once the issuing threads are out of the way); whole tiles only (KC = 1).
+template <int BN, typename TOut, int KC, bool IN8, int CG = 1>
+__global__ void __launch_bounds__((ClusterKCfg<BN, KC, CG>::THREADS), 1)
 umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
-    using C_ = Cfg<1, BN>;
-    using K_ = ClusterKCfg<BN, KC>;
+    using C_ = Cfg<CG, BN>;
+    using K_ = ClusterKCfg<BN, KC, CG>;
     constexpr int STAGES = C_::STAGES;
     constexpr int SW = K_::SW;
     extern __shared__ uint8_t smem_raw[];
@@ -85,11 +89,15 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     constexpr int MN_ATOM = IN8 ? 2 * ATOM_BYTES : ATOM_BYTES;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t me = KC > 1 ? ptx::cluster_ctarank() : 0u;  // k-slice of this CTA, and the column slice it finalises
-    const int tile = blockIdx.x / KC;
+    const uint32_t crank = (KC > 1 || CG > 1) ? ptx::cluster_ctarank() : 0u;
+    const uint32_t me = crank / CG;            // k-slice of this CTA, and the column slice it finalises
+    const uint32_t rank = crank % CG;          // position inside a CTA pair (always 0 for single-CTA tiles)
+    const uint32_t leader_crank = crank - rank;
+    const bool leader = rank == 0;
+    const int tile = blockIdx.x / (KC * CG);
     int64_t tm, tn;
     tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-    const int m0 = (int)tm * BM, n0 = (int)tn * BN;
+    const int m0 = (int)tm * (BM * CG) + (int)rank * BM, n0 = (int)tn * BN;
     const int kb0 = (int)me * p.kb_per_split;
     const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);  // the host guarantees kb0 < kb1
     // How the k-slices travel (KC > 1).  A tile with at most 32 rows: the one warp that owns them writes its few
@@ -121,13 +129,15 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (p.tma_store) ptx::prefetch_tensormap(&tmC);
     }
     if (warp == 1) {
-        ptx::tmem_alloc<1>(ptx::smem_u32(tmem_slot), K_::TMEM_COLS);
-        ptx::tmem_relinquish<1>();
+        ptx::tmem_alloc<CG>(ptx::smem_u32(tmem_slot), K_::TMEM_COLS);
+        ptx::tmem_relinquish<CG>();
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    // this CTA's barriers exist: tell the peers (they wait for it only when the main loop is over)
-    if (KC > 1) ptx::cluster_arrive();
+    // this CTA's barriers exist: tell the peers (k-slices wait for it only when the main loop is over; the CTAs of a
+    // pair signal each other's barriers from the first copy on and wait here)
+    if (CG == 2) ptx::cluster_sync();
+    else if (KC > 1) ptx::cluster_arrive();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's shared and tensor memory and may overlap the previous kernel
@@ -172,18 +182,20 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int h = is_a ? lane : lane - a_ops;
         const CUtensorMap *tmap = is_a ? &tmA : &tmB;
         const bool mn = is_a ? p.a_mn != 0 : p.b_mn != 0;
-        const int mn0 = (is_a ? m0 : n0) + h * (mn ? MN_ELEMS : (is_a ? 0 : C_::B_BOX_ROWS));
+        const int mn0 = (is_a ? m0 : n0 + (int)rank * C_::HROWS) + h * (mn ? MN_ELEMS : (is_a ? 0 : C_::B_BOX_ROWS));
         const uint32_t off = (is_a ? 0u : (uint32_t)A_STAGE_BYTES) +
                              (uint32_t)h * (mn ? (uint32_t)MN_ATOM : (uint32_t)(C_::B_BOX_ROWS * 128));
         uint32_t it = (uint32_t)pw;
         for (int kb = kb0 + pw; kb < kb1; kb += 2, it += 2) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            const uint32_t bar = full0 + 8 * s;
+            // the bytes of a stage are counted by the barrier of the pair's leader (its own, for single-CTA tiles)
+            const uint32_t bar = CG == 2 ? ptx::map_to_cta(full0 + 8 * s, leader_crank) : full0 + 8 * s;
             bool go = true;
             if (lane == 0) {
-                go = ptx::mbar_wait<false>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles);
+                go = ptx::mbar_wait<CG == 2>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.wait_cycles);
                 if (!go) report_timeout(p, abort_flag, 1, s);
-                else if (!(p.inject_stall && blockIdx.x == 0 && kb == kb1 - 1)) ptx::mbar_arrive_expect_tx(bar, p.stage_tx);
+                else if (leader && !(p.inject_stall && blockIdx.x == 0 && kb == kb1 - 1))
+                    ptx::mbar_arrive_expect_tx(full0 + 8 * s, p.stage_tx);
             }
             go = __shfl_sync(0xffffffffu, go, 0);
             if (!go) break;
@@ -192,7 +204,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             if (mine) {
                 const int k0 = kb * (IN8 ? 2 * BK : BK);
                 const uint32_t dst = stage_base + s * C_::STAGE_BYTES + off;
-                ptx::tma_load_2d(dst, tmap, mn ? mn0 : k0, mn ? k0 : mn0, bar);  // one instruction for all lanes
+                if (CG == 2) ptx::tma_load_2d_pair(dst, tmap, mn ? mn0 : k0, mn ? k0 : mn0, bar);
+                else ptx::tma_load_2d(dst, tmap, mn ? mn0 : k0, mn ? k0 : mn0, bar);  // one instruction for all lanes
             }
             __syncwarp();
         }
@@ -204,7 +217,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         // when the accumulators are read.
         constexpr int NI = K_::DUAL ? 2 : 1;
         const int iw = warp == 1 ? 0 : 1;
-        if (lane == 0 && iw < NI) {
+        if (lane == 0 && iw < NI && leader) {
             const uint32_t a_lbo = p.a_mn ? (uint32_t)MN_ATOM : 16u, b_lbo = p.b_mn ? (uint32_t)MN_ATOM : 16u;
             constexpr uint32_t MN_KSTEP = IN8 ? 4096u : 2048u;
             const uint32_t a_kstep = p.a_mn ? MN_KSTEP : 32u, b_kstep = p.b_mn ? MN_KSTEP : 32u;
@@ -213,7 +226,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool mma_ok = true;
             for (int kb = kb0 + iw; kb < kb1; kb += NI, it += NI) {
                 const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                if (!ptx::mbar_wait<false>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
+                if (!ptx::mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.wait_cycles)) {
                     report_timeout(p, abort_flag, 4, s);
                     mma_ok = false;
                     break;
@@ -225,12 +238,18 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 for (int k = 0; k < BK / UMMA_K; ++k) {
                     const uint64_t ad = smem_desc(a_base + k * a_kstep, a_lbo, 1024u);
                     const uint64_t bd = smem_desc(b_base + k * b_kstep, b_lbo, 1024u);
-                    if (IN8) ptx::umma_f8<1>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
-                    else ptx::umma_f16<1>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
+                    if (IN8) ptx::umma_f8<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
+                    else ptx::umma_f16<CG>(d_tmem, ad, bd, p.idesc, (uint32_t)((kb > kb0 + iw) | (k != 0)));
                 }
-                ptx::umma_commit_1cta(empty0 + 8 * s);
+                // release the stage (in both CTAs of a pair) once these MMAs have read it
+                if (CG == 1) ptx::umma_commit_1cta(empty0 + 8 * s);
+                else ptx::umma_commit_pair(empty0 + 8 * s, (uint16_t)(3u << leader_crank));
             }
-            if (mma_ok) ptx::umma_commit_1cta(accfull);  // (an issuer without k-blocks arrives at once)
+            // (an issuer without k-blocks arrives at once)
+            if (mma_ok) {
+                if (CG == 1) ptx::umma_commit_1cta(accfull);
+                else ptx::umma_commit_pair(accfull, (uint16_t)(3u << leader_crank));
+            }
         }
         __syncwarp();
     } else {
@@ -241,7 +260,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             if (!cf.single && c_first + CC < c_limit) cfetch_issue<TOut, false>(cf, my_stage, 1, &tmC, c_first, row0, 0);
         }
         __syncwarp();
-        const bool got = ptx::mbar_wait<false>(accfull, 0u, abort_flag, p.wait_cycles);
+        const bool got = ptx::mbar_wait<CG == 2>(accfull, 0u, abort_flag, p.wait_cycles);
         ok = __all_sync(0xffffffffu, got);
         if (!ok && lane == 0) report_timeout(p, abort_flag, 5, 0);
         ptx::tc_fence_after_sync();
@@ -413,9 +432,10 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (CG == 2) ptx::cluster_sync();  // the peer may still signal this CTA's barriers or read its tiles
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc<1>(tmem_base, K_::TMEM_COLS);
+        ptx::tmem_dealloc<CG>(tmem_base, K_::TMEM_COLS);
     }
 }
 

@@ -418,11 +418,11 @@ int run_umma_static_ws(const GemmArgs &g, int splits, float *ws) {
 // ---- k-slices on the CTAs of a cluster, added through distributed shared memory (umma_clusterk.cuh) -------
 // One launch instead of tile kernel + reduction kernel, no workspace.  Single matrices, single-CTA tiles,
 // every tile split KC = 2 or 4 ways.
-template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const GemmArgs &g, const Plan &plan) {
-    using C_ = Cfg<1, BN>;
+template <int BN, typename TOut, int KC, bool IN8, int CG = 1> int launch_clusterk(const GemmArgs &g, const Plan &plan) {
+    using C_ = Cfg<CG, BN>;
     constexpr int BKE = IN8 ? 2 * BK : BK;
     constexpr int MNE = IN8 ? 128 : 64;
-    auto kernel = umma_clusterk_kernel<BN, TOut, KC, IN8>;
+    auto kernel = umma_clusterk_kernel<BN, TOut, KC, IN8, CG>;
     static PerDeviceOnce attr_once;
     const cudaError_t attr_err = attr_once.run(current_device(), [&] {
         return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM_BYTES);
@@ -431,7 +431,7 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
     const Elem ein = in_elem(g.dtype), eout = out_elem(g.dtype);
     const int a_mn = g.transA ? 1 : 0, b_mn = g.transB ? 0 : 1;
     if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
-    const bool short_a = g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
+    const bool short_a = CG == 1 && g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
     const int a_rows = short_a ? (int)((g.M + 7) / 8 * 8) : 128;
     const int a_boxes = short_a ? (int)((g.M + MNE - 1) / MNE) : 128 / MNE;
     CUtensorMap tmA, tmB, tmC;
@@ -442,22 +442,23 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
     UmmaParams p = {};
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.num_kb = (int)((g.K + BKE - 1) / BKE);
-    p.tiles_m = (int)((g.M + BM - 1) / BM);
+    p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((g.N + BN - 1) / BN);
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 16;
     p.tiles_per_batch = p.tiles_m * p.tiles_n;
     p.full_tiles = 0;
     p.tail_splits = KC;
     p.kb_per_split = (p.num_kb + KC - 1) / KC;
-    p.total_items = p.tiles_per_batch * KC;
+    p.total_items = p.tiles_per_batch * KC * CG;  // CTAs
     p.a_mn = a_mn; p.b_mn = b_mn;
     p.a_boxes = a_boxes;
-    p.stage_tx = (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128));
+    p.stage_tx = CG == 1 ? (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128))
+                         : (uint32_t)(CG * C_::STAGE_BYTES);  // both CTAs' parts arrive at the leader's barrier
     p.bulk_exchange = tuning(PEAK_TUNE_CLUSTER_K) == 2 ? 1 : 0;
     p.bn_eff = BN; p.slot_eff = BN; p.hrows_eff = BN;
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.ldc = g.ldc;
     p.bias = g.bias; p.act = g.act;
@@ -478,12 +479,12 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.total_items);
-    cfg.blockDim = dim3(ClusterKCfg<BN, KC>::THREADS);
+    cfg.blockDim = dim3(ClusterKCfg<BN, KC, CG>::THREADS);
     cfg.dynamicSmemBytes = C_::SMEM_BYTES;
     cfg.stream = g.stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = KC; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.x = KC * CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
@@ -496,9 +497,9 @@ template <int BN, typename TOut, int KC, bool IN8> int launch_clusterk(const Gem
         return PEAK_ERR_UNSUPPORTED;
     }
     count_launch();
-    note_kernel("umma_clusterk_kernel<%d, %s, %d, %d> grid=%d clusters=%d", BN,
+    note_kernel("umma_clusterk_kernel<%d, %s, %d, %d%s> grid=%d clusters=%d", BN,
                 sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"), KC, (int)IN8,
-                p.total_items, p.tiles_per_batch);
+                CG == 2 ? ", 2" : "", p.total_items, p.tiles_per_batch);
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
@@ -561,7 +562,35 @@ int clusterk_max_clusters(int bn, int kc) {
     return kc == 2 ? max_clusters_of<256, 2>() : max_clusters_of<256, 4>();
 }
 
+// Whole tiles as 256 x 128 pair tiles (a quarter fewer operand bytes per SM) when the problem has at least two
+// 128-row blocks and its pair tiles still run at once; 16-bit inputs, or 8-bit ones with B stored N x K.
+// PEAK_TUNE_CLUSTER_K = 3 keeps single-CTA tiles.
+template <typename TOut, bool IN8> int launch_pair_tiles(const GemmArgs &g, const Plan &plan) {
+    return launch_clusterk<128, TOut, 1, IN8, 2>(g, plan);
+}
+bool pair_tiles_apply(const GemmArgs &g) {
+    if (tuning(PEAK_TUNE_CLUSTER_K) == 3 || g.M <= 128) return false;
+    if (is_fp8(in_elem(g.dtype)) && !g.transB) return false;  // an 8-bit B stored K x N needs 128 columns per CTA
+    // (from 32 k-blocks on: measured, us, pair against single tiles: 512x4096x4096 18.8 / 21.6, 2048x1024x4096
+    // 18.8 / 22.1, 1024x2048x2048 11.1 / 11.6, but 1536^3 10.9 / 9.8 and 1024^3 7.5 / 7.2)
+    const int bke = is_fp8(in_elem(g.dtype)) ? 2 * BK : BK;
+    if ((g.K + bke - 1) / bke < 32 && tuning(PEAK_TUNE_CLUSTER_K) != 4) return false;  // 4 = pairs whenever possible
+    const int64_t pair_tiles = ((g.M + 255) / 256) * ((g.N + 127) / 128);
+    return 2 * pair_tiles <= (int64_t)sm_count();
+}
+
 int run_clusterk(const GemmArgs &g, const Plan &plan) {
+    if (plan.tail_splits == 1 && pair_tiles_apply(g)) {
+        const bool in8 = is_fp8(in_elem(g.dtype));
+        switch (out_elem(g.dtype)) {
+            case Elem::F32: return in8 ? launch_pair_tiles<float, true>(g, plan) : launch_pair_tiles<float, false>(g, plan);
+            case Elem::F16: return launch_pair_tiles<__half, false>(g, plan);
+            case Elem::BF16:
+                return in8 ? launch_pair_tiles<__nv_bfloat16, true>(g, plan) : launch_pair_tiles<__nv_bfloat16, false>(g, plan);
+            default: break;
+        }
+        return PEAK_ERR_INVALID_VALUE;
+    }
     if (plan.tail_splits == 1) return launch_clusterk_typed<128, 1>(g, plan);
     if (plan.bn == 128)
         return plan.tail_splits == 2 ? launch_clusterk_typed<128, 2>(g, plan) : launch_clusterk_typed<128, 4>(g, plan);

@@ -815,6 +815,52 @@ def test_one_tile_per_cta_kernel_two_issuers_exact(reset_tuning):
     assert np.array_equal(first, dc.result())
 
 
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_one_tile_per_pair_kernel_exact(ta, tb, reset_tuning):
+    """Whole tiles of a one-wave problem with at least two 128-row blocks run as 256 x 128 CTA-pair tiles (the pair's
+    leader issues cta_group::2 MMAs from two threads into two accumulators; each CTA stages its rows of A and its
+    half of the B tile).  Exact on integers in every layout for ragged M (a pair whose second CTA has no rows), N,
+    K, one k-block, odd counts, every output type, 8-bit inputs with B stored N x K, beta != 0; the same bits as
+    single-CTA tiles; chosen by the dispatcher from 32 k-blocks on."""
+    shapes = [(256, 1024, 64), (300, 1000, 136), (129, 520, 1544), (512, 4100, 520), (700, 1280, 2056)]
+    for idx, (M, N, K) in enumerate(shapes):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16, W.PEAK_E4M3_BF16):
+            in8 = dtype == W.PEAK_E4M3_BF16
+            if in8 and not tb:
+                continue
+            unit = 16 if in8 else 8
+            pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb,
+                   pad_c=[0, 8, 3][idx % 3], case=idx)
+            outs = []
+            for mode in (4, 3):
+                P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 128)
+                P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 1)
+                P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, mode)
+                dc = R.DeviceCase(c)
+                dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+                name = P.peak_last_kernel()
+                assert "umma_clusterk_kernel<128," in name and (", 2> " in name) == (mode == 4), name
+                ref, _ = dc.oracle_full()
+                want = oracle.round_to(R.OT[c.out_type], ref)
+                got = dc.result()
+                got = got.view(np.uint32) if c.out_type == "f32" else got
+                assert np.array_equal(got, want), f"{c} cluster_k={mode}"
+                outs.append(got.copy())
+            assert np.array_equal(outs[0], outs[1])
+    for k in range(P.PEAK_TUNE_COUNT):
+        P.peak_set_tuning(k, 0)
+    c = mk(W.PEAK_BF16_BF16, ta, tb, 512, 4096, 2048, alpha=0.5, beta=2.0)
+    dc = R.DeviceCase(c)
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert "umma_clusterk_kernel<128, __nv_bfloat16, 1, 0, 2>" in P.peak_last_kernel(), P.peak_last_kernel()
+    R.check_sampled(dc, tile_m=256, tile_n=128, what=f"{c}")
+    first = dc.result().copy()
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_AUTO)
+    assert np.array_equal(first, dc.result())
+
+
 def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
     """The stalled-stage hook in the cluster-split kernel: the CTA whose stage never fills gives up after its
     budget, still reaches both cluster barriers (its peers wait there, not on a flag), the status word reports the
@@ -836,6 +882,24 @@ def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
     dc.reset_c()
     dc.run(P.PEAK_VARIANT_UMMA_1CTA)
     assert "umma_clusterk_kernel" in P.peak_last_kernel()
+    R.check_full(dc)
+    # the same with whole 256 x 128 pair tiles: the leader's last stage never fills, both CTAs of the pair unwind
+    c = mk(W.PEAK_BF16_BF16, 0, 1, 256, 512, 2048)
+    dc = R.DeviceCase(c)
+    P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 1)
+    P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, 4)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 20)
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 1)
+    P.peak_gemm_variant(P.PEAK_VARIANT_UMMA_1CTA, c.dtype, c.transA, c.transB, c.M, c.N, c.K, 1.0, dc.A, c.lda, dc.B, c.ldb,
+                        0.0, dc.C, c.ldc)
+    assert ", 2> " in P.peak_last_kernel(), P.peak_last_kernel()
+    rc, detail = P.peak_check()
+    assert rc == P.PEAK_ERR_TIMEOUT and (detail & 0x80000000)
+    P.peak_set_tuning(P.PEAK_TUNE_INJECT_STALL, 0)
+    P.peak_set_tuning(P.PEAK_TUNE_WAIT_MS, 0)
+    dc.reset_c()
+    dc.run(P.PEAK_VARIANT_UMMA_1CTA)
+    assert ", 2> " in P.peak_last_kernel()
     R.check_full(dc)
 
 

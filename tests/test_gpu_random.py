@@ -53,7 +53,7 @@ def test_random_cases_against_the_oracle(seed):
                      P.PEAK_TUNE_SWAP_AB: int(rng.choice([0, 0, 1, 2])),
                      P.PEAK_TUNE_SGEMM_TRANSPOSE: int(rng.choice([0, 1, 2])),
                      P.PEAK_TUNE_SHORT_A: int(rng.choice([0, 0, 1])),
-                     P.PEAK_TUNE_CLUSTER_K: int(rng.choice([0, 0, 1]))}
+                     P.PEAK_TUNE_CLUSTER_K: int(rng.choice([0, 0, 1, 2, 3, 4]))}
             for k, v in knobs.items():
                 P.peak_set_tuning(k, v)
             variant = int(rng.choice([P.PEAK_VARIANT_AUTO, P.PEAK_VARIANT_AUTO, P.PEAK_VARIANT_UMMA_1CTA,
