@@ -52,7 +52,7 @@ template <int BN, int KC, int CG = 1> struct ClusterKCfg {
     static constexpr int ISSUER2 = PRODUCER2 + 1;
     static constexpr int THREADS = 32 * (ISSUER2 + 1);
     static_assert(KC == 1 || KC == 2 || KC == 4, "cluster sizes");
-    static_assert(CG == 1 || (CG == 2 && KC == 1 && BN == 128), "CTA pairs: whole 256 x 128 tiles");
+    static_assert(CG == 1 || (CG == 2 && KC <= 2 && BN == 128), "CTA pairs: 256 x 128 tiles, whole or in two k-slices");
     static_assert(SW % 32 == 0 && SW >= 32, "a slice is a whole number of 32-column chunks");
     static_assert(RECV_BYTES <= C_::STAGES * C_::STAGE_BYTES, "the receive area lives in the stage ring");
     static_assert((DUAL ? 2 : 1) * BN <= TMEM_COLS, "accumulators fit the allocation");
@@ -60,7 +60,8 @@ template <int BN, int KC, int CG = 1> struct ClusterKCfg {
 
 // CG = 2: the tile is 256 x 128, computed by a CTA pair (cta_group::2 MMAs issued by the pair's leader; each CTA
 // stages its 128 rows of A and its 64-row half of the B tile, a quarter less per SM than two 128 x 128 tiles, which
-// is what bounds one-wave problems once the issuing threads are out of the way); whole tiles only (KC = 1).
+// is what bounds one-wave problems once the issuing threads are out of the way); whole tiles, or two k-slices on the
+// two pairs of a four-CTA cluster (each CTA exchanges its partial sums with the CTA of the same position in the other pair).
 template <int BN, typename TOut, int KC, bool IN8, int CG = 1>
 __global__ void __launch_bounds__((ClusterKCfg<BN, KC, CG>::THREADS), 1)
 umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -107,8 +108,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // free first (cluster barrier after the main loop); the receiver's mbarrier counts the bytes and the senders
     // are told when their staging may go away (256x4096x4096: 17.0 us with per-thread remote stores between two
     // cluster barriers, 16.4 this way).
-    const int live_warps = min(4, (p.M - m0 + 31) / 32);
-    const bool direct = KC > 1 && live_warps == 1 && !p.bulk_exchange;
+    const int live_warps = max(0, min(4, (p.M - m0 + 31) / 32));  // (the second CTA of a pair may lie wholly beyond M)
+    const bool direct = CG == 1 && KC > 1 && live_warps == 1 && !p.bulk_exchange;  // (pairs: every CTA of a cluster must agree)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -145,7 +146,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     ptx::grid_launch_dependents();
 
     bool ok = true;
-    if (KC > 1 && !direct && threadIdx.x == 0) {
+    if (KC > 1 && !direct && live_warps > 0 && threadIdx.x == 0) {
         // what the peers will send: from each of them, for every 32-row block of the tile that exists, one 4 KiB
         // piece per 32-column chunk of this CTA's slice
         ptx::mbar_arrive_expect_tx(recvbar, (uint32_t)((KC - 1) * K_::CHUNKS * live_warps * 4096));
@@ -267,7 +268,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
 
     if (KC > 1) {
-        ptx::cluster_wait();              // the peers' barriers exist (they arrived long ago)
+        if (CG == 1) ptx::cluster_wait(); // the peers' barriers exist (they arrived long ago; pairs waited at the start)
         if (!direct) ptx::cluster_sync(); // every CTA's main loop is over (or has given up): every ring may be overwritten
     }
 
@@ -306,7 +307,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (m0 + trow < p.M) {
                         const int slot = ord_there * K_::CHUNKS + c;
                         const uint32_t local = epi_base + (uint32_t)((slot < 4 ? slot : slot + 2) * 4096 + lane * 128);
-                        const uint32_t remote = ptx::map_to_cta(local, d);
+                        const uint32_t remote = ptx::map_to_cta(local, d * CG + rank);
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             ptx::st_cluster_v4(remote + (uint32_t)((j ^ (lane & 7)) * 16), r[4 * j], r[4 * j + 1], r[4 * j + 2],
@@ -336,13 +337,13 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the bulk copy
             __syncwarp();
             if (lane == 0) {
-                const uint32_t bar_there = ptx::map_to_cta(recvbar, d);
+                const uint32_t bar_there = ptx::map_to_cta(recvbar, d * CG + rank);
 #pragma unroll 1
                 for (int c = 0; c < K_::CHUNKS; ++c) {
                     const uint32_t src = stage_base + (uint32_t)K_::AREA_BYTES +
                                          (uint32_t)((((dd - 1) * K_::CHUNKS + c) * BM + q * 32) * 128);
                     const uint32_t dst = stage_base + (uint32_t)(((ord_there * K_::CHUNKS + c) * BM + q * 32) * 128);
-                    ptx::bulk_copy_to_cluster(ptx::map_to_cta(dst, d), src, 4096u, bar_there);
+                    ptx::bulk_copy_to_cluster(ptx::map_to_cta(dst, d * CG + rank), src, 4096u, bar_there);
                 }
             }
         }
@@ -354,7 +355,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             exchange_ok = false;
         } else if (!direct && q == 0 && lane == 0) {
             // everything the peers sent has been written here, so their send areas are no longer read: tell them
-            for (int dd = 1; dd < KC; ++dd) ptx::mbar_arrive_cluster(ptx::map_to_cta(ackbar, (me + (uint32_t)dd) % KC));
+            for (int dd = 1; dd < KC; ++dd)
+                ptx::mbar_arrive_cluster(ptx::map_to_cta(ackbar, ((me + (uint32_t)dd) % KC) * CG + rank));
         }
     }
 
@@ -423,7 +425,9 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // ---------------------------------------------------------------------- teardown
     if (KC > 1 && !direct && warp >= 2 && warp < K_::PRODUCER2 && (warp & 3) == 0 && lane == 0) {
         // this CTA's send area must outlive the bulk copies that read it: every peer has acknowledged receipt
-        if (ok && exchange_ok && !ptx::mbar_wait<true>(ackbar, 0u, abort_flag, p.wait_cycles)) report_timeout(p, abort_flag, 8, 0);
+        // (a CTA whose rows all lie beyond M sent nothing and is owed nothing)
+        if (ok && exchange_ok && m0 < p.M && !ptx::mbar_wait<true>(ackbar, 0u, abort_flag, p.wait_cycles))
+            report_timeout(p, abort_flag, 8, 0);
     }
     __syncwarp();
     if (*abort_flag != 0) {

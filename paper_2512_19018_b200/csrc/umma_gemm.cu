@@ -592,6 +592,16 @@ int run_clusterk(const GemmArgs &g, const Plan &plan) {
         return PEAK_ERR_INVALID_VALUE;
     }
     if (plan.tail_splits == 1) return launch_clusterk_typed<128, 1>(g, plan);
+    if (plan.tail_splits == 2 && plan.bn == 128 && pair_tiles_apply(g) && !is_fp8(in_elem(g.dtype))) {
+        // two k-slices of 256 x 128 pair tiles on the two pairs of a four-CTA cluster
+        switch (out_elem(g.dtype)) {
+            case Elem::F32: return launch_clusterk<128, float, 2, false, 2>(g, plan);
+            case Elem::F16: return launch_clusterk<128, __half, 2, false, 2>(g, plan);
+            case Elem::BF16: return launch_clusterk<128, __nv_bfloat16, 2, false, 2>(g, plan);
+            default: break;
+        }
+        return PEAK_ERR_INVALID_VALUE;
+    }
     if (plan.bn == 128)
         return plan.tail_splits == 2 ? launch_clusterk_typed<128, 2>(g, plan) : launch_clusterk_typed<128, 4>(g, plan);
     return plan.tail_splits == 2 ? launch_clusterk_typed<256, 2>(g, plan) : launch_clusterk_typed<256, 4>(g, plan);

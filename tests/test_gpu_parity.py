@@ -820,8 +820,9 @@ def test_one_tile_per_pair_kernel_exact(ta, tb, reset_tuning):
     """Whole tiles of a one-wave problem with at least two 128-row blocks run as 256 x 128 CTA-pair tiles (the pair's
     leader issues cta_group::2 MMAs from two threads into two accumulators; each CTA stages its rows of A and its
     half of the B tile).  Exact on integers in every layout for ragged M (a pair whose second CTA has no rows), N,
-    K, one k-block, odd counts, every output type, 8-bit inputs with B stored N x K, beta != 0; the same bits as
-    single-CTA tiles; chosen by the dispatcher from 32 k-blocks on."""
+    K, one k-block, odd counts, every output type, 8-bit inputs with B stored N x K, beta != 0, whole and in two
+    k-slices (the two pairs of a four-CTA cluster exchange their partial sums); the same bits as single-CTA tiles;
+    chosen by the dispatcher from 32 k-blocks on."""
     shapes = [(256, 1024, 64), (300, 1000, 136), (129, 520, 1544), (512, 4100, 520), (700, 1280, 2056)]
     for idx, (M, N, K) in enumerate(shapes):
         for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16, W.PEAK_E4M3_BF16):
@@ -833,21 +834,26 @@ def test_one_tile_per_pair_kernel_exact(ta, tb, reset_tuning):
             c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb,
                    pad_c=[0, 8, 3][idx % 3], case=idx)
             outs = []
-            for mode in (4, 3):
+            kblocks = (K + (127 if in8 else 63)) // (128 if in8 else 64)
+            for mode, split in ((4, 1), (3, 1), (4, 2), (3, 2)):
+                if split == 2 and kblocks < 2:
+                    continue
                 P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 128)
-                P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, 1)
+                P.peak_set_tuning(P.PEAK_TUNE_SPLIT_K, split)
                 P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, mode)
                 dc = R.DeviceCase(c)
                 dc.run(P.PEAK_VARIANT_UMMA_1CTA)
                 name = P.peak_last_kernel()
-                assert "umma_clusterk_kernel<128," in name and (", 2> " in name) == (mode == 4), name
+                # (two k-slices of pair tiles -- the two pairs of a four-CTA cluster -- exist for 16-bit inputs)
+                pair = mode == 4 and not (split == 2 and in8)
+                assert f"umma_clusterk_kernel<128," in name and f", {split}, " in name and (", 2> " in name) == pair, name
                 ref, _ = dc.oracle_full()
                 want = oracle.round_to(R.OT[c.out_type], ref)
                 got = dc.result()
                 got = got.view(np.uint32) if c.out_type == "f32" else got
-                assert np.array_equal(got, want), f"{c} cluster_k={mode}"
+                assert np.array_equal(got, want), f"{c} cluster_k={mode} split={split}"
                 outs.append(got.copy())
-            assert np.array_equal(outs[0], outs[1])
+            assert all(np.array_equal(outs[0], o) for o in outs[1:])
     for k in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(k, 0)
     c = mk(W.PEAK_BF16_BF16, ta, tb, 512, 4096, 2048, alpha=0.5, beta=2.0)
