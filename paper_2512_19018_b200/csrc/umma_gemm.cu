@@ -592,7 +592,9 @@ int run_clusterk(const GemmArgs &g, const Plan &plan) {
         return PEAK_ERR_INVALID_VALUE;
     }
     if (plan.tail_splits == 1) return launch_clusterk_typed<128, 1>(g, plan);
-    if (plan.tail_splits == 2 && plan.bn == 128 && pair_tiles_apply(g) && !is_fp8(in_elem(g.dtype))) {
+    // (... when all of the four-CTA clusters are resident at once: 33 on this device, like those of four k-slices)
+    if (plan.tail_splits == 2 && plan.bn == 128 && pair_tiles_apply(g) && !is_fp8(in_elem(g.dtype)) &&
+        ((g.M + 255) / 256) * ((g.N + 127) / 128) <= (int64_t)clusterk_max_clusters(128, 4)) {
         // two k-slices of 256 x 128 pair tiles on the two pairs of a four-CTA cluster
         switch (out_elem(g.dtype)) {
             case Elem::F32: return launch_clusterk<128, float, 2, false, 2>(g, plan);
