@@ -314,7 +314,7 @@ typedef enum peak_tuning_key {
                                    a cluster and are added through distributed shared memory, one launch; one-wave problems
                                    of whole 128-wide tiles run the same one-tile-per-CTA kernel); 2 = as default, but
                                    the slices always travel by bulk copies (default: plain remote stores for tiles of
-                                   at most 32 rows); 3 = whole tiles never as 256 x 128 CTA-pair tiles; 4 = as pair tiles
+                                   at most 32 rows); 3 = whole tiles never as CTA-pair tiles on the one-tile kernel (256 x 128, or one wave of 256 x 256); 4 = as pair tiles
                                    whenever possible (default: from 32 k-blocks on) */
     PEAK_TUNE_SHARE = 18,       /* single-GPU plug-in, 16-bit inputs: single-CTA tiles in clusters of CM x CN tiles that share
                                    their A / B tiles by multicast copies: 1 = never, 100 * w + 10 * CM + CN (w = 1: 128-wide

@@ -52,7 +52,8 @@ template <int BN, int KC, int CG = 1> struct ClusterKCfg {
     static constexpr int ISSUER2 = PRODUCER2 + 1;
     static constexpr int THREADS = 32 * (ISSUER2 + 1);
     static_assert(KC == 1 || KC == 2 || KC == 4, "cluster sizes");
-    static_assert(CG == 1 || (CG == 2 && KC <= 2 && BN == 128), "CTA pairs: 256 x 128 tiles, whole or in two k-slices");
+    static_assert(CG == 1 || (CG == 2 && KC <= 2 && BN == 128) || (CG == 2 && KC == 1 && BN == 256),
+                  "CTA pairs: 256 x 128 tiles, whole or in two k-slices; whole 256 x 256 tiles");
     static_assert(SW % 32 == 0 && SW >= 32, "a slice is a whole number of 32-column chunks");
     static_assert(RECV_BYTES <= C_::STAGES * C_::STAGE_BYTES, "the receive area lives in the stage ring");
     static_assert((DUAL ? 2 : 1) * BN <= TMEM_COLS, "accumulators fit the allocation");

@@ -609,6 +609,26 @@ int run_clusterk(const GemmArgs &g, const Plan &plan) {
     return plan.tail_splits == 2 ? launch_clusterk_typed<256, 2>(g, plan) : launch_clusterk_typed<256, 4>(g, plan);
 }
 
+// One wave of whole 256 x 256 pair tiles (at most one tile per CTA pair) on the one-tile kernel: two producer warps per
+// CTA and no persistent-loop bookkeeping (measured, us, against the persistent kernel / the multicast plug-in: 2048^3
+// 16.9 / 17.5 / 18.0, 1792^3 15.5 / 16.2, 1024x4096x1024 11.7 / 12.2 / 12.5; cuBLAS 16.5 / 12.9 / 11.4).  16-bit inputs.
+bool one_wave_pair_tiles_apply(const GemmArgs &g, int cta_group, const Plan &plan, int units) {
+    const int mode = tuning(PEAK_TUNE_CLUSTER_K);
+    if (mode == 1 || mode == 3 || cta_group != 2 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype))) return false;
+    const int forced = tuning(PEAK_TUNE_TILE_N);
+    if ((forced != 0 && forced != 256) || plan.bn != 256 || plan.tail_splits != 1) return false;
+    return tiles_of(g, 2, 256) <= units;
+}
+int run_one_wave_pair_tiles(const GemmArgs &g, const Plan &plan) {
+    switch (out_elem(g.dtype)) {
+        case Elem::F32: return launch_clusterk<256, float, 1, false, 2>(g, plan);
+        case Elem::F16: return launch_clusterk<256, __half, 1, false, 2>(g, plan);
+        case Elem::BF16: return launch_clusterk<256, __nv_bfloat16, 1, false, 2>(g, plan);
+        default: break;
+    }
+    return PEAK_ERR_INVALID_VALUE;
+}
+
 // ---- exchanged operands for very skinny problems (M <= 64) -----------------------------------------------
 // C^T = op(B)^T op(A)^T: N takes the role of the MMA's M (128-row tiles over N) and M that of its N (one 64-wide
 // tile), so the small operand costs 8 KiB of shared memory and a few hundred bytes of traffic per k-block
@@ -762,6 +782,10 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // 1108 (256-wide); +12 % at 5000x3000x2500; but with 16-bit output, where the exposed epilogue of the wide
     // tile is half as long, the wide tile wins (bf16 4096^3: 1231 against 1244-1249), and from 2.7e11 flop on
     // the plug-in loses 3-6 % (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
+    if (one_wave_pair_tiles_apply(g, cta_group, plan, units) && tuning(PEAK_TUNE_MULTICAST) != 2) {
+        const int rc = run_one_wave_pair_tiles(g, plan);
+        if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+    }
     // Narrower tiles on the 256- / 512-wide pair kernels (192 / 384 columns; B with k contiguous, whole tiles): taken
     // when a cycle estimate -- waves x k-blocks x the slower of the tensor pipe (2 cycles per column) and the operand
     // stream (56 bytes per clock per SM), plus the exposed epilogue of a two-half tile -- says they beat the plan

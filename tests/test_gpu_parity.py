@@ -868,6 +868,52 @@ def test_one_tile_per_pair_kernel_exact(ta, tb, reset_tuning):
     assert np.array_equal(first, dc.result())
 
 
+@pytest.mark.parametrize("ta,tb", LAYOUTS)
+def test_one_wave_of_256_wide_pair_tiles_exact(ta, tb, reset_tuning):
+    """At most one 256 x 256 tile per CTA pair: the one-tile kernel's pair form with a 256-wide tile (one issuer, two
+    producers per CTA, two groups of epilogue warps).  Exact on integers for ragged shapes, every output type,
+    beta != 0, the fused tail; the same bits as the persistent kernel (PEAK_TUNE_CLUSTER_K = 3); not used when the
+    tiles need more than one wave."""
+    from tests.test_gpu_fused import run_fused, check_fused, make_residual
+    rng = np.random.default_rng(53)
+    for idx, (M, N, K) in enumerate([(512, 768, 256), (700, 1000, 264), (130, 2000, 72), (1024, 1920, 1032)]):
+        for dtype in (W.PEAK_BF16_BF16, W.PEAK_F16_F32, W.PEAK_F16_F16):
+            pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+            c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=[0.0, 1.0, -2.0][idx % 3], pad_a=pa, pad_b=pb,
+                   pad_c=[0, 8, 3][idx % 3], case=idx)
+            outs = []
+            for mode in (0, 3):
+                P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, mode)
+                P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 256)
+                P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, 1)
+                dc = R.DeviceCase(c)
+                dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+                name = P.peak_last_kernel()
+                assert ("umma_clusterk_kernel<256," in name and ", 2> " in name) == (mode == 0), name
+                ref, _ = dc.oracle_full()
+                want = oracle.round_to(R.OT[c.out_type], ref)
+                got = dc.result()
+                got = got.view(np.uint32) if c.out_type == "f32" else got
+                assert np.array_equal(got, want), f"{c} cluster_k={mode}"
+                outs.append(got.copy())
+            assert np.array_equal(outs[0], outs[1])
+    for k in range(P.PEAK_TUNE_COUNT):
+        P.peak_set_tuning(k, 0)
+    c = W.GemmCase("one_wave_fused", W.PEAK_BF16_BF16, bool(ta), bool(tb), 520, 1100, 264, 0.5, 2.0, "uniform",
+                   pad_a=(-(520 if ta else 264)) % 8, pad_b=(-(264 if tb else 1100)) % 8)
+    bias = rng.standard_normal(c.N).astype(np.float32)
+    res = make_residual(c, rng, 2)
+    P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 256)
+    dc = run_fused(c, P.PEAK_VARIANT_UMMA_2CTA, bias, P.PEAK_ACT_GELU, res)
+    assert "umma_clusterk_kernel<256," in P.peak_last_kernel(), P.peak_last_kernel()
+    check_fused(dc, bias, P.PEAK_ACT_GELU, f"one wave of pair tiles, fused {c.layout}", res)
+    big = mk(W.PEAK_BF16_BF16, ta, tb, 2560, 2304, 128, dist="smallint")     # 90 tiles: more than one per pair
+    dc = R.DeviceCase(big)
+    P.peak_set_tuning(P.PEAK_TUNE_MULTICAST, 1)
+    dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+    assert "umma_gemm_kernel<2," in P.peak_last_kernel(), P.peak_last_kernel()
+
+
 def test_cluster_k_bounded_wait_reports_timeout(reset_tuning):
     """The stalled-stage hook in the cluster-split kernel: the CTA whose stage never fills gives up after its
     budget, still reaches both cluster barriers (its peers wait there, not on a flag), the status word reports the
