@@ -99,7 +99,8 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int tile = blockIdx.x / (KC * CG);
     int64_t tm, tn;
     tile_coord(tile, p.tiles_m, p.tiles_n, p.group, tm, tn);
-    const int m0 = (int)tm * (BM * CG) + (int)rank * BM, n0 = (int)tn * BN;
+    // (p.bn_eff < BN: narrower whole tiles of a pair, see UmmaParams; bn_eff = BN otherwise)
+    const int m0 = (int)tm * (BM * CG) + (int)rank * BM, n0 = (int)tn * p.bn_eff;
     const int kb0 = (int)me * p.kb_per_split;
     const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);  // the host guarantees kb0 < kb1
     // How the k-slices travel (KC > 1).  A tile with at most 32 rows: the one warp that owns them writes its few
@@ -162,7 +163,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int grp = (warp - 2) >> 2;
     const bool tma = p.tma_store != 0 && GW >= CC;
     const int c_first = n0 + (int)me * SW + grp * GW;
-    const int c_limit = min(p.N, c_first + GW);
+    const int c_limit = min(min(p.N, n0 + p.bn_eff), c_first + GW);
     // staging: two buffers per warp with one group, one per warp with two
     const uint32_t my_stage = epi_base + (uint32_t)(warp - 2) * (K_::GROUPS == 1 ? 2u : 1u) * EPI_BUF_BYTES;
     CFetch cf{K_::GROUPS == 1 ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
@@ -184,7 +185,7 @@ umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int h = is_a ? lane : lane - a_ops;
         const CUtensorMap *tmap = is_a ? &tmA : &tmB;
         const bool mn = is_a ? p.a_mn != 0 : p.b_mn != 0;
-        const int mn0 = (is_a ? m0 : n0 + (int)rank * C_::HROWS) + h * (mn ? MN_ELEMS : (is_a ? 0 : C_::B_BOX_ROWS));
+        const int mn0 = (is_a ? m0 : n0 + (int)rank * p.hrows_eff) + h * (mn ? MN_ELEMS : (is_a ? 0 : C_::B_BOX_ROWS));
         const uint32_t off = (is_a ? 0u : (uint32_t)A_STAGE_BYTES) +
                              (uint32_t)h * (mn ? (uint32_t)MN_ATOM : (uint32_t)(C_::B_BOX_ROWS * 128));
         uint32_t it = (uint32_t)pw;

@@ -431,19 +431,23 @@ template <int BN, typename TOut, int KC, bool IN8, int CG = 1> int launch_cluste
     const Elem ein = in_elem(g.dtype), eout = out_elem(g.dtype);
     const int a_mn = g.transA ? 1 : 0, b_mn = g.transB ? 0 : 1;
     if (IN8 && b_mn && C_::HROWS < MNE) return PEAK_ERR_UNSUPPORTED;
+    // narrower whole tiles of a pair (plan.bn_eff, e.g. 192 on the 256-wide instantiation): B with k contiguous only
+    const int bn_eff = plan.bn_eff > 0 ? plan.bn_eff : BN;
+    const int hrows_eff = bn_eff / CG;
+    if (bn_eff != BN && (CG != 2 || KC != 1 || b_mn || bn_eff % 64 || bn_eff > BN)) return PEAK_ERR_UNSUPPORTED;
     const bool short_a = CG == 1 && g.M < 128 && tuning(PEAK_TUNE_SHORT_A) != 1;
     const int a_rows = short_a ? (int)((g.M + 7) / 8 * 8) : 128;
     const int a_boxes = short_a ? (int)((g.M + MNE - 1) / MNE) : 128 / MNE;
     CUtensorMap tmA, tmB, tmC;
     bool ok = a_mn ? make_map(&tmA, ein, g.A, g.M, g.K, g.lda, MNE, BKE) : make_map(&tmA, ein, g.A, g.K, g.M, g.lda, BKE, a_rows);
     ok = ok && (b_mn ? make_map(&tmB, ein, g.B, g.N, g.K, g.ldb, MNE, BKE)
-                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, C_::B_BOX_ROWS));
+                     : make_map(&tmB, ein, g.B, g.K, g.N, g.ldb, BKE, bn_eff != BN ? hrows_eff : C_::B_BOX_ROWS));
     if (!ok) return PEAK_ERR_CUDA;
     UmmaParams p = {};
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.num_kb = (int)((g.K + BKE - 1) / BKE);
     p.tiles_m = (int)((g.M + BM * CG - 1) / (BM * CG));
-    p.tiles_n = (int)((g.N + BN - 1) / BN);
+    p.tiles_n = (int)((g.N + bn_eff - 1) / bn_eff);
     p.group = tuning(PEAK_TUNE_RASTER_GROUP) > 0 ? tuning(PEAK_TUNE_RASTER_GROUP) : 16;
     p.tiles_per_batch = p.tiles_m * p.tiles_n;
     p.full_tiles = 0;
@@ -453,12 +457,12 @@ template <int BN, typename TOut, int KC, bool IN8, int CG = 1> int launch_cluste
     p.a_mn = a_mn; p.b_mn = b_mn;
     p.a_boxes = a_boxes;
     p.stage_tx = CG == 1 ? (uint32_t)(C_::B_STAGE_BYTES + (a_mn ? a_boxes * MNE * 128 : a_rows * 128))
-                         : (uint32_t)(CG * C_::STAGE_BYTES);  // both CTAs' parts arrive at the leader's barrier
+                         : (uint32_t)(CG * (A_STAGE_BYTES + hrows_eff * 128));  // both CTAs' parts arrive at the leader's barrier
     p.bulk_exchange = tuning(PEAK_TUNE_CLUSTER_K) == 2 ? 1 : 0;
-    p.bn_eff = BN; p.slot_eff = BN; p.hrows_eff = BN;
+    p.bn_eff = bn_eff; p.slot_eff = bn_eff; p.hrows_eff = hrows_eff;
     const uint32_t fmt = (ein == Elem::BF16 || ein == Elem::E5M2) ? 1u : 0u;
     p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
+              ((uint32_t)(bn_eff >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.ldc = g.ldc;
     p.bias = g.bias; p.act = g.act;
@@ -500,6 +504,9 @@ template <int BN, typename TOut, int KC, bool IN8, int CG = 1> int launch_cluste
     note_kernel("umma_clusterk_kernel<%d, %s, %d, %d%s> grid=%d clusters=%d", BN,
                 sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"), KC, (int)IN8,
                 CG == 2 ? ", 2" : "", p.total_items, p.tiles_per_batch);
+    if (bn_eff != BN) note_kernel("umma_clusterk_kernel<%d, %s, %d, %d, 2> grid=%d clusters=%d width=%d", BN,
+                                  sizeof(TOut) == 4 ? "float" : (std::is_same<TOut, __half>::value ? "__half" : "__nv_bfloat16"),
+                                  KC, (int)IN8, p.total_items, p.tiles_per_batch, bn_eff);
     if (e != cudaSuccess) { set_cuda_error(e); return PEAK_ERR_CUDA; }
     return PEAK_OK;
 }
@@ -782,6 +789,21 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // 1108 (256-wide); +12 % at 5000x3000x2500; but with 16-bit output, where the exposed epilogue of the wide
     // tile is half as long, the wide tile wins (bf16 4096^3: 1231 against 1244-1249), and from 2.7e11 flop on
     // the plug-in loses 3-6 % (8192x8192x2048, 4096x8192x4096, 16384x4096x4096).
+    {
+        // ... 192 columns wide where that still is one wave (B with k contiguous): more pairs at work, an eighth fewer
+        // operand bytes per k-block and CTA
+        Plan p1 = plan;
+        const int forced = tuning(PEAK_TUNE_TILE_N);
+        const int64_t t192 = ((g.M + 255) / 256) * ((g.N + 191) / 192);
+        const bool can192 = cta_group == 2 && g.transB && g.nbatch() == 1 && !in8 && plan.tail_splits == 1 &&
+                            (plan.bn == 256 || forced == 192) && t192 <= units && tuning(PEAK_TUNE_CLUSTER_K) != 1 &&
+                            tuning(PEAK_TUNE_CLUSTER_K) != 3 && tuning(PEAK_TUNE_MULTICAST) != 2;
+        if (can192 && (forced == 192 || (forced == 0 && tuning(PEAK_TUNE_NARROW) != 1 && t192 > tiles_of(g, 2, 256)))) {
+            p1.bn = 256; p1.bn_eff = 192;
+            const int rc = run_one_wave_pair_tiles(g, p1);
+            if (rc != PEAK_ERR_UNSUPPORTED) return rc;
+        }
+    }
     if (one_wave_pair_tiles_apply(g, cta_group, plan, units) && tuning(PEAK_TUNE_MULTICAST) != 2) {
         const int rc = run_one_wave_pair_tiles(g, plan);
         if (rc != PEAK_ERR_UNSUPPORTED) return rc;

@@ -872,8 +872,9 @@ def test_one_tile_per_pair_kernel_exact(ta, tb, reset_tuning):
 def test_one_wave_of_256_wide_pair_tiles_exact(ta, tb, reset_tuning):
     """At most one 256 x 256 tile per CTA pair: the one-tile kernel's pair form with a 256-wide tile (one issuer, two
     producers per CTA, two groups of epilogue warps).  Exact on integers for ragged shapes, every output type,
-    beta != 0, the fused tail; the same bits as the persistent kernel (PEAK_TUNE_CLUSTER_K = 3); not used when the
-    tiles need more than one wave."""
+    beta != 0, the fused tail; the same bits as the persistent kernel (PEAK_TUNE_CLUSTER_K = 3) and on 192-column
+    tiles (B with k contiguous; chosen where they still make one wave); not used when the tiles need more than
+    one wave."""
     from tests.test_gpu_fused import run_fused, check_fused, make_residual
     rng = np.random.default_rng(53)
     for idx, (M, N, K) in enumerate([(512, 768, 256), (700, 1000, 264), (130, 2000, 72), (1024, 1920, 1032)]):
@@ -896,9 +897,25 @@ def test_one_wave_of_256_wide_pair_tiles_exact(ta, tb, reset_tuning):
                 got = got.view(np.uint32) if c.out_type == "f32" else got
                 assert np.array_equal(got, want), f"{c} cluster_k={mode}"
                 outs.append(got.copy())
+            if tb:   # B with k contiguous: the same kernel on 192-column tiles
+                P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, 0)
+                P.peak_set_tuning(P.PEAK_TUNE_TILE_N, 192)
+                dc = R.DeviceCase(c)
+                dc.run(P.PEAK_VARIANT_UMMA_2CTA)
+                name = P.peak_last_kernel()
+                assert "umma_clusterk_kernel<256," in name and "width=192" in name, name
+                got = dc.result()
+                got = got.view(np.uint32) if c.out_type == "f32" else got
+                assert np.array_equal(got, want), f"{c} width=192"
             assert np.array_equal(outs[0], outs[1])
     for k in range(P.PEAK_TUNE_COUNT):
         P.peak_set_tuning(k, 0)
+    if tb:
+        c = mk(W.PEAK_BF16_BF16, ta, tb, 768, 4096, 256, alpha=0.5, beta=2.0)      # 66 tiles of 192 against 48 of 256
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_AUTO)
+        assert "width=192" in P.peak_last_kernel(), P.peak_last_kernel()
+        R.check_full(dc, what=f"{c}")
     c = W.GemmCase("one_wave_fused", W.PEAK_BF16_BF16, bool(ta), bool(tb), 520, 1100, 264, 0.5, 2.0, "uniform",
                    pad_a=(-(520 if ta else 264)) % 8, pad_b=(-(264 if tb else 1100)) % 8)
     bias = rng.standard_normal(c.N).astype(np.float32)
