@@ -618,19 +618,23 @@ int run_clusterk(const GemmArgs &g, const Plan &plan) {
 
 // One wave of whole 256 x 256 pair tiles (at most one tile per CTA pair) on the one-tile kernel: two producer warps per
 // CTA and no persistent-loop bookkeeping (measured, us, against the persistent kernel / the multicast plug-in: 2048^3
-// 16.9 / 17.5 / 18.0, 1792^3 15.5 / 16.2, 1024x4096x1024 11.7 / 12.2 / 12.5; cuBLAS 16.5 / 12.9 / 11.4).  16-bit inputs.
+// 16.9 / 17.5 / 18.0, 1792^3 15.5 / 16.2, 1024x4096x1024 11.7 / 12.2 / 12.5; cuBLAS 16.5 / 12.9 / 11.4).
 bool one_wave_pair_tiles_apply(const GemmArgs &g, int cta_group, const Plan &plan, int units) {
     const int mode = tuning(PEAK_TUNE_CLUSTER_K);
-    if (mode == 1 || mode == 3 || cta_group != 2 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype))) return false;
+    if (mode == 1 || mode == 3 || cta_group != 2 || g.nbatch() > 1) return false;
     const int forced = tuning(PEAK_TUNE_TILE_N);
     if ((forced != 0 && forced != 256) || plan.bn != 256 || plan.tail_splits != 1) return false;
     return tiles_of(g, 2, 256) <= units;
 }
 int run_one_wave_pair_tiles(const GemmArgs &g, const Plan &plan) {
+    const bool in8 = is_fp8(in_elem(g.dtype));
     switch (out_elem(g.dtype)) {
-        case Elem::F32: return launch_clusterk<256, float, 1, false, 2>(g, plan);
+        case Elem::F32:
+            return in8 ? launch_clusterk<256, float, 1, true, 2>(g, plan) : launch_clusterk<256, float, 1, false, 2>(g, plan);
         case Elem::F16: return launch_clusterk<256, __half, 1, false, 2>(g, plan);
-        case Elem::BF16: return launch_clusterk<256, __nv_bfloat16, 1, false, 2>(g, plan);
+        case Elem::BF16:
+            return in8 ? launch_clusterk<256, __nv_bfloat16, 1, true, 2>(g, plan)
+                       : launch_clusterk<256, __nv_bfloat16, 1, false, 2>(g, plan);
         default: break;
     }
     return PEAK_ERR_INVALID_VALUE;
