@@ -31,6 +31,8 @@ def whole_matrix_check(dc: R.DeviceCase, max_flops=2.5e12):
     def absolute(t):
         if t.dtype == torch.float32:
             return t.abs()
+        if t.element_size() == 1:                       # 8-bit floats: the sign is the top bit of every byte
+            return (t.view(torch.uint8) & 0x7F).view(t.dtype)
         return (t.view(torch.int16) & 0x7FFF).view(t.dtype)
     S = torch.empty((c.M, c.N), dtype=torch.float64, device="cuda")
     P.peak_gemm_xcheck_f64(c.dtype, c.transA, c.transB, c.M, c.N, c.K, 1.0, absolute(dc.A), c.lda, absolute(dc.B), c.ldb,
