@@ -186,6 +186,13 @@ def test_bench_traffic_is_read_from_the_profile_of_the_launched_kernel():
     assert t is None and "differs" in src
     t, src = bench.profile_traffic("no_such_workload", "x_kernel<1>")
     assert t is None and "no ncu summary" in src
+    # the two skinny benchmark shapes: the summary of the one-tile-per-CTA kernel, not the older one beside it
+    t, src = bench.profile_traffic("bf16_128x14336x4096_tn", "umma_clusterk_kernel<128, __nv_bfloat16, 1, 0> grid=112 clusters=112")
+    assert t is not None and 1.2e8 < t < 1.4e8 and "umma_clusterk" in src
+    t, src = bench.profile_traffic("bf16_16x4096x4096_tn", "umma_clusterk_kernel<128, __nv_bfloat16, 4, 0> grid=128 clusters=32")
+    assert t is not None and 3.3e7 < t < 3.6e7
+    t, src = bench.profile_traffic("bf16_128x14336x4096_tn", "umma_clusterk_kernel<128, __nv_bfloat16, 1, 0, 2> grid=112")
+    assert t is None                                        # the pair form is another kernel
 
 
 def test_bench_rotation_rule():
