@@ -59,10 +59,12 @@ template <int BN, int KC, int CG = 1> struct ClusterKCfg {
     static_assert((DUAL ? 2 : 1) * BN <= TMEM_COLS, "accumulators fit the allocation");
 };
 
-// CG = 2: the tile is 256 x 128, computed by a CTA pair (cta_group::2 MMAs issued by the pair's leader; each CTA
-// stages its 128 rows of A and its 64-row half of the B tile, a quarter less per SM than two 128 x 128 tiles, which
-// is what bounds one-wave problems once the issuing threads are out of the way); whole tiles, or two k-slices on the
-// two pairs of a four-CTA cluster (each CTA exchanges its partial sums with the CTA of the same position in the other pair).
+// CG = 2: the tile is 256 x BN, computed by a CTA pair (cta_group::2 MMAs issued by the pair's leader; each CTA stages
+// its 128 rows of A and its half of the B tile).  BN = 128: a quarter less per SM than two 128 x 128 tiles, which is
+// what bounds one-wave problems once the issuing threads are out of the way; whole tiles, or two k-slices on the two
+// pairs of a four-CTA cluster (each CTA exchanges its partial sums with the CTA of the same position in the other
+// pair).  BN = 256: whole tiles of a problem with at most one tile per pair (one issuer), also p.bn_eff = 192 columns
+// wide when B is stored with k contiguous.
 template <int BN, typename TOut, int KC, bool IN8, int CG = 1>
 __global__ void __launch_bounds__((ClusterKCfg<BN, KC, CG>::THREADS), 1)
 umma_clusterk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
