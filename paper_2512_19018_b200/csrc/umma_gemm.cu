@@ -94,6 +94,12 @@ Plan choose_plan(const GemmArgs &g, int cg, int units) {
             }
             return Plan{128, (int)t128, 1};
         }
+        // Fewer tiles than an eighth of the SMs: four slices in a cluster beat both whole tiles and the two-launch
+        // split with a workspace while a slice stays short -- measured (NT, us; whole tiles / workspace split /
+        // four slices): 256x256x2048 9.4 / - / 7.2, 128x512x4096 13.8 / 12.0 / 8.6, 512x512x8192 26.8 / 15.1 / 13.5;
+        // from 256 k-blocks the sixteen-way workspace split wins (512x512x16384: 19.5 against 21.6).
+        if (t128 * 8 <= units && num_kb >= 16 && num_kb <= 160 && t128 <= clusterk_max_clusters(128, 4))
+            return Plan{128, 0, 4};
     }
     for (int bn : {512, 256, 128}) {
         if (force_bn ? bn != force_bn : bn == 512) continue;  // 512-wide tiles only on request (see launch_umma)

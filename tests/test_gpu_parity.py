@@ -770,6 +770,19 @@ def test_cluster_k_real_values_fused_tail_and_selection(reset_tuning):
     dc.run(P.PEAK_VARIANT_AUTO)
     assert "umma_gemm_kernel<1," in P.peak_last_kernel()
     R.check_full(dc, what=c.name)
+    # fewer tiles than an eighth of the SMs: four slices in a cluster from 16 to 160 k-blocks (exact on integers,
+    # ragged edges included), the workspace split beyond
+    P.peak_set_tuning(P.PEAK_TUNE_CLUSTER_K, 0)
+    for idx, (ta, tb, M, N, K, four) in enumerate([(0, 1, 256, 512, 4096, True), (0, 0, 250, 300, 1032, True),
+                                                   (1, 1, 16, 1000, 10240, True), (0, 1, 128, 256, 16384, False)]):
+        pa, pb = (-(M if ta else K)) % 8, (-(K if tb else N)) % 8
+        c = mk(W.PEAK_BF16_BF16 if idx % 2 == 0 else W.PEAK_F16_F32, ta, tb, M, N, K, dist="smallint", alpha=0.5,
+               beta=[0.0, 1.0][idx % 2], pad_a=pa, pad_b=pb, pad_c=idx, case=idx)
+        dc = R.DeviceCase(c)
+        dc.run(P.PEAK_VARIANT_AUTO)
+        name = P.peak_last_kernel()
+        assert ("umma_clusterk_kernel<128," in name and ", 4, 0>" in name) == four, name
+        R.check_full(dc, what=f"few tiles {c}")
 
 
 def test_one_tile_per_cta_kernel_two_issuers_exact(reset_tuning):
