@@ -80,6 +80,8 @@ def workloads_table():
     for i in range(3):
         t[W.config3(i).name] = W.config3(i)
         t[W.config4_ragged(i).name] = W.config4_ragged(i)
+    for k in (128, 512):
+        t[W.short_k_workload(k).name] = W.short_k_workload(k)
     return t
 
 

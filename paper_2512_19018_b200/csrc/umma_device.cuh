@@ -313,7 +313,8 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
         const int col0 = cbase + c * CHUNK_COLS;
         if (col0 >= ncols) break;  // warp-uniform
-        const uint32_t buf = my_stage + ((cf.on && !cf.single) ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
+        // a warp with two staging buffers alternates between them (with and without prefetched old C)
+        const uint32_t buf = my_stage + (!cf.single ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
         // the whole chunk is requested from tensor memory before the first wait
         uint32_t r[CHUNK_COLS / 32][32];
 #pragma unroll
@@ -395,9 +396,13 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
             }
             if (tma) {
                 if (h == 0 && !cf.on) {
-                    // the store of the previous chunk must have read the staging buffer; it had the time of
-                    // this chunk's tensor-memory load and arithmetic to do so
-                    if (lane == 0) ptx::tma_store_wait_read<0>();
+                    // the last store out of this staging buffer must have read it: with one buffer that is the
+                    // previous chunk's, with two the one before (a tile starts with every store read, so that an odd
+                    // number of chunks in the previous tile cannot leave this buffer busy)
+                    if (lane == 0) {
+                        if (cf.single || c == 0) ptx::tma_store_wait_read<0>();
+                        else ptx::tma_store_wait_read<1>();
+                    }
                     __syncwarp();
                 }
                 stage_row32<T>(buf, lane, h, v);  // with prefetched C: in place, over this thread's own row
@@ -768,7 +773,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const bool vec = p.vec_ok != 0;
         CFetch cf{ONE_GROUP ? cbar0 + 16u * (uint32_t)(warp - 2) : cbar0 + 8u * (uint32_t)(warp - 2), 0u,
                   p.c_prefetch != 0, !ONE_GROUP};
-        CFetch no_cf{0u, 0u, false, false};
+        CFetch no_cf{0u, 0u, false, !ONE_GROUP};
         uint32_t tl = 0;
         bool ok = true;
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {

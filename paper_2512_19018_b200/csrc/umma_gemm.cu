@@ -311,6 +311,8 @@ template <int BN> bool want_two_groups(const GemmArgs &g, const Plan &plan, int 
     if (BN == 512 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype))) return false;
     const int mode = tuning(PEAK_TUNE_EPILOGUE_WARPS);  // 1 = four warps, 2 = eight warps
     if (mode) return mode == 2;
+    // (also up to eight k-blocks, where the epilogue bounds every tile: 8192x8192x512 70 -> 64 us)
+    if (plan.tail_splits == 1 && (g.K + BK - 1) / BK <= 8) return true;
     return plan.tail_splits == 1 && (int64_t)plan.full_tiles <= 2 * (int64_t)units;
 }
 
@@ -778,7 +780,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // k-blocks take the same time but hold twice the K, from 96 k-blocks (K = 12288) on (a tie at 64 k-blocks,
     // +2.6 % at 96, +3..5 % at 128).  They must fill the grid as well as the 256-wide tiles do (4096x8192x4096: 3.46 waves
     // against 6.9, -3 %).
-    bool wide = false;
+    bool wide = false, short_k = false;
     if (whole256 && !tuning(PEAK_TUNE_TILE_N)) {
         const int bke = in8 ? 2 * BK : BK;
         const int64_t num_kb = (g.K + bke - 1) / bke;
@@ -793,6 +795,13 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         if (!wide && light_tail && !in8 && elem_bytes(out_elem(g.dtype)) == 2 && num_kb >= 32 && t512 <= units &&
             t256 > units && t512 * 10 >= (int64_t)units * 6)
             wide = true;
+        // Up to four k-blocks the epilogue, not the main loop, bounds a tile, and the wide tile's eight epilogue warps
+        // drain it faster than four (8192x8192x64: 58 -> 41 us, 8192x8192x256: 61 -> 53, 4096x4096x128: 20 -> 15.5);
+        // the multicast plug-in has nothing to share there.
+        // (taken where the wide tiles waste no more columns than the 256-wide ones: 128 matrices of 256 x 256 x 128
+        // ran 13.6 us on 256-wide tiles and 15.3 on half-empty wide ones)
+        if (!wide && num_kb <= 4 && t256 > units && t512 * 16 <= t256 * 9) wide = true;
+        if (num_kb <= 8) short_k = true;
     }
     // Whole 256-wide pair tiles, at least two pairs tall: the multicast plug-in can run it, if it is there.
     // Measured (sustained, random inputs, interleaved): fp16 4096^3 -> fp32 1162 against 1132 (512-wide) and
@@ -838,7 +847,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
         };
         int narrow = 0;
         if (forced == 192 || forced == 384) narrow = forced;
-        else if (forced == 0 && tuning(PEAK_TUNE_NARROW) != 1 && g.M > 128) {
+        else if (forced == 0 && tuning(PEAK_TUNE_NARROW) != 1 && g.M > 128 && !short_k) {  // (the estimate knows no epilogue-bound tiles)
             const double now = estimate(wide ? 512 : plan.bn);
             const double e192 = estimate(192), e384 = estimate(384);
             if (plan.bn >= 256 && e192 < 0.85 * now && e192 <= e384) narrow = 192;
@@ -857,7 +866,7 @@ int launch_umma(const GemmArgs &g, int cta_group) {
     // (8-bit inputs, 256-wide tiles only: 2048^3 1295 -> 1415, 4096^3 unchanged, larger problems excluded as above)
     const bool wide_first = wide && elem_bytes(out_elem(g.dtype)) == 2;
     const bool whole512 = cta_group == 2 && plan.bn == 512 && plan.tail_splits == 1 && mc_mode == 2;  // forced
-    if ((whole256 || whole512) && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && mc_entry()) {
+    if ((whole256 || whole512) && mc_mode != 1 && g.M > 256 && g.nbatch() == 1 && (!short_k || mc_mode == 2) && mc_entry()) {
         const int mc_tile_n = ((whole512 || wide_first) && !in8) ? 512 : 256;
         const int64_t super_tiles = ((g.M + 511) / 512) * ((g.N + mc_tile_n - 1) / mc_tile_n);
         const double flops = 2.0 * (double)g.M * (double)g.N * (double)g.K;

@@ -250,6 +250,12 @@ def config4_ragged(which: int) -> GemmCase:
                     case=100 + which)
 
 
+def short_k_workload(k: int = 128) -> GemmCase:
+    """bf16 8192 x 8192 x k NT with a short k (a rank-k update): the output, not the operands, bounds the launch."""
+    return GemmCase(f"bf16_8192x8192x{k}_nt", PEAK_BF16_BF16, False, True, 8192, 8192, k, 1.0, 0.0, "uniform", config=4,
+                    case=200 + k // 64)
+
+
 def bench_workload() -> GemmCase:
     """The configuration the headline throughput is quoted on."""
     return config1()
