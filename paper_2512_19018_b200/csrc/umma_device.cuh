@@ -274,6 +274,21 @@ __device__ __forceinline__ void cfetch_issue(const CFetch &cf, uint32_t my_stage
     else ptx::tma_load_2d(dst, tm, x0 + c * CHUNK_COLS, y0, bar);
 }
 
+// tile_coord() in 32-bit arithmetic for the kernels (the host checks that tile counts fit): the 64-bit divisions of the
+// general form cost a lone thread about 2700 cycles per tile, which sat between the epilogues of consecutive tiles.
+__device__ __forceinline__ void tile_coord32(int tile, int tiles_m, int tiles_n, int group, int &tm, int &tn) {
+    const uint32_t grp = (uint32_t)(group < 1 ? 1 : (group > tiles_m ? tiles_m : group));
+    const uint32_t per_group = grp * (uint32_t)tiles_n;
+    const uint32_t g = (uint32_t)tile / per_group;
+    const uint32_t first_m = g * grp;
+    const uint32_t left = (uint32_t)tiles_m - first_m;
+    const uint32_t rows = left < grp ? left : grp;
+    const uint32_t r = (uint32_t)tile - g * per_group;
+    const uint32_t q = r / rows;
+    tn = (int)q;
+    tm = (int)(first_m + (r - q * rows));
+}
+
 // Work item -> tile, k-block range and destination (ws_block < 0: the tile is whole and goes to C;
 // otherwise the index of the (tile, slice) block of the partial-tile workspace).
 struct Item {
@@ -309,6 +324,47 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                                               volatile uint32_t *abort_flag, long long wait_cycles,
                                               uint32_t t_addr2 = 0u) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
+    if (tma && !cf.on && beta == 0.0f && bias == nullptr && act == 0 && rbase == nullptr && (!ACC2 || t_addr2 == 0u)) {
+        // Plain C = alpha * acc through TMA stores, the case that bounds problems with few k-blocks: a loop of its own,
+        // small enough to stay in the instruction cache, in which the tensor-memory load of the next chunk is in
+        // flight while the current one is fenced and stored.
+        constexpr int H = CHUNK_COLS / 32;
+        const int left = ncols - cbase;
+        const int nchunks = left <= 0 ? 0 : min(BN / CHUNK_COLS, (left + CHUNK_COLS - 1) / CHUNK_COLS);
+        if (nchunks == 0) return true;
+        uint32_t r[H][32];
+#pragma unroll
+        for (int h = 0; h < H; ++h) ptx::tmem_ld_32x32(t_addr + h * 32, r[h]);
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c) {
+            const uint32_t buf = my_stage + (!cf.single ? (uint32_t)(c & 1) * EPI_BUF_BYTES : 0u);
+            if (lane == 0) {  // the last store out of this buffer has read it (see below for c == 0)
+                if (cf.single || c == 0) ptx::tma_store_wait_read<0>();
+                else ptx::tma_store_wait_read<1>();
+            }
+            ptx::tmem_ld_wait();
+            __syncwarp();
+#pragma unroll
+            for (int h = 0; h < H; ++h) {
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[h][i]);
+                stage_row32<T>(buf, lane, h, v);
+            }
+            if (c + 1 < nchunks) {
+#pragma unroll
+                for (int h = 0; h < H; ++h) ptx::tmem_ld_32x32(t_addr + (c + 1) * CHUNK_COLS + h * 32, r[h]);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && row0 < nrows) {
+                if (MAP3D) ptx::tma_store_3d(tm, x0 + c * CHUNK_COLS, y0, z0, buf);
+                else ptx::tma_store_2d(tm, x0 + c * CHUNK_COLS, y0, buf);
+                ptx::tma_store_commit();
+            }
+        }
+        return true;
+    }
 #pragma unroll 1
     for (int c = 0; c < BN / CHUNK_COLS; ++c) {
         const int col0 = cbase + c * CHUNK_COLS;
@@ -585,8 +641,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 // with it, but it is a fixed function of the launch, so results stay run-to-run identical.
                 const bool rev = p.k_alternate && (tl & 1u);
                 const int bz = BATCHED ? w.tile / p.tiles_per_batch : 0;  // matrix of the batch
-                int64_t tm, tn;
-                tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
+                int tm, tn;
+                tile_coord32(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
                 const int m_cta = (int)tm * (BM * CLUSTER) + (int)crank * BM;
                 const int n_cta = (int)tn * p.bn_eff + (int)rank * p.hrows_eff;  // first B row of this CTA (half 0)
                 for (int j = 0, nk = w.kb1 - w.kb0; j < nk; ++j, ++it) {
@@ -779,8 +835,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int item = unit; item < total_items && ok; item += num_units, ++tl) {
             const Item w = decode_item(p, item);
             const int bz = BATCHED ? w.tile / p.tiles_per_batch : 0;
-            int64_t tm, tn;
-            tile_coord(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
+            int tm, tn;
+            tile_coord32(w.tile - bz * p.tiles_per_batch, p.tiles_m, p.tiles_n, p.group, tm, tn);
             const int row0 = (int)tm * (BM * CLUSTER) + (int)crank * BM + q * 32;  // first row of this warp
             const int n0 = (int)tn * p.bn_eff;
             const bool live = row0 < p.M;  // none of this warp's 32 rows exists otherwise: nothing to drain
@@ -899,8 +955,8 @@ splitk_reduce_kernel(const float *__restrict__ ws, int splits, int full_tiles, i
     const int gt = full_tiles + t;           // tile number over the whole batch
     const int bz = gt / tiles_per_batch;
     C += (int64_t)bz * stride_c;
-    int64_t tm, tn;
-    tile_coord(gt - bz * tiles_per_batch, tiles_m, tiles_n, group, tm, tn);
+    int tm, tn;
+    tile_coord32(gt - bz * tiles_per_batch, tiles_m, tiles_n, group, tm, tn);
     const int vec_per_row = bn / 4;
     const int64_t rows_left = (int64_t)M - tm * rows_t;  // rows of this tile that exist
     const int total_vec = (int)(rows_left < rows_t ? rows_left : rows_t) * vec_per_row;
