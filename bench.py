@@ -53,7 +53,7 @@ OTHER_WORKLOADS = [
     "bf16_4096_nn",
     "fp16_2048_nn", "fp16_2048_tn", "fp16_4096_nn", "fp16_4096_tn", "fp16_8192_nn", "fp16_8192_tn",
     "bf16_tfm_16384x4096x4096_nt", "bf16_tfm_16384x14336x4096_nt", "bf16_tfm_16384x4096x14336_nt",
-    "bf16_5000x3000x2500_tn", "bf16_16x4096x4096_tn", "bf16_128x14336x4096_tn",
+    "bf16_5000x3000x2500_tn", "bf16_16x4096x4096_tn", "bf16_128x14336x4096_tn", "bf16_8192x8192x128_nt",
     "fp32_4096_nn", "fp32_8192_nn",
     "e4m3_8192_nt", "e4m3_8192_nn",
 ]
