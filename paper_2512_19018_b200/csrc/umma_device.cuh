@@ -324,7 +324,7 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                                               volatile uint32_t *abort_flag, long long wait_cycles,
                                               uint32_t t_addr2 = 0u) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
-    if (tma && !cf.on && beta == 0.0f && bias == nullptr && act == 0 && rbase == nullptr && (!ACC2 || t_addr2 == 0u)) {
+    if (tma && !cf.on && beta == 0.0f && bias == nullptr && act == 0 && rbase == nullptr) {
         // Plain C = alpha * acc through TMA stores, the case that bounds problems with few k-blocks: a loop of its own,
         // small enough to stay in the instruction cache, in which the tensor-memory load of the next chunk is in
         // flight while the current one is fenced and stored.
@@ -343,6 +343,18 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                 else ptx::tma_store_wait_read<1>();
             }
             ptx::tmem_ld_wait();
+            if constexpr (ACC2) {
+                if (t_addr2 != 0u) {  // the sums of the second MMA issuer
+#pragma unroll
+                    for (int h = 0; h < H; ++h) {
+                        uint32_t r2[32];
+                        ptx::tmem_ld_32x32(t_addr2 + c * CHUNK_COLS + h * 32, r2);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[h][i] = __float_as_uint(__uint_as_float(r[h][i]) + __uint_as_float(r2[i]));
+                    }
+                }
+            }
             __syncwarp();
 #pragma unroll
             for (int h = 0; h < H; ++h) {
