@@ -309,6 +309,12 @@ __device__ __forceinline__ Item decode_item(const UmmaParams &p, int item) {
     return w;
 }
 
+// The case the plain-store loop of epilogue_tile() handles: C = alpha * acc, TMA stores, nothing fused, no old C.
+__device__ __forceinline__ bool plain_store_case(bool tma, bool c_prefetch, float beta, const float *bias, int act,
+                                                 const void *rbase) {
+    return tma && !c_prefetch && beta == 0.0f && bias == nullptr && act == 0 && rbase == nullptr;
+}
+
 // Epilogue of one accumulator tile for one warp: TMEM -> registers -> alpha/beta -> T -> staging + TMA
 // store (or direct stores).  `cbase` is the column of chunk 0 used for bounds and addressing, `ncols` the
 // column limit, `nrows` the row limit for `row`; (x0, y0[, z0]) is where chunk 0 of this warp lands in `tm`
@@ -322,16 +328,28 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                                               bool vec, float alpha, float beta, const float *bias, int act,
                                               const T *rbase, int64_t ldr, bool rvec, CFetch &cf,
                                               volatile uint32_t *abort_flag, long long wait_cycles,
-                                              uint32_t t_addr2 = 0u) {
+                                              uint32_t t_addr2 = 0u, uint32_t release_bar = 0u,
+                                              bool release_remote = false) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
-    if (tma && !cf.on && beta == 0.0f && bias == nullptr && act == 0 && rbase == nullptr) {
+    if (plain_store_case(tma, cf.on, beta, bias, act, rbase)) {
         // Plain C = alpha * acc through TMA stores, the case that bounds problems with few k-blocks: a loop of its own,
         // small enough to stay in the instruction cache, in which the tensor-memory load of the next chunk is in
         // flight while the current one is fenced and stored.
         constexpr int H = CHUNK_COLS / 32;
         const int left = ncols - cbase;
         const int nchunks = left <= 0 ? 0 : min(BN / CHUNK_COLS, (left + CHUNK_COLS - 1) / CHUNK_COLS);
-        if (nchunks == 0) return true;
+        // `release_bar` (plain-store case only): the accumulator is handed back to the MMA issuer as soon as its last
+        // chunk is in registers, so that the next tile's MMAs run under this tile's last stores
+        auto release = [&]() {
+            if (release_bar == 0u) return;
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                if (release_remote) ptx::mbar_arrive_cluster(release_bar);
+                else ptx::mbar_arrive(release_bar);
+            }
+        };
+        if (nchunks == 0) { release(); return true; }
         uint32_t r[H][32];
 #pragma unroll
         for (int h = 0; h < H; ++h) ptx::tmem_ld_32x32(t_addr + h * 32, r[h]);
@@ -355,6 +373,7 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                     }
                 }
             }
+            if (c + 1 == nchunks) release();
             __syncwarp();
 #pragma unroll
             for (int h = 0; h < H; ++h) {
@@ -895,6 +914,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                         (SPLIT_COLS ? (uint32_t)(grp * W) : 0u);
                 const int nh = n0 + cn;
                 const int n_end = min(p.N, n0 + ((C_::HALVES == 2) ? (hf + 1) * p.slot_eff : p.bn_eff));
+                bool released = false;  // the epilogue handed the accumulator back itself
                 if (!live) {
                     // rows beyond M: the partial-tile reduction and C never look at them
                 } else if (SWAP && w.ws_block < 0) {
@@ -906,10 +926,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // whole tile: alpha/beta epilogue straight to C
                     TOut *c_base = reinterpret_cast<TOut *>(p.C);
                     if (BATCHED) c_base += (int64_t)bz * p.stride_c;
+                    const uint32_t rel = CG == 1 ? accempty0 + 8 * b : ptx::map_to_cta(accempty0 + 8 * b, leader_crank);
+                    released = plain_store_case(p.tma_store != 0, cf.on, p.beta, p.bias, p.act, p.R);
                     if (!epilogue_tile<TOut, W, BATCHED>(t_addr, my_stage, lane, c_base, p.ldc, row0 + lane, row0, p.M,
                                                          nh, n_end, &tmC, nh, row0, bz, p.tma_store != 0, vec, p.alpha,
                                                          p.beta, p.bias, p.act, reinterpret_cast<const TOut *>(p.R),
-                                                         p.ldr, p.r_vec != 0, cf, abort_flag, p.wait_cycles)) {
+                                                         p.ldr, p.r_vec != 0, cf, abort_flag, p.wait_cycles, 0u,
+                                                         released ? rel : 0u, CG == 2)) {
                         if (lane == 0) report_timeout(p, abort_flag, 6, b);
                         ok = false;
                         break;
@@ -924,7 +947,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 // hand the accumulator slot back to the MMA issuer
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) {
+                if (lane == 0 && !released) {
                     if (CG == 1) ptx::mbar_arrive(accempty0 + 8 * b);
                     else ptx::mbar_arrive_cluster(ptx::map_to_cta(accempty0 + 8 * b, leader_crank));
                 }
