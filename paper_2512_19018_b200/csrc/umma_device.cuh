@@ -321,17 +321,18 @@ __device__ __forceinline__ bool plain_store_case(bool tma, bool c_prefetch, floa
 // (z0 is used when MAP3D says that `tm` is three-dimensional).
 // ACC2: the tile's sums are split over two accumulators (t_addr and, when nonzero, t_addr2: two MMA issuers that
 // took the k-blocks in turn); they are added as they are read.
-template <typename T, int BN, bool MAP3D = false, bool ACC2 = false>
-__device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage, int lane,
+// FUSED = false compiles the bias / activation / residual code out: the loop of a plain alpha / beta epilogue then is a
+// fraction of the size, which matters to a warp that walks it once per 64 columns.
+template <typename T, int BN, bool MAP3D, bool ACC2, bool FUSED>
+__device__ __forceinline__ bool epilogue_tile_impl(uint32_t t_addr, uint32_t my_stage, int lane,
                                               T *base, int64_t ld, int row, int row0, int nrows, int cbase,
                                               int ncols, const CUtensorMap *tm, int x0, int y0, int z0, bool tma,
                                               bool vec, float alpha, float beta, const float *bias, int act,
                                               const T *rbase, int64_t ldr, bool rvec, CFetch &cf,
                                               volatile uint32_t *abort_flag, long long wait_cycles,
-                                              uint32_t t_addr2 = 0u, uint32_t release_bar = 0u,
-                                              bool release_remote = false) {
+                                              uint32_t t_addr2, uint32_t release_bar, bool release_remote) {
     constexpr int CHUNK_COLS = 128 / (int)sizeof(T);  // columns per staged chunk: 32 (fp32) or 64 (16-bit)
-    if (plain_store_case(tma, cf.on, beta, bias, act, rbase)) {
+    if (!FUSED && plain_store_case(tma, cf.on, beta, bias, act, rbase)) {
         // Plain C = alpha * acc through TMA stores, the case that bounds problems with few k-blocks: a loop of its own,
         // small enough to stay in the instruction cache, in which the tensor-memory load of the next chunk is in
         // flight while the current one is fenced and stored.
@@ -454,7 +455,7 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = alpha * __uint_as_float(r[h][i]);
             }
-            if (bias != nullptr) {  // fused tail: every thread of the warp adds the same 32 bias values
+            if (FUSED && bias != nullptr) {  // fused tail: every thread of the warp adds the same 32 bias values
                 if (valid == 32 && (reinterpret_cast<uintptr_t>(bias + col) & 15u) == 0) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
@@ -467,14 +468,14 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
                         if (i < valid) v[i] += __ldg(bias + col + i);
                 }
             }
-            if (act == PEAK_ACT_RELU) {
+            if (FUSED && act == PEAK_ACT_RELU) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.0f);
-            } else if (act == PEAK_ACT_GELU) {
+            } else if (FUSED && act == PEAK_ACT_GELU) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = activate_f32(v[i], PEAK_ACT_GELU);
             }
-            if (rbase != nullptr && row < nrows && valid > 0) {
+            if (FUSED && rbase != nullptr && row < nrows && valid > 0) {
                 // residual: each thread reads its own row's contiguous run (the same access as old C without TMA)
                 float rr[32];
                 load_row32<T>(rbase + (int64_t)row * ldr + col, rr, valid, rvec);
@@ -510,6 +511,24 @@ __device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage
         }
     }
     return true;
+}
+
+template <typename T, int BN, bool MAP3D = false, bool ACC2 = false>
+__device__ __forceinline__ bool epilogue_tile(uint32_t t_addr, uint32_t my_stage, int lane, T *base, int64_t ld, int row,
+                                              int row0, int nrows, int cbase, int ncols, const CUtensorMap *tm, int x0,
+                                              int y0, int z0, bool tma, bool vec, float alpha, float beta,
+                                              const float *bias, int act, const T *rbase, int64_t ldr, bool rvec,
+                                              CFetch &cf, volatile uint32_t *abort_flag, long long wait_cycles,
+                                              uint32_t t_addr2 = 0u, uint32_t release_bar = 0u,
+                                              bool release_remote = false) {
+    if (bias != nullptr || act != 0 || rbase != nullptr)
+        return epilogue_tile_impl<T, BN, MAP3D, ACC2, true>(t_addr, my_stage, lane, base, ld, row, row0, nrows, cbase, ncols,
+                                                            tm, x0, y0, z0, tma, vec, alpha, beta, bias, act, rbase, ldr,
+                                                            rvec, cf, abort_flag, wait_cycles, t_addr2, release_bar,
+                                                            release_remote);
+    return epilogue_tile_impl<T, BN, MAP3D, ACC2, false>(t_addr, my_stage, lane, base, ld, row, row0, nrows, cbase, ncols, tm,
+                                                         x0, y0, z0, tma, vec, alpha, beta, nullptr, 0, nullptr, ldr, rvec,
+                                                         cf, abort_flag, wait_cycles, t_addr2, release_bar, release_remote);
 }
 
 // Epilogue of a tile computed with the operands exchanged (C^T = op(B)^T op(A)^T: the accumulator's rows are
