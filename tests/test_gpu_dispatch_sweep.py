@@ -1,5 +1,5 @@
 """The dispatcher's own choices over a few hundred seeded random problems -- skinny, few-tile, one-wave, multi-wave,
-long-K; every tensor-core type pair, layout, ragged sizes, alpha / beta -- checked over the WHOLE output against the
+long-K, short-K with large outputs; every tensor-core type pair, layout, ragged sizes, alpha / beta -- checked over the WHOLE output against the
 fp64 cross-check kernel (itself pinned to the oracle on small cases in test_gpu_parity.py) with the per-element bound
 of tests/parity.py.  Complements the hand-picked shapes of the other files: whatever kernel, tile width, k-split or
 cluster shape the rules pick for a shape nobody thought of must still be right."""
@@ -28,7 +28,10 @@ def draw(rng, cls):
         return int(rng.integers(1, 600)), int(rng.integers(1, 600)), int(rng.integers(1, 20000))
     if cls == 4:     # several waves
         return int(rng.integers(1000, 4200)), int(rng.integers(1000, 4200)), int(rng.integers(1000, 4200))
-    return int(rng.integers(1, 300)), int(rng.integers(2000, 30000)), int(rng.integers(1000, 5000))
+    if cls == 5:     # very wide, few rows
+        return int(rng.integers(1, 300)), int(rng.integers(2000, 30000)), int(rng.integers(1000, 5000))
+    # several waves of tiles with few k-blocks: the epilogue bounds the launch
+    return int(rng.integers(1500, 6000)), int(rng.integers(1500, 6000)), int(rng.integers(8, 700))
 
 
 @pytest.mark.parametrize("seed", [5, 6])
@@ -39,7 +42,7 @@ def test_dispatcher_choices_whole_matrix(seed):
     worst = 0.0
     while done < 160:
         dt = TYPES[int(rng.integers(len(TYPES)))]
-        M, N, K = draw(rng, int(rng.integers(6)))
+        M, N, K = draw(rng, int(rng.integers(7)))
         if dt == W.PEAK_F32_F32:
             M, N, K = min(M, 1500), min(N, 3000), min(K, 3000)      # the CUDA-core path is 20 times slower
         if 2.0 * M * N * K > 1.2e12:
