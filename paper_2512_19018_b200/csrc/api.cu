@@ -91,6 +91,16 @@ int choose_variant(const GemmArgs &g) {
     if ((tv == PEAK_VARIANT_UMMA_1CTA || tv == PEAK_VARIANT_UMMA_2CTA) && umma_supports(g, tv == PEAK_VARIANT_UMMA_2CTA ? 2 : 1) &&
         (tv == PEAK_VARIANT_UMMA_1CTA || g.M > 128))
         return tv;
+    // More than a wave of tiles with at most four k-blocks each (eight when the epilogue also reads C): the epilogue
+    // bounds the launch, and single-CTA tiles -- CTA-local barriers between the epilogue warps and the MMA issuer, two
+    // accumulator slots -- drain faster than pairs, whose smaller operand traffic buys nothing there (bf16, us, single /
+    // pair tiles / cuBLAS: 8192x8192x64 26.0 / 33.5 / 26.7, x128 29.1 / 36.6 / 31.8, x256 41.2 / 46.1 / 40.9;
+    // x512 72 / 63 with beta = 0 but 91 / 100 with beta = 1).
+    if (umma_supports(g, 1) && g.M > 128) {
+        const int64_t pair_tiles = ((g.M + 255) / 256) * ((g.N + 255) / 256) * g.nbatch();
+        const int64_t num_kb = (g.K + (is_fp8(in_elem(g.dtype)) ? 127 : 63)) / (is_fp8(in_elem(g.dtype)) ? 128 : 64);
+        if (pair_tiles > umma_units(2) && (num_kb <= 4 || (num_kb <= 8 && g.beta != 0.0f))) return PEAK_VARIANT_UMMA_1CTA;
+    }
     if (umma_supports(g, 2) && g.M > 128) {
         const int64_t pair_tiles = ((g.M + 255) / 256) * ((g.N + 255) / 256) * g.nbatch();
         if (2 * pair_tiles > umma_units(2) || !umma_supports(g, 1)) return PEAK_VARIANT_UMMA_2CTA;

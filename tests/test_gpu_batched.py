@@ -99,16 +99,16 @@ def test_batched_many_small_and_split(reset_tuning):
     b.check(exact=True, what="batch with k-split")
 
 
-def test_batched_short_k_wide_tiles(reset_tuning):
-    """Batches whose tiles have at most four k-blocks and fill more than a wave take the 512-wide tiles (eight epilogue
-    warps; the plain-store loop with beta = 0, the general one otherwise): exact on integers, ragged edges included;
-    narrow matrices that would leave half of a wide tile empty keep the 256-wide ones."""
-    for ta, tb, M, N, K, beta, wide in [(0, 1, 1024, 1024, 128, 0.0, True), (0, 0, 1000, 1016, 200, 0.0, True),
-                                        (1, 0, 1024, 1024, 64, 1.0, True), (0, 1, 256, 256, 128, 0.0, False)]:
-        b = Batch(mk(W.PEAK_BF16_BF16, ta, tb, M, N, K, alpha=0.5, beta=beta, dist="smallint"), batch=5 if M > 256 else 96,
+def test_batched_short_k_tiles(reset_tuning):
+    """Batches of more than a wave of tiles with at most four k-blocks (eight with beta != 0) take single-CTA
+    128 x 256 tiles (the plain-store loop with beta = 0, the general one otherwise): exact on integers, ragged edges
+    included."""
+    for ta, tb, M, N, K, beta in [(0, 1, 1024, 1024, 128, 0.0), (0, 0, 1000, 1016, 200, 0.0), (1, 0, 1024, 1024, 64, 1.0),
+                                  (0, 1, 256, 256, 128, 0.0), (1, 1, 520, 776, 448, -1.0)]:
+        b = Batch(mk(W.PEAK_BF16_BF16, ta, tb, M, N, K, alpha=0.5, beta=beta, dist="smallint"), batch=5 if M > 520 else 96,
                   gap=8)
         b.run()
-        assert ("umma_gemm_kernel<2, 512," in P.peak_last_kernel()) == wide, P.peak_last_kernel()
+        assert "umma_gemm_kernel<1, 256," in P.peak_last_kernel(), P.peak_last_kernel()
         b.check(exact=True, what=f"short-k batch {M}x{N}x{K} beta={beta}")
 
 

@@ -787,24 +787,29 @@ def test_cluster_k_real_values_fused_tail_and_selection(reset_tuning):
 
 def test_short_k_epilogue_bound_exact_and_selected(reset_tuning):
     """Problems of more than a wave whose tiles have few k-blocks are bounded by the epilogue: up to four k-blocks
-    they take the 512-wide tiles, up to eight the 256-wide kernel with eight epilogue warps.  beta = 0 runs the
+    (eight with beta != 0) they take single-CTA 128 x 256 tiles with eight epilogue warps; pair tiles forced onto
+    them take the 512-wide tile up to four k-blocks and eight epilogue warps up to eight.  beta = 0 runs the
     plain-store loop (ragged last chunk of a row, odd chunk counts, rows beyond M), beta != 0 and the fused tail the
     general one; exact on integers for 16-bit and 8-bit inputs and for a 32-bit output, bitwise repeatable."""
-    cases = [(0, 1, 2304, 2560, 64, W.PEAK_BF16_BF16, 0.0, "<2, 512,"), (0, 0, 2300, 2504, 200, W.PEAK_BF16_BF16, 0.0, "<2, 512,"),
-             (1, 0, 2304, 2568, 256, W.PEAK_F16_F32, 0.0, "<2, 512,"), (1, 1, 2200, 2560, 136, W.PEAK_BF16_BF16, -1.0, "<2, 512,"),
-             (0, 1, 2304, 2560, 512, W.PEAK_E4M3_BF16, 0.0, "<2, 512,"), (0, 1, 2304, 2560, 448, W.PEAK_BF16_BF16, 0.0, "0, 0, 1, 0>"),
-             (0, 0, 2304, 2600, 320, W.PEAK_F16_F16, 2.0, "0, 0, 1, 0>")]
-    for idx, (ta, tb, M, N, K, dtype, beta, tag) in enumerate(cases):
+    A, P2 = P.PEAK_VARIANT_AUTO, P.PEAK_VARIANT_UMMA_2CTA
+    cases = [(0, 1, 2304, 2560, 64, W.PEAK_BF16_BF16, 0.0, A, "<1, 256,"), (0, 0, 2300, 2504, 200, W.PEAK_BF16_BF16, 0.0, A, "0, 0, 1, 0>"),
+             (1, 0, 2304, 2568, 256, W.PEAK_F16_F32, 0.0, A, "<1, 256,"), (1, 1, 2200, 2560, 136, W.PEAK_BF16_BF16, -1.0, A, "<1, 256,"),
+             (0, 1, 2304, 2560, 512, W.PEAK_E4M3_BF16, 0.0, A, "<1, 256,"), (0, 0, 2304, 2600, 448, W.PEAK_F16_F16, 2.0, A, "<1, 256,"),
+             (0, 1, 2304, 2560, 64, W.PEAK_BF16_BF16, 0.0, P2, "<2, 512,"), (0, 0, 2300, 2504, 200, W.PEAK_BF16_BF16, 0.0, P2, "<2, 512,"),
+             (1, 0, 2304, 2568, 256, W.PEAK_F16_F32, 0.0, P2, "<2, 512,"), (0, 1, 2304, 2560, 512, W.PEAK_E4M3_BF16, 0.0, P2, "<2, 512,"),
+             (0, 1, 2304, 2560, 448, W.PEAK_BF16_BF16, 0.0, A, "<2, 256, __nv_bfloat16, 0, 0, 0, 1, 0>"),
+             (0, 0, 2304, 2600, 320, W.PEAK_F16_F16, 2.0, P2, "0, 0, 1, 0>")]
+    for idx, (ta, tb, M, N, K, dtype, beta, variant, tag) in enumerate(cases):
         unit = 16 if dtype == W.PEAK_E4M3_BF16 else 8
         pa, pb = (-(M if ta else K)) % unit, (-(K if tb else N)) % unit
         c = mk(dtype, ta, tb, M, N, K, dist="smallint", alpha=0.5, beta=beta, pad_a=pa, pad_b=pb, pad_c=[0, 8][idx % 2], case=idx)
         dc = R.DeviceCase(c)
-        dc.run(P.PEAK_VARIANT_AUTO)
+        dc.run(variant)
         assert "umma_gemm_kernel" in P.peak_last_kernel() and tag in P.peak_last_kernel(), P.peak_last_kernel()
         R.check_full(dc, what=f"short k {c}")
         first = dc.result().copy()
         dc.reset_c()
-        dc.run(P.PEAK_VARIANT_AUTO)
+        dc.run(variant)
         assert np.array_equal(first, dc.result())
     # real values with bias and GELU through the general loop of the same kernels
     from tests.test_gpu_fused import run_fused, check_fused
