@@ -308,7 +308,9 @@ int launch_kernel(const GemmArgs &g, const Plan &plan, int units_max, float *ws)
 // last tile's epilogue is an exposed tail of the launch (fp16 2048^3 -> fp32: see the A/B notes); on longer
 // runs the extra warps cost about 1 %.  16-bit inputs, single matrices.
 template <int BN> bool want_two_groups(const GemmArgs &g, const Plan &plan, int units) {
-    if (BN == 512 || g.nbatch() > 1 || is_fp8(in_elem(g.dtype))) return false;
+    if (BN == 512 || is_fp8(in_elem(g.dtype))) return false;
+    // batches: instantiated for the single-CTA 256-wide tiles of epilogue-bound problems only (launch_typed)
+    if (g.nbatch() > 1) return BN == 256 && plan.tail_splits == 1 && (g.K + BK - 1) / BK <= 8 && tuning(PEAK_TUNE_EPILOGUE_WARPS) != 1;
     const int mode = tuning(PEAK_TUNE_EPILOGUE_WARPS);  // 1 = four warps, 2 = eight warps
     if (mode) return mode == 2;
     // (also up to eight k-blocks, where the epilogue bounds every tile: 8192x8192x512 70 -> 64 us)
@@ -323,12 +325,20 @@ template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, 
             if (is_fp8(in_elem(g.dtype)))
                 return g.nbatch() > 1 ? launch_kernel<CG, BN, float, true, true>(g, plan, units, ws)
                                       : launch_kernel<CG, BN, float, false, true>(g, plan, units, ws);
-            if (g.nbatch() > 1) return launch_kernel<CG, BN, float, true>(g, plan, units, ws);
+            if (g.nbatch() > 1) {
+                if constexpr (CG == 1 && BN == 256)
+                    if (g2) return launch_kernel<CG, BN, float, true, false, true>(g, plan, units, ws);
+                return launch_kernel<CG, BN, float, true>(g, plan, units, ws);
+            }
             if constexpr (BN != 512)
                 if (g2) return launch_kernel<CG, BN, float, false, false, true>(g, plan, units, ws);
             return launch_kernel<CG, BN, float, false>(g, plan, units, ws);
         case Elem::F16:
-            if (g.nbatch() > 1) return launch_kernel<CG, BN, __half, true>(g, plan, units, ws);
+            if (g.nbatch() > 1) {
+                if constexpr (CG == 1 && BN == 256)
+                    if (g2) return launch_kernel<CG, BN, __half, true, false, true>(g, plan, units, ws);
+                return launch_kernel<CG, BN, __half, true>(g, plan, units, ws);
+            }
             if constexpr (BN != 512)
                 if (g2) return launch_kernel<CG, BN, __half, false, false, true>(g, plan, units, ws);
             return launch_kernel<CG, BN, __half, false>(g, plan, units, ws);
@@ -336,7 +346,11 @@ template <int CG, int BN> int launch_typed(const GemmArgs &g, const Plan &plan, 
             if (is_fp8(in_elem(g.dtype)))
                 return g.nbatch() > 1 ? launch_kernel<CG, BN, __nv_bfloat16, true, true>(g, plan, units, ws)
                                       : launch_kernel<CG, BN, __nv_bfloat16, false, true>(g, plan, units, ws);
-            if (g.nbatch() > 1) return launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws);
+            if (g.nbatch() > 1) {
+                if constexpr (CG == 1 && BN == 256)
+                    if (g2) return launch_kernel<CG, BN, __nv_bfloat16, true, false, true>(g, plan, units, ws);
+                return launch_kernel<CG, BN, __nv_bfloat16, true>(g, plan, units, ws);
+            }
             if constexpr (BN != 512)
                 if (g2) return launch_kernel<CG, BN, __nv_bfloat16, false, false, true>(g, plan, units, ws);
             return launch_kernel<CG, BN, __nv_bfloat16, false>(g, plan, units, ws);

@@ -108,7 +108,8 @@ def test_batched_short_k_tiles(reset_tuning):
         b = Batch(mk(W.PEAK_BF16_BF16, ta, tb, M, N, K, alpha=0.5, beta=beta, dist="smallint"), batch=5 if M > 520 else 96,
                   gap=8)
         b.run()
-        assert "umma_gemm_kernel<1, 256," in P.peak_last_kernel(), P.peak_last_kernel()
+        # single-CTA 256-wide tiles of a batch, eight epilogue warps (the last template flag but one)
+        assert "umma_gemm_kernel<1, 256," in P.peak_last_kernel() and ", 1, 0, 1, 0>" in P.peak_last_kernel(), P.peak_last_kernel()
         b.check(exact=True, what=f"short-k batch {M}x{N}x{K} beta={beta}")
 
 
