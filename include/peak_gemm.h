@@ -296,7 +296,8 @@ typedef enum peak_tuning_key {
                                      same number of waves */
     PEAK_TUNE_EPILOGUE_WARPS = 12, /* one-slot (128- / 256-wide) tiles: 1 = one group of four epilogue warps, 2 = two
                                       groups that drain half of the columns each (default: two for problems of at
-                                      most two waves) */
+                                      most two waves and for tiles of at most eight k-blocks; in a strided batch only
+                                      the single-CTA 256-wide tiles of such short-k problems have the second form) */
     PEAK_TUNE_K_ORDER = 13,     /* tensor-core kernels: 1 = every tile walks its k-blocks upwards, 2 = every other tile
                                    of a CTA walks them downwards, so that a wave of tiles starts in the k-range the
                                    previous wave left in L2 (default: 2 for 512-wide tiles, 1 otherwise) */
